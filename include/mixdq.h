@@ -1,0 +1,185 @@
+/*
+ * mixdq.h -- C ABI of the B200 (sm_100a) library for MixDQ's quantized inference path.
+ *
+ * The library runs the mixed-precision quantized linear and 3x3 convolution layers
+ * of a diffusion UNet: every layer carries its own weight width (3, 4 or 8 bits) and
+ * activation width (8 or 16 bits).  The bit-width table itself is an input: the
+ * paper's sensitivity analysis and integer program (Sec. 3.2, 3.3) run offline.
+ *
+ * Conventions shared by every call
+ *   - Return value: 0 on success, a negative MIXDQ_ERR_* code otherwise.  Argument
+ *     errors are found on the host before anything is launched.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the
+ *     caller.  The library allocates and frees no memory that the caller sees.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it and
+ *     never synchronize.
+ *   - fp16 tensors are IEEE binary16, row-major, densely packed unless a stride is given.
+ *   - Weight matrices are [N, K]: N output channels, K reduction length.  A 3x3 conv
+ *     weight is passed flattened to [N, 9*Cin] in (kh, kw, cin) order.
+ *   - `status` (optional, may be NULL) is a device int32 word.  A kernel whose bounded
+ *     wait on a barrier runs out writes a non-zero code there and returns early; the
+ *     host reads it after synchronizing.  A correct run leaves it untouched.
+ *
+ * Quantizer (paper Sec. 4.1 "Quantization Scheme": min-max uniform quantization with one
+ * scale / zero-point per activation tensor and one per weight output channel):
+ *   inv = fp32(1 / scale); code = clamp(round_half_even(v * inv) [+ zero]);
+ *   symmetric codes lie in [-qmax, qmax], qmax = 2^(b-1) - 1, asymmetric ones in [0, 2^b - 1].
+ */
+#ifndef MIXDQ_H_
+#define MIXDQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MIXDQ_OK 0
+#define MIXDQ_ERR_INVALID_ARG (-1) /* NULL pointer, non-positive size, bad enum */
+#define MIXDQ_ERR_UNSUPPORTED (-2) /* a width / shape combination the library does not run */
+#define MIXDQ_ERR_ALIGNMENT (-3)   /* pointer or stride not aligned as documented */
+#define MIXDQ_ERR_WORKSPACE (-4)   /* workspace missing or too small */
+#define MIXDQ_ERR_CUDA (-5)        /* a CUDA runtime / driver call failed */
+#define MIXDQ_ERR_TIMEOUT (-6)     /* written to `status` by a kernel whose wait ran out */
+
+#define MIXDQ_LAYOUT_CANONICAL 0 /* documented, engine-independent byte layout */
+#define MIXDQ_LAYOUT_DEVICE 1    /* layout the GEMM / conv kernels read */
+
+#define MIXDQ_TOKENS_PER_PROMPT 77 /* text tokens per prompt; token 0 is BOS (Sec. 3.1) */
+
+/* Library version as major*10000 + minor*100 + patch. */
+int mixdq_version(void);
+
+/* Static, NUL-terminated description of an error code (host pointer, never NULL). */
+const char* mixdq_strerror(int code);
+
+/*
+ * Bytes of a packed [N, K] weight matrix.  `out` is a HOST pointer.
+ * Canonical layout: row pitch K (8-bit), ceil(K/2) (4-bit, even k in the low nibble),
+ * ceil(K/32)*12 (3-bit: per group of 32 codes three little-endian u32 bit-planes, bit j of
+ * plane p = bit p of code 32g+j; a ragged last group is padded with the row's zero-point).
+ * Device layout: 8-bit rows padded to a multiple of 16 bytes; 4-bit rows padded to a
+ * multiple of 32 codes with, inside every group of 8 codes, byte j holding code j in the
+ * low nibble and code j+4 in the high nibble; 3-bit rows padded to a multiple of 128
+ * codes, each block of 128 codes stored as three 16-byte bit-planes.
+ */
+int mixdq_packed_bytes(int64_t N, int64_t K, int bits, int layout, size_t* out);
+
+/*
+ * Per-output-channel min-max parameters of W (fp16 [N, K]) -- Sec. 4.1.
+ * symmetric != 0: scale[n] = max_k |w| / qmax, zero[n] = 0.
+ * symmetric == 0: lo = min(min_k w, 0), hi = max(max_k w, 0), L = 2^bits - 1,
+ *                 scale[n] = (hi - lo) / L, zero[n] = clamp(rne(-lo * inv), 0, L).
+ * A constant-zero row gets scale 1.  `zero_out` may be NULL when symmetric.
+ */
+int mixdq_weight_minmax_params(const void* W, int64_t N, int64_t K, int bits, int symmetric,
+                               float* scale_out, int32_t* zero_out, void* stream);
+
+/*
+ * Quantize W (fp16 [N, K]) with the given per-channel scale (and zero-point) and pack the
+ * codes.  bits in {3, 4, 8}.  zero == NULL selects symmetric signed codes (not available
+ * for 3 bits).  `packed_out` must hold mixdq_packed_bytes(N, K, bits, layout) bytes and be
+ * 16-byte aligned.  This is the offline step of the path: it runs once per layer.
+ */
+int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits, const float* scale,
+                       const int32_t* zero, int layout, void* packed_out, void* stream);
+
+/*
+ * Parity hook: integer codes (int16 [N, K]) back out of a packed buffer in either layout.
+ * is_signed tells how 4- and 8-bit fields are read.
+ */
+int mixdq_unpack_weights(const void* packed, int64_t N, int64_t K, int bits, int is_signed,
+                         int layout, int16_t* codes_out, void* stream);
+
+/*
+ * max |x| over an fp16 matrix [rows, cols] with row stride `row_stride` elements, written to
+ * amax_out[0] (fp32).  skip_rows_mod > 0 leaves out every row whose index is a multiple of
+ * it: 77 removes the BOS token of every prompt from the range (Sec. 3.1).
+ */
+int mixdq_act_absmax(const void* X, int64_t rows, int64_t cols, int64_t row_stride,
+                     int skip_rows_mod, float* amax_out, void* stream);
+
+/* scale_out[0] = amax[0] / 127 (one fp32 division; 1 when amax is 0): the per-tensor
+ * symmetric int8 activation scale of Sec. 4.1 computed on the device. */
+int mixdq_act_scale_from_absmax(const float* amax, float* scale_out, void* stream);
+
+/*
+ * Bytes of scratch memory the layer calls below need for a given problem (HOST `out`).
+ * rows = output rows (tokens or output pixels), N, K as in the layer call.  The scratch
+ * must be 256-byte aligned and zero-filled once before its first use; the kernels leave
+ * it zero-filled again.  Calls that share a workspace must not overlap on the GPU.
+ * A result of 0 means the call runs without scratch (workspace may then be NULL).
+ */
+int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_bits, int act_bits,
+                          size_t* out);
+
+/*
+ * Quantized linear layer  Y[M, N] = X[M, K] * dequant(W)^T + bias   (paper Sec. 4.1, 4.3).
+ *   act_bits == 8 : W8A8 / W4A8.  X is quantized per tensor with *act_scale (device fp32)
+ *                   inside the kernel, multiplied with the integer weight codes in int32
+ *                   and dequantized as  y = fp16(acc * act_scale * w_scale[n] + bias[n]).
+ *                   Weights must be symmetric (w_zero == NULL), w_bits in {4, 8}.
+ *   act_bits == 16: weight-only W3/W4/W8-A16 (Table 1 "weight only" rows): X stays fp16,
+ *                   y = fp16(w_scale[n] * sum_k x[k] * (q[n,k] - w_zero[n]) + bias[n]).
+ *                   act_scale is ignored.  w_zero == NULL means signed codes, zero-point 0.
+ * packed_W is in MIXDQ_LAYOUT_DEVICE.  ldx is the row stride of X in elements (>= K,
+ * multiple of 8).  bias (fp16 [N]) may be NULL.  Y is dense [M, N].  X, Y 16-byte aligned.
+ */
+int mixdq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
+                 int w_bits, const float* w_scale, const int32_t* w_zero, int act_bits,
+                 const float* act_scale, const void* bias, void* Y, void* workspace,
+                 size_t workspace_bytes, int32_t* status, void* stream);
+
+/* Parity hook of the int8 path: the raw int32 accumulators acc[M, N] = sum_k qx * qw that
+ * mixdq_linear(act_bits = 8) would dequantize. */
+int mixdq_linear_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
+                         int64_t N, int w_bits, const float* act_scale, int32_t* acc_out,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * Quantized 3x3 convolution as an implicit GEMM (all linear and conv layers are quantized,
+ * Sec. 4.1 "Mixed Precision Allocation").  X fp16 NHWC [B, H, W, Cin], zero padding 1,
+ * stride in {1, 2}; packed_W is the [Cout, 9*Cin] matrix in (kh, kw, cin) order; Y fp16 NHWC
+ * [B, Ho, Wo, Cout] with Ho = (H - 1) / stride + 1.  Width arguments as in mixdq_linear.
+ */
+int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                  int64_t Cout, int stride, int w_bits, const float* w_scale, const int32_t* w_zero,
+                  int act_bits, const float* act_scale, const void* bias, void* Y, void* workspace,
+                  size_t workspace_bytes, int32_t* status, void* stream);
+
+/* Parity hook: int32 accumulators [B, Ho, Wo, Cout] of the int8 conv path. */
+int mixdq_conv3x3_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                          const void* packed_W, int64_t Cout, int stride, int w_bits,
+                          const float* act_scale, int32_t* acc_out, void* workspace,
+                          size_t workspace_bytes, int32_t* status, void* stream);
+
+/* 1x1 convolution on NHWC = mixdq_linear on the [B*H*W, Cin] pixel matrix. */
+int mixdq_conv1x1(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                  int64_t Cout, int w_bits, const float* w_scale, const int32_t* w_zero, int act_bits,
+                  const float* act_scale, const void* bias, void* Y, void* workspace,
+                  size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * BOS-aware cross-attention K or V projection (Sec. 3.1).  text_emb fp16 [B, 77, Kt].
+ * Token 0 of every prompt takes no part in the computation: Y[b, 0, :] is a bit-for-bit
+ * copy of bos_out (fp16 [N], the floating-point projection of the BOS embedding computed
+ * ahead of time), rows 1..76 run the W8A8 / W4A8 path with *act_scale (whose range the
+ * caller takes over tokens 1..76 only, e.g. mixdq_act_absmax with skip_rows_mod = 77).
+ * Y fp16 [B, 77, N].  No bias (to_k / to_v have none).
+ */
+int mixdq_crossattn_kv(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W, int64_t N,
+                       int w_bits, const float* w_scale, const float* act_scale,
+                       const void* bos_out, void* Y, void* workspace, size_t workspace_bytes,
+                       int32_t* status, void* stream);
+
+/* Parity hook: int32 accumulators [B, 76, N] of the rows the int8 path computes. */
+int mixdq_crossattn_kv_acc_i32(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W,
+                               int64_t N, int w_bits, const float* act_scale, int32_t* acc_out,
+                               void* workspace, size_t workspace_bytes, int32_t* status,
+                               void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXDQ_H_ */
