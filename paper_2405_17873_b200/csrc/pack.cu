@@ -1,0 +1,290 @@
+// Offline side of the path: per-channel min-max parameters, weight quantization and
+// packing (3 / 4 / 8 bits, canonical and device layouts), the unpack parity hook, and the
+// per-tensor activation range helpers.  None of this is on the per-step hot path, so the
+// kernels favour exactness (products in double, one IEEE divide per scale) over speed.
+#include "common.cuh"
+
+namespace mixdq {
+
+namespace {
+
+// round-half-even of the exact product w * inv (11-bit x 24-bit significands fit a double)
+__device__ __forceinline__ long long rne_product(float w, float inv)
+{
+    double p = static_cast<double>(w) * static_cast<double>(inv);
+    p = fmin(fmax(p, -1e15), 1e15);
+    return __double2ll_rn(p);
+}
+
+__device__ __forceinline__ int clampi(long long v, int lo, int hi)
+{
+    return v < lo ? lo : (v > hi ? hi : static_cast<int>(v));
+}
+
+// One block per output channel: min / max of the row, then scale and zero-point.
+__global__ void weight_minmax_kernel(const __half* __restrict__ W, int64_t K, int bits, int symmetric,
+                                     float* __restrict__ scale_out, int32_t* __restrict__ zero_out)
+{
+    const int64_t n = blockIdx.x;
+    const __half* row = W + n * K;
+    float lo = 0.f, hi = 0.f;
+    for (int64_t k = threadIdx.x; k < K; k += blockDim.x) {
+        float w = __half2float(row[k]);
+        lo = fminf(lo, w);
+        hi = fmaxf(hi, w);
+    }
+    __shared__ float s_lo[32], s_hi[32];
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        s_lo[threadIdx.x >> 5] = lo;
+        s_hi[threadIdx.x >> 5] = hi;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        for (int i = 1; i < nw; ++i) {
+            lo = fminf(lo, s_lo[i]);
+            hi = fmaxf(hi, s_hi[i]);
+        }
+        if (symmetric) {
+            const float amax = fmaxf(-lo, hi);
+            const float qmax = static_cast<float>((1 << (bits - 1)) - 1);
+            scale_out[n] = (amax == 0.f) ? 1.f : __fdiv_rn(amax, qmax);
+            if (zero_out) zero_out[n] = 0;
+        } else {
+            const int L = (1 << bits) - 1;
+            const float range = __fsub_rn(hi, lo);
+            const float scale = (range == 0.f) ? 1.f : __fdiv_rn(range, static_cast<float>(L));
+            scale_out[n] = scale;
+            if (zero_out) zero_out[n] = clampi(rne_product(-lo, __fdiv_rn(1.f, scale)), 0, L);
+        }
+    }
+}
+
+// Code of element (n, k); positions beyond K hold the pad code (0 signed, zero-point unsigned).
+__device__ __forceinline__ int code_at(const __half* __restrict__ W, int64_t n, int64_t k, int64_t K,
+                                       int bits, float inv, bool has_zero, int z)
+{
+    if (k >= K) return has_zero ? z : 0;
+    const long long r = rne_product(__half2float(W[n * K + k]), inv);
+    if (has_zero) return clampi(r + z, 0, (1 << bits) - 1);
+    const int qmax = (1 << (bits - 1)) - 1;
+    return clampi(r, -qmax, qmax);
+}
+
+// One thread per 32-bit output word of a packed row.
+__global__ void pack_kernel(const __half* __restrict__ W, int64_t N, int64_t K, int bits,
+                            const float* __restrict__ scale, const int32_t* __restrict__ zero,
+                            int layout, int64_t pitch, uint8_t* __restrict__ out)
+{
+    const int64_t words_per_row = (pitch + 3) / 4;
+    const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (idx >= N * words_per_row) return;
+    const int64_t n = idx / words_per_row;
+    const int64_t w = idx - n * words_per_row;
+    const float inv = __fdiv_rn(1.f, scale[n]);
+    const bool hz = zero != nullptr;
+    const int z = hz ? zero[n] : 0;
+    uint8_t* row = out + n * pitch;
+    uint32_t word = 0;
+
+    if (bits == 8) {
+        for (int j = 0; j < 4; ++j)
+            word |= static_cast<uint32_t>(code_at(W, n, 4 * w + j, K, 8, inv, hz, z) & 0xff) << (8 * j);
+    } else if (bits == 4) {
+        if (layout == MIXDQ_LAYOUT_CANONICAL) {
+            // an odd K leaves the last high nibble empty (0) in the canonical layout
+            for (int j = 0; j < 8; ++j)
+                if (8 * w + j < K)
+                    word |= static_cast<uint32_t>(code_at(W, n, 8 * w + j, K, 4, inv, hz, z) & 0xf)
+                            << (4 * j);
+        } else {
+            // byte j of the word: code j in the low nibble, code j + 4 in the high nibble
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t lo = code_at(W, n, 8 * w + j, K, 4, inv, hz, z) & 0xf;
+                const uint32_t hi = code_at(W, n, 8 * w + 4 + j, K, 4, inv, hz, z) & 0xf;
+                word |= (lo | (hi << 4)) << (8 * j);
+            }
+        }
+    } else {  // 3-bit planes
+        int64_t k0;
+        int plane;
+        if (layout == MIXDQ_LAYOUT_CANONICAL) {
+            k0 = 32 * (w / 3);  // group g: words 3g .. 3g+2 are planes 0..2
+            plane = static_cast<int>(w % 3);
+        } else {
+            const int64_t blk = w / 12;  // block of 128 codes: 4 words per plane, planes in order
+            const int r = static_cast<int>(w % 12);
+            plane = r / 4;
+            k0 = 128 * blk + 32 * (r % 4);
+        }
+        for (int j = 0; j < 32; ++j)
+            word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << j;
+    }
+    // the last word of an odd-sized canonical row may be partial
+    const int64_t byte0 = 4 * w;
+    for (int b = 0; b < 4 && byte0 + b < pitch; ++b) row[byte0 + b] = (word >> (8 * b)) & 0xff;
+}
+
+// One thread per code.
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, int64_t N, int64_t K, int bits,
+                              int is_signed, int layout, int64_t pitch, int16_t* __restrict__ codes)
+{
+    const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (idx >= N * K) return;
+    const int64_t n = idx / K;
+    const int64_t k = idx - n * K;
+    const uint8_t* row = packed + n * pitch;
+    int c;
+    if (bits == 8) {
+        c = is_signed ? static_cast<int>(static_cast<int8_t>(row[k])) : static_cast<int>(row[k]);
+    } else if (bits == 4) {
+        int nib;
+        if (layout == MIXDQ_LAYOUT_CANONICAL) {
+            nib = (k & 1) ? (row[k >> 1] >> 4) : (row[k >> 1] & 0xf);
+        } else {
+            const int64_t g = k >> 3;
+            const int j = static_cast<int>(k & 7);
+            const uint8_t b = row[4 * g + (j & 3)];
+            nib = (j >= 4) ? (b >> 4) : (b & 0xf);
+        }
+        c = (is_signed && nib >= 8) ? nib - 16 : nib;
+    } else {
+        c = 0;
+        for (int p = 0; p < 3; ++p) {
+            int64_t byte;
+            if (layout == MIXDQ_LAYOUT_CANONICAL) {
+                byte = (k / 32) * 12 + p * 4 + ((k % 32) >> 3);
+            } else {
+                const int64_t blk = k / 128;
+                const int r = static_cast<int>(k % 128);
+                byte = blk * 48 + p * 16 + (r >> 5) * 4 + ((r & 31) >> 3);
+            }
+            c |= ((row[byte] >> (k & 7)) & 1) << p;
+        }
+    }
+    codes[idx] = static_cast<int16_t>(c);
+}
+
+// max |x| as an atomic max on the bit pattern (non-negative floats order like integers).
+__global__ void absmax_kernel(const __half* __restrict__ X, int64_t rows, int64_t cols,
+                              int64_t row_stride, int skip_mod, unsigned int* __restrict__ amax_bits)
+{
+    float m = 0.f;
+    const int64_t chunks_per_row = (cols + 7) / 8;
+    const int64_t total = rows * chunks_per_row;
+    const bool vec_ok = (cols % 8 == 0) && (row_stride % 8 == 0) &&
+                        ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / chunks_per_row;
+        const int64_t c = (i - r * chunks_per_row) * 8;
+        if (skip_mod > 0 && r % skip_mod == 0) continue;
+        const __half* p = X + r * row_stride + c;
+        if (vec_ok) {
+            const uint4 v = *reinterpret_cast<const uint4*>(p);
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __half22float2(h[j]);
+                m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+            }
+        } else {
+            for (int j = 0; j < 8 && c + j < cols; ++j) m = fmaxf(m, fabsf(__half2float(p[j])));
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(amax_bits, __float_as_uint(m));
+}
+
+__global__ void act_scale_kernel(const float* __restrict__ amax, float* __restrict__ scale_out)
+{
+    const float a = amax[0];
+    scale_out[0] = (a == 0.f) ? 1.f : __fdiv_rn(a, 127.f);
+}
+
+bool width_ok(int bits) { return bits == 3 || bits == 4 || bits == 8; }
+
+}  // namespace
+
+}  // namespace mixdq
+
+using namespace mixdq;
+
+extern "C" int mixdq_packed_bytes(int64_t N, int64_t K, int bits, int layout, size_t* out)
+{
+    if (!out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (layout != MIXDQ_LAYOUT_CANONICAL && layout != MIXDQ_LAYOUT_DEVICE) return MIXDQ_ERR_INVALID_ARG;
+    if (!width_ok(bits)) return MIXDQ_ERR_UNSUPPORTED;
+    if (layout == MIXDQ_LAYOUT_CANONICAL) {
+        *out = static_cast<size_t>(N * row_pitch_bytes(K, bits, layout));
+    } else {
+        // device buffers are read in whole 16-byte units
+        *out = static_cast<size_t>(round_up(N * row_pitch_bytes(K, bits, layout), 16));
+    }
+    return MIXDQ_OK;
+}
+
+extern "C" int mixdq_weight_minmax_params(const void* W, int64_t N, int64_t K, int bits, int symmetric,
+                                          float* scale_out, int32_t* zero_out, void* stream)
+{
+    if (!W || !scale_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (!symmetric && !zero_out) return MIXDQ_ERR_INVALID_ARG;
+    weight_minmax_kernel<<<static_cast<unsigned>(N), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(W), K, bits, symmetric, scale_out, zero_out);
+    return check_launch();
+}
+
+extern "C" int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits, const float* scale,
+                                  const int32_t* zero, int layout, void* packed_out, void* stream)
+{
+    if (!W || !scale || !packed_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (layout != MIXDQ_LAYOUT_CANONICAL && layout != MIXDQ_LAYOUT_DEVICE) return MIXDQ_ERR_INVALID_ARG;
+    if (!width_ok(bits)) return MIXDQ_ERR_UNSUPPORTED;
+    if (bits == 3 && !zero) return MIXDQ_ERR_UNSUPPORTED;  // 3-bit codes are unsigned only
+    if (reinterpret_cast<uintptr_t>(packed_out) & 15) return MIXDQ_ERR_ALIGNMENT;
+    const int64_t pitch = row_pitch_bytes(K, bits, layout);
+    const int64_t words = N * ((pitch + 3) / 4);
+    pack_kernel<<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(W), N, K, bits, scale, zero, layout, pitch,
+        static_cast<uint8_t*>(packed_out));
+    return check_launch();
+}
+
+extern "C" int mixdq_unpack_weights(const void* packed, int64_t N, int64_t K, int bits, int is_signed,
+                                    int layout, int16_t* codes_out, void* stream)
+{
+    if (!packed || !codes_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (layout != MIXDQ_LAYOUT_CANONICAL && layout != MIXDQ_LAYOUT_DEVICE) return MIXDQ_ERR_INVALID_ARG;
+    if (!width_ok(bits)) return MIXDQ_ERR_UNSUPPORTED;
+    if (bits == 3 && is_signed) return MIXDQ_ERR_UNSUPPORTED;
+    const int64_t pitch = row_pitch_bytes(K, bits, layout);
+    unpack_kernel<<<static_cast<unsigned>(ceil_div(N * K, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(packed), N, K, bits, is_signed, layout, pitch, codes_out);
+    return check_launch();
+}
+
+extern "C" int mixdq_act_absmax(const void* X, int64_t rows, int64_t cols, int64_t row_stride,
+                                int skip_rows_mod, float* amax_out, void* stream)
+{
+    if (!X || !amax_out || rows <= 0 || cols <= 0 || row_stride < cols || skip_rows_mod < 0)
+        return MIXDQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MIXDQ_CUDA_TRY(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
+    const int64_t chunks = rows * ((cols + 7) / 8);
+    const unsigned grid = static_cast<unsigned>(chunks < 256 * 1184 ? ceil_div(chunks, 256) : 1184);
+    absmax_kernel<<<grid, 256, 0, st>>>(static_cast<const __half*>(X), rows, cols, row_stride,
+                                        skip_rows_mod, reinterpret_cast<unsigned int*>(amax_out));
+    return check_launch();
+}
+
+extern "C" int mixdq_act_scale_from_absmax(const float* amax, float* scale_out, void* stream)
+{
+    if (!amax || !scale_out) return MIXDQ_ERR_INVALID_ARG;
+    act_scale_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(amax, scale_out);
+    return check_launch();
+}
