@@ -62,7 +62,8 @@ const char* mixdq_strerror(int code);
  * Device layout: 8-bit rows padded to a multiple of 16 bytes; 4-bit rows padded to a
  * multiple of 32 codes with, inside every group of 8 codes, byte j holding code j in the
  * low nibble and code j+4 in the high nibble; 3-bit rows padded to a multiple of 128
- * codes, each block of 128 codes stored as three 16-byte bit-planes.
+ * codes, each block of 128 codes stored as three 16-byte bit-planes whose bits are
+ * interleaved for the register decode (mixdq_unpack_weights undoes it).
  */
 int mixdq_packed_bytes(int64_t N, int64_t K, int bits, int layout, size_t* out);
 

@@ -1,0 +1,255 @@
+// C ABI: argument validation and dispatch to the int8 and weight-only engines.
+#include "common.cuh"
+#include "engines.h"
+
+using namespace mixdq;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_widths(int w_bits, int act_bits, const int32_t* w_zero)
+{
+    if (act_bits == 8) {
+        if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+        if (w_zero) return MIXDQ_ERR_UNSUPPORTED;  // the int8 path takes symmetric weights
+        return MIXDQ_OK;
+    }
+    if (act_bits == 16) {
+        if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+        if (w_bits == 3 && !w_zero) return MIXDQ_ERR_UNSUPPORTED;
+        return MIXDQ_OK;
+    }
+    return MIXDQ_ERR_UNSUPPORTED;
+}
+
+bool fits_int(int64_t v) { return v > 0 && v <= 0x7fffffff; }
+
+int linear_impl(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
+                int w_bits, const float* w_scale, const int32_t* w_zero, int act_bits,
+                const float* act_scale, const void* bias, void* Y, int32_t* acc_out, void* workspace,
+                size_t ws_bytes, int32_t* status, void* stream)
+{
+    if (!X || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(M) || !fits_int(K) || !fits_int(N) || ldx < K) return MIXDQ_ERR_INVALID_ARG;
+    if (Y && !w_scale) return MIXDQ_ERR_INVALID_ARG;
+    int rc = check_widths(w_bits, act_bits, w_zero);
+    if (rc != MIXDQ_OK) return rc;
+    if (!aligned16(packed_W)) return MIXDQ_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (act_bits == 8) {
+        if (!act_scale) return MIXDQ_ERR_INVALID_ARG;
+        i8::Params p;
+        p.X = static_cast<const __half*>(X);
+        p.ldx = ldx;
+        p.M = static_cast<int>(M);
+        p.N = static_cast<int>(N);
+        p.K = static_cast<int>(K);
+        p.act_scale = act_scale;
+        p.w_scale = w_scale;
+        p.bias = static_cast<const __half*>(bias);
+        p.Y = static_cast<__half*>(Y);
+        p.ldy = N;
+        p.acc_out = acc_out;
+        p.status = status;
+        return i8::run(p, A_LINEAR, packed_W, w_bits, workspace, ws_bytes, st);
+    }
+    if (acc_out) return MIXDQ_ERR_UNSUPPORTED;
+    wo::Params p;
+    p.X = static_cast<const __half*>(X);
+    p.ldx = ldx;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.w_scale = w_scale;
+    p.w_zero = w_zero;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = N;
+    p.status = status;
+    return wo::run(p, A_LINEAR, packed_W, w_bits, st);
+}
+
+int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+               int64_t Cout, int stride, int w_bits, const float* w_scale, const int32_t* w_zero,
+               int act_bits, const float* act_scale, const void* bias, void* Y, int32_t* acc_out,
+               void* workspace, size_t ws_bytes, int32_t* status, void* stream)
+{
+    if (!X || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(B) || !fits_int(H) || !fits_int(W) || !fits_int(Cin) || !fits_int(Cout))
+        return MIXDQ_ERR_INVALID_ARG;
+    if (stride != 1 && stride != 2) return MIXDQ_ERR_INVALID_ARG;
+    if (Y && !w_scale) return MIXDQ_ERR_INVALID_ARG;
+    int rc = check_widths(w_bits, act_bits, w_zero);
+    if (rc != MIXDQ_OK) return rc;
+    if (!aligned16(packed_W)) return MIXDQ_ERR_ALIGNMENT;
+    const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    if (!fits_int(B * Ho * Wo) || !fits_int(9 * Cin) || !fits_int(B * H * W * Cin)) return MIXDQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (act_bits == 8) {
+        if (!act_scale) return MIXDQ_ERR_INVALID_ARG;
+        i8::Params p;
+        p.X = static_cast<const __half*>(X);
+        p.ldx = 8;  // unused by the gather; keeps the alignment test of the dispatcher neutral
+        p.M = static_cast<int>(B * Ho * Wo);
+        p.N = static_cast<int>(Cout);
+        p.K = static_cast<int>(9 * Cin);
+        p.H = static_cast<int>(H);
+        p.W = static_cast<int>(W);
+        p.Cin = static_cast<int>(Cin);
+        p.Ho = static_cast<int>(Ho);
+        p.Wo = static_cast<int>(Wo);
+        p.stride = stride;
+        p.act_scale = act_scale;
+        p.w_scale = w_scale;
+        p.bias = static_cast<const __half*>(bias);
+        p.Y = static_cast<__half*>(Y);
+        p.ldy = Cout;
+        p.acc_out = acc_out;
+        p.status = status;
+        return i8::run(p, A_CONV3, packed_W, w_bits, workspace, ws_bytes, st);
+    }
+    if (acc_out) return MIXDQ_ERR_UNSUPPORTED;
+    wo::Params p;
+    p.X = static_cast<const __half*>(X);
+    p.ldx = 8;
+    p.M = static_cast<int>(B * Ho * Wo);
+    p.N = static_cast<int>(Cout);
+    p.K = static_cast<int>(9 * Cin);
+    p.H = static_cast<int>(H);
+    p.W = static_cast<int>(W);
+    p.Cin = static_cast<int>(Cin);
+    p.Ho = static_cast<int>(Ho);
+    p.Wo = static_cast<int>(Wo);
+    p.stride = stride;
+    p.w_scale = w_scale;
+    p.w_zero = w_zero;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = Cout;
+    p.status = status;
+    return wo::run(p, A_CONV3, packed_W, w_bits, st);
+}
+
+int kv_impl(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W, int64_t N, int w_bits,
+            const float* w_scale, const float* act_scale, const void* bos_out, void* Y, int32_t* acc_out,
+            void* workspace, size_t ws_bytes, int32_t* status, void* stream)
+{
+    if (!text_emb || !packed_W || !act_scale || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (Y && (!w_scale || !bos_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(B) || !fits_int(Kt) || !fits_int(N) || !fits_int(B * MIXDQ_TOKENS_PER_PROMPT))
+        return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (!aligned16(packed_W)) return MIXDQ_ERR_ALIGNMENT;
+    i8::Params p;
+    p.X = static_cast<const __half*>(text_emb);
+    p.ldx = Kt;
+    p.M = static_cast<int>(B * (MIXDQ_TOKENS_PER_PROMPT - 1));
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(Kt);
+    p.batch = static_cast<int>(B);
+    p.act_scale = act_scale;
+    p.w_scale = w_scale;
+    p.bos_out = static_cast<const __half*>(bos_out);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = N;
+    p.acc_out = acc_out;
+    p.status = status;
+    return i8::run(p, A_BOS, packed_W, w_bits, workspace, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+
+extern "C" int mixdq_version(void) { return 100; }
+
+extern "C" const char* mixdq_strerror(int code)
+{
+    switch (code) {
+        case MIXDQ_OK: return "success";
+        case MIXDQ_ERR_INVALID_ARG: return "invalid argument";
+        case MIXDQ_ERR_UNSUPPORTED: return "unsupported bit-width or shape";
+        case MIXDQ_ERR_ALIGNMENT: return "misaligned pointer or stride";
+        case MIXDQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case MIXDQ_ERR_CUDA: return "CUDA call failed";
+        case MIXDQ_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_bits, int act_bits, size_t* out)
+{
+    if (!out || rows <= 0 || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    *out = (act_bits == 8) ? i8::workspace_bytes(rows, N) : 0;
+    return MIXDQ_OK;
+}
+
+extern "C" int mixdq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
+                            int w_bits, const float* w_scale, const int32_t* w_zero, int act_bits,
+                            const float* act_scale, const void* bias, void* Y, void* workspace,
+                            size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return linear_impl(X, M, K, ldx, packed_W, N, w_bits, w_scale, w_zero, act_bits, act_scale, bias, Y,
+                       nullptr, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_linear_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
+                                    int64_t N, int w_bits, const float* act_scale, int32_t* acc_out,
+                                    void* workspace, size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!acc_out) return MIXDQ_ERR_INVALID_ARG;
+    return linear_impl(X, M, K, ldx, packed_W, N, w_bits, nullptr, nullptr, 8, act_scale, nullptr, nullptr,
+                       acc_out, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                             int64_t Cout, int stride, int w_bits, const float* w_scale,
+                             const int32_t* w_zero, int act_bits, const float* act_scale, const void* bias,
+                             void* Y, void* workspace, size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return conv3_impl(X, B, H, W, Cin, packed_W, Cout, stride, w_bits, w_scale, w_zero, act_bits, act_scale,
+                      bias, Y, nullptr, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_conv3x3_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                                     const void* packed_W, int64_t Cout, int stride, int w_bits,
+                                     const float* act_scale, int32_t* acc_out, void* workspace,
+                                     size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!acc_out) return MIXDQ_ERR_INVALID_ARG;
+    return conv3_impl(X, B, H, W, Cin, packed_W, Cout, stride, w_bits, nullptr, nullptr, 8, act_scale, nullptr,
+                      nullptr, acc_out, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_conv1x1(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                             int64_t Cout, int w_bits, const float* w_scale, const int32_t* w_zero,
+                             int act_bits, const float* act_scale, const void* bias, void* Y, void* workspace,
+                             size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (B <= 0 || H <= 0 || W <= 0) return MIXDQ_ERR_INVALID_ARG;
+    return mixdq_linear(X, B * H * W, Cin, Cin, packed_W, Cout, w_bits, w_scale, w_zero, act_bits, act_scale,
+                        bias, Y, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_crossattn_kv(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W, int64_t N,
+                                  int w_bits, const float* w_scale, const float* act_scale,
+                                  const void* bos_out, void* Y, void* workspace, size_t workspace_bytes,
+                                  int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return kv_impl(text_emb, B, Kt, packed_W, N, w_bits, w_scale, act_scale, bos_out, Y, nullptr, workspace,
+                   workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_crossattn_kv_acc_i32(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W,
+                                          int64_t N, int w_bits, const float* act_scale, int32_t* acc_out,
+                                          void* workspace, size_t workspace_bytes, int32_t* status,
+                                          void* stream)
+{
+    if (!acc_out) return MIXDQ_ERR_INVALID_ARG;
+    return kv_impl(text_emb, B, Kt, packed_W, N, w_bits, nullptr, act_scale, nullptr, nullptr, acc_out,
+                   workspace, workspace_bytes, status, stream);
+}

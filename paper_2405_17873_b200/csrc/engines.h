@@ -1,0 +1,64 @@
+// Internal interface between the C ABI (api.cu) and the two engines.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace mixdq {
+
+// How the rows of the A operand are found in memory.
+enum : int {
+    A_LINEAR = 0,  // row m of a [M, K] matrix with row stride ldx
+    A_BOS = 1,     // row m = (prompt, token - 1): token 0 of every 77-token prompt is skipped
+    A_CONV3 = 2,   // row m = (b, ho, wo): im2col gather of a 3x3 window, zero padding 1
+};
+
+namespace i8 {
+
+struct Params {
+    const __half* X = nullptr;
+    long long ldx = 0;
+    int M = 0, N = 0, K = 0, k_blocks = 0;
+    int H = 0, W = 0, Cin = 0, Ho = 0, Wo = 0, stride = 1;  // conv geometry
+    int batch = 0;                                          // prompts (BOS mode)
+    const float* act_scale = nullptr;
+    const float* w_scale = nullptr;
+    const __half* bias = nullptr;
+    const __half* bos_out = nullptr;
+    __half* Y = nullptr;
+    long long ldy = 0;
+    int32_t* acc_out = nullptr;
+    int32_t* status = nullptr;
+    int32_t* ws_tickets = nullptr;  // split-K: one arrival counter per output tile
+    int32_t* ws_acc = nullptr;      // split-K: int32 partial sums, padded to whole tiles
+    int force_splits = 0;           // > 0: use exactly this many reduction splits
+};
+
+size_t workspace_bytes(int64_t rows, int64_t N);
+int run(Params p, int amode, const void* packed, int w_bits, void* workspace, size_t ws_bytes,
+        cudaStream_t stream);
+
+}  // namespace i8
+
+namespace wo {
+
+struct Params {
+    const __half* X = nullptr;
+    long long ldx = 0;
+    int M = 0, N = 0, K = 0;
+    int H = 0, W = 0, Cin = 0, Ho = 0, Wo = 0, stride = 1;
+    const float* w_scale = nullptr;
+    const int32_t* w_zero = nullptr;  // nullptr: signed codes, zero-point 0
+    const __half* bias = nullptr;
+    __half* Y = nullptr;
+    long long ldy = 0;
+    int32_t* status = nullptr;
+};
+
+int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream);
+
+}  // namespace wo
+
+}  // namespace mixdq

@@ -110,19 +110,25 @@ __global__ void pack_kernel(const __half* __restrict__ W, int64_t N, int64_t K, 
             }
         }
     } else {  // 3-bit planes
-        int64_t k0;
-        int plane;
         if (layout == MIXDQ_LAYOUT_CANONICAL) {
-            k0 = 32 * (w / 3);  // group g: words 3g .. 3g+2 are planes 0..2
-            plane = static_cast<int>(w % 3);
+            const int64_t k0 = 32 * (w / 3);  // group g: words 3g .. 3g+2 are planes 0..2
+            const int plane = static_cast<int>(w % 3);
+            for (int j = 0; j < 32; ++j)
+                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << j;
         } else {
-            const int64_t blk = w / 12;  // block of 128 codes: 4 words per plane, planes in order
+            // block of 128 codes: planes in order, 4 words each; word t of a plane covers codes
+            // 32t .. 32t+31 with bit 4f + s = code 8s + (f even ? f/2 : 4 + f/2), which is the
+            // field order of the 4-bit device layout spread over four shifts of the word
+            const int64_t blk = w / 12;
             const int r = static_cast<int>(w % 12);
-            plane = r / 4;
-            k0 = 128 * blk + 32 * (r % 4);
+            const int plane = r / 4;
+            const int64_t k0 = 128 * blk + 32 * (r % 4);
+            for (int pos = 0; pos < 32; ++pos) {
+                const int f = pos >> 2, sft = pos & 3;
+                const int j = 8 * sft + ((f & 1) ? 4 + (f >> 1) : (f >> 1));
+                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << pos;
+            }
         }
-        for (int j = 0; j < 32; ++j)
-            word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << j;
     }
     // the last word of an odd-sized canonical row may be partial
     const int64_t byte0 = 4 * w;
@@ -156,14 +162,20 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ packed, int64_t N, int
         c = 0;
         for (int p = 0; p < 3; ++p) {
             int64_t byte;
+            int bit;
             if (layout == MIXDQ_LAYOUT_CANONICAL) {
                 byte = (k / 32) * 12 + p * 4 + ((k % 32) >> 3);
+                bit = static_cast<int>(k & 7);
             } else {
                 const int64_t blk = k / 128;
                 const int r = static_cast<int>(k % 128);
-                byte = blk * 48 + p * 16 + (r >> 5) * 4 + ((r & 31) >> 3);
+                const int t = r >> 5, sft = (r & 31) >> 3, j = r & 7;
+                const int f = (j < 4) ? 2 * j : 2 * (j - 4) + 1;
+                const int pos = 4 * f + sft;
+                byte = blk * 48 + p * 16 + t * 4 + (pos >> 3);
+                bit = pos & 7;
             }
-            c |= ((row[byte] >> (k & 7)) & 1) << p;
+            c |= ((row[byte] >> bit) & 1) << p;
         }
     }
     codes[idx] = static_cast<int16_t>(c);

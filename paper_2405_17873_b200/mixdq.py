@@ -1,0 +1,238 @@
+"""ctypes binding of the C-ABI CUDA library (``libmixdq.so``).
+
+Argument marshalling only: torch tensors supply device memory and the current stream,
+every step of the path runs in the library's kernels.  There is no CPU fallback: if the
+shared library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmixdq.so")
+
+LAYOUT_CANONICAL = 0
+LAYOUT_DEVICE = 1
+TOKENS_PER_PROMPT = 77
+
+_i64, _int, _vp, _sz = C.c_int64, C.c_int, C.c_void_p, C.c_size_t
+
+_SIGNATURES = {
+    "mixdq_version": (C.c_int, []),
+    "mixdq_strerror": (C.c_char_p, [_int]),
+    "mixdq_packed_bytes": (_int, [_i64, _i64, _int, _int, C.POINTER(_sz)]),
+    "mixdq_weight_minmax_params": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp, _vp]),
+    "mixdq_pack_weights": (_int, [_vp, _i64, _i64, _int, _vp, _vp, _int, _vp, _vp]),
+    "mixdq_unpack_weights": (_int, [_vp, _i64, _i64, _int, _int, _int, _vp, _vp]),
+    "mixdq_act_absmax": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp]),
+    "mixdq_act_scale_from_absmax": (_int, [_vp, _vp, _vp]),
+    "mixdq_workspace_bytes": (_int, [_i64, _i64, _i64, _int, _int, C.POINTER(_sz)]),
+    "mixdq_linear": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp, _sz,
+                            _vp, _vp]),
+    "mixdq_linear_acc_i32": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_conv3x3": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _int, _vp, _vp, _vp,
+                             _vp, _sz, _vp, _vp]),
+    "mixdq_conv3x3_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp, _sz,
+                                     _vp, _vp]),
+    "mixdq_conv1x1": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp,
+                             _sz, _vp, _vp]),
+    "mixdq_crossattn_kv": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_crossattn_kv_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _sz, _vp, _vp]),
+}
+
+EXPORTS = tuple(_SIGNATURES)
+
+_lib = None
+
+
+class MixdqError(RuntimeError):
+    pass
+
+
+def lib():
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise MixdqError(f"{LIB_PATH} is missing: build it with python -m paper_2405_17873_b200.build")
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _chk(rc: int, what: str):
+    if rc != 0:
+        raise MixdqError(f"{what}: {lib().mixdq_strerror(rc).decode()} ({rc})")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def version() -> int:
+    return lib().mixdq_version()
+
+
+def packed_bytes(N: int, K: int, bits: int, layout: int = LAYOUT_DEVICE) -> int:
+    out = _sz(0)
+    _chk(lib().mixdq_packed_bytes(N, K, bits, layout, C.byref(out)), "mixdq_packed_bytes")
+    return out.value
+
+
+def workspace_bytes(rows: int, N: int, K: int, w_bits: int, act_bits: int) -> int:
+    out = _sz(0)
+    _chk(lib().mixdq_workspace_bytes(rows, N, K, w_bits, act_bits, C.byref(out)), "mixdq_workspace_bytes")
+    return out.value
+
+
+def new_workspace(nbytes: int, device="cuda") -> Optional[torch.Tensor]:
+    """Zero-filled scratch buffer of the size mixdq_workspace_bytes reported."""
+    if nbytes == 0:
+        return None
+    return torch.zeros(nbytes, dtype=torch.uint8, device=device)
+
+
+def weight_minmax_params(W: torch.Tensor, bits: int, symmetric: bool):
+    N, K = W.shape
+    scale = torch.empty(N, dtype=torch.float32, device=W.device)
+    zero = torch.zeros(N, dtype=torch.int32, device=W.device)
+    _chk(lib().mixdq_weight_minmax_params(_ptr(W), N, K, bits, int(symmetric), _ptr(scale), _ptr(zero),
+                                          _stream()), "mixdq_weight_minmax_params")
+    return scale, zero
+
+
+def pack_weights(W: torch.Tensor, bits: int, scale: torch.Tensor, zero: Optional[torch.Tensor] = None,
+                 layout: int = LAYOUT_DEVICE) -> torch.Tensor:
+    N, K = W.shape
+    out = torch.zeros(packed_bytes(N, K, bits, layout), dtype=torch.uint8, device=W.device)
+    _chk(lib().mixdq_pack_weights(_ptr(W), N, K, bits, _ptr(scale), _ptr(zero), layout, _ptr(out), _stream()),
+         "mixdq_pack_weights")
+    return out
+
+
+def unpack_weights(packed: torch.Tensor, N: int, K: int, bits: int, is_signed: bool,
+                   layout: int = LAYOUT_DEVICE) -> torch.Tensor:
+    codes = torch.empty((N, K), dtype=torch.int16, device=packed.device)
+    _chk(lib().mixdq_unpack_weights(_ptr(packed), N, K, bits, int(is_signed), layout, _ptr(codes), _stream()),
+         "mixdq_unpack_weights")
+    return codes
+
+
+def act_absmax(X: torch.Tensor, skip_rows_mod: int = 0) -> torch.Tensor:
+    X2 = X.reshape(-1, X.shape[-1])
+    out = torch.empty(1, dtype=torch.float32, device=X.device)
+    _chk(lib().mixdq_act_absmax(_ptr(X2), X2.shape[0], X2.shape[1], X2.shape[1], skip_rows_mod, _ptr(out),
+                                _stream()), "mixdq_act_absmax")
+    return out
+
+
+def act_scale_from_absmax(amax: torch.Tensor) -> torch.Tensor:
+    out = torch.empty(1, dtype=torch.float32, device=amax.device)
+    _chk(lib().mixdq_act_scale_from_absmax(_ptr(amax), _ptr(out), _stream()), "mixdq_act_scale_from_absmax")
+    return out
+
+
+def act_scale(X: torch.Tensor, skip_rows_mod: int = 0) -> torch.Tensor:
+    """Dynamic per-tensor int8 scale max|X| / 127, computed on the device."""
+    return act_scale_from_absmax(act_absmax(X, skip_rows_mod))
+
+
+def _ws(workspace):
+    return (_ptr(workspace), workspace.numel() if workspace is not None else 0)
+
+
+def linear(X, packed_W, N: int, w_bits: int, w_scale, w_zero=None, act_bits: int = 8, act_scale=None,
+           bias=None, workspace=None, status=None, out=None):
+    M, K = X.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits, _ptr(w_scale), _ptr(w_zero),
+                            act_bits, _ptr(act_scale), _ptr(bias), _ptr(Y), wp, wb, _ptr(status), _stream()),
+         "mixdq_linear")
+    return Y
+
+
+def linear_acc_i32(X, packed_W, N: int, w_bits: int, act_scale, workspace=None, status=None):
+    M, K = X.shape
+    acc = torch.empty((M, N), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear_acc_i32(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits, _ptr(act_scale),
+                                    _ptr(acc), wp, wb, _ptr(status), _stream()), "mixdq_linear_acc_i32")
+    return acc
+
+
+def _out_hw(H, W, stride):
+    return (H - 1) // stride + 1, (W - 1) // stride + 1
+
+
+def conv3x3(X, packed_W, Cout: int, w_bits: int, w_scale, w_zero=None, act_bits: int = 8, act_scale=None,
+            bias=None, stride: int = 1, workspace=None, status=None, out=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    Y = out if out is not None else torch.empty((B, Ho, Wo, Cout), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits, _ptr(w_scale),
+                             _ptr(w_zero), act_bits, _ptr(act_scale), _ptr(bias), _ptr(Y), wp, wb,
+                             _ptr(status), _stream()), "mixdq_conv3x3")
+    return Y
+
+
+def conv3x3_acc_i32(X, packed_W, Cout: int, w_bits: int, act_scale, stride: int = 1, workspace=None,
+                    status=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    acc = torch.empty((B, Ho, Wo, Cout), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3_acc_i32(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits,
+                                     _ptr(act_scale), _ptr(acc), wp, wb, _ptr(status), _stream()),
+         "mixdq_conv3x3_acc_i32")
+    return acc
+
+
+def conv1x1(X, packed_W, Cout: int, w_bits: int, w_scale, w_zero=None, act_bits: int = 8, act_scale=None,
+            bias=None, workspace=None, status=None):
+    B, H, W, Cin = X.shape
+    Y = torch.empty((B, H, W, Cout), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv1x1(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, w_bits, _ptr(w_scale), _ptr(w_zero),
+                             act_bits, _ptr(act_scale), _ptr(bias), _ptr(Y), wp, wb, _ptr(status), _stream()),
+         "mixdq_conv1x1")
+    return Y
+
+
+def crossattn_kv(text_emb, packed_W, N: int, w_bits: int, w_scale, act_scale, bos_out, workspace=None,
+                 status=None, out=None):
+    B, T, Kt = text_emb.shape
+    assert T == TOKENS_PER_PROMPT
+    Y = out if out is not None else torch.empty((B, T, N), dtype=torch.float16, device=text_emb.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_crossattn_kv(_ptr(text_emb), B, Kt, _ptr(packed_W), N, w_bits, _ptr(w_scale),
+                                  _ptr(act_scale), _ptr(bos_out), _ptr(Y), wp, wb, _ptr(status), _stream()),
+         "mixdq_crossattn_kv")
+    return Y
+
+
+def crossattn_kv_acc_i32(text_emb, packed_W, N: int, w_bits: int, act_scale, workspace=None, status=None):
+    B, T, Kt = text_emb.shape
+    assert T == TOKENS_PER_PROMPT
+    acc = torch.empty((B, T - 1, N), dtype=torch.int32, device=text_emb.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_crossattn_kv_acc_i32(_ptr(text_emb), B, Kt, _ptr(packed_W), N, w_bits, _ptr(act_scale),
+                                          _ptr(acc), wp, wb, _ptr(status), _stream()),
+         "mixdq_crossattn_kv_acc_i32")
+    return acc

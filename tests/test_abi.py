@@ -1,0 +1,93 @@
+"""The C-ABI library loads without a GPU, exports what include/mixdq.h declares, and its
+host-side argument checks answer before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2405_17873_b200 import build, mixdq
+    build.build()
+    return mixdq.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "mixdq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mixdq_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2405_17873_b200 import mixdq
+    names = _declared()
+    assert len(names) >= 16
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(mixdq.EXPORTS) == names
+
+
+def test_no_link_time_dependency_on_the_driver():
+    import subprocess
+    from paper_2405_17873_b200 import mixdq
+    out = subprocess.run(["ldd", mixdq.LIB_PATH], capture_output=True, text=True).stdout
+    assert "libcuda.so" not in out and "libtorch" not in out
+
+
+def test_version_and_strerror(lib):
+    assert lib.mixdq_version() >= 100
+    assert lib.mixdq_strerror(0) == b"success"
+    for code in range(-6, 0):
+        assert lib.mixdq_strerror(code) not in (b"", b"unknown error")
+    assert lib.mixdq_strerror(-99) == b"unknown error"
+
+
+def test_packed_bytes_size_laws(lib):
+    out = C.c_size_t(0)
+    for N, K in ((320, 320), (1280, 320), (7, 77), (640, 2048)):
+        for bits, canon in ((8, K), (4, (K + 1) // 2), (3, ((K + 31) // 32) * 12)):
+            assert lib.mixdq_packed_bytes(N, K, bits, 0, C.byref(out)) == 0
+            assert out.value == N * canon
+            assert lib.mixdq_packed_bytes(N, K, bits, 1, C.byref(out)) == 0
+            assert out.value >= N * canon and out.value % 16 == 0
+    # multiples of 128 codes pack without padding in the device layout too
+    for bits in (3, 4, 8):
+        lib.mixdq_packed_bytes(64, 1280, bits, 1, C.byref(out))
+        assert out.value == 64 * 1280 * bits // 8
+    assert lib.mixdq_packed_bytes(4, 4, 5, 0, C.byref(out)) == -2
+    assert lib.mixdq_packed_bytes(0, 4, 4, 0, C.byref(out)) == -1
+    assert lib.mixdq_packed_bytes(4, 4, 4, 7, C.byref(out)) == -1
+    assert lib.mixdq_packed_bytes(4, 4, 4, 0, None) == -1
+
+
+def test_argument_errors_come_back_before_any_launch(lib):
+    out = C.c_size_t(0)
+    assert lib.mixdq_workspace_bytes(256, 320, 320, 8, 8, C.byref(out)) == 0 and out.value > 0
+    assert lib.mixdq_workspace_bytes(256, 320, 320, 4, 16, C.byref(out)) == 0 and out.value == 0
+    assert lib.mixdq_workspace_bytes(256, 320, 320, 5, 8, C.byref(out)) == -2
+    assert lib.mixdq_workspace_bytes(0, 320, 320, 8, 8, C.byref(out)) == -1
+    null = None
+    fake = C.c_void_p(0x1000)       # never dereferenced: the checks below fail first
+    odd = C.c_void_p(0x1008)
+    # NULL tensors
+    assert lib.mixdq_linear(null, 4, 32, 32, fake, 16, 8, fake, null, 8, fake, null, fake, null, 0, null, null) == -1
+    assert lib.mixdq_linear(fake, 4, 32, 32, fake, 16, 8, fake, null, 8, fake, null, null, null, 0, null, null) == -1
+    # row stride smaller than K, non-positive sizes
+    assert lib.mixdq_linear(fake, 4, 32, 16, fake, 16, 8, fake, null, 8, fake, null, fake, null, 0, null, null) == -1
+    assert lib.mixdq_linear(fake, 0, 32, 32, fake, 16, 8, fake, null, 8, fake, null, fake, null, 0, null, null) == -1
+    # widths: 3-bit weights with int8 activations, asymmetric weights on the int8 path, 5-bit
+    assert lib.mixdq_linear(fake, 4, 32, 32, fake, 16, 3, fake, null, 8, fake, null, fake, null, 0, null, null) == -2
+    assert lib.mixdq_linear(fake, 4, 32, 32, fake, 16, 8, fake, fake, 8, fake, null, fake, null, 0, null, null) == -2
+    assert lib.mixdq_linear(fake, 4, 32, 32, fake, 16, 5, fake, fake, 16, null, null, fake, null, 0, null, null) == -2
+    assert lib.mixdq_linear(fake, 4, 32, 32, fake, 16, 8, fake, null, 12, fake, null, fake, null, 0, null, null) == -2
+    # misaligned packed weights
+    assert lib.mixdq_linear(fake, 4, 32, 32, odd, 16, 8, fake, null, 8, fake, null, fake, null, 0, null, null) == -3
+    # conv stride, BOS call without the stored row
+    assert lib.mixdq_conv3x3(fake, 1, 8, 8, 16, fake, 16, 3, 8, fake, null, 8, fake, null, fake, null, 0, null, null) == -1
+    assert lib.mixdq_crossattn_kv(fake, 1, 2048, fake, 640, 8, fake, fake, null, fake, null, 0, null, null) == -1
+    assert lib.mixdq_pack_weights(fake, 4, 32, 3, fake, null, 1, fake, null) == -2
+    assert lib.mixdq_pack_weights(fake, 4, 32, 4, fake, null, 1, odd, null) == -3
