@@ -1,0 +1,158 @@
+"""GPU parity of the W8A8 / W4A8 engine: int32 accumulators bit-exact, fp16 outputs within
+the path's tolerance, on linear layers, the BOS-aware K/V projection and 3x3 convs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mixdq_oracle as orc
+from paper_2405_17873_b200 import mixdq, synth
+from helpers import (assert_close, dev, device_weights, host, oracle_weights, status_word, workspace_for)
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_linear(X, W, b, bits, use_ws):
+    M, K = X.shape
+    N = W.shape[0]
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.linear_a8(X, codes, s_ref, sx_ref, b)
+
+    Xd = dev(X)
+    s, _, packed = device_weights(W, bits, True)
+    sx = mixdq.act_scale(Xd)
+    assert host(sx)[0] == sx_ref
+    st = status_word()
+    ws = workspace_for(M, N, K, bits) if use_ws else None
+    acc = mixdq.linear_acc_i32(Xd, packed, N, bits, sx, workspace=ws, status=st)
+    y = mixdq.linear(Xd, packed, N, bits, s, None, 8, sx, None if b is None else dev(b), workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+    if ws is not None:
+        assert not bool(ws.any())          # the scratch is left zero-filled
+
+
+def test_single_linear_w8a8_seed0():
+    X, W, b = synth.single_linear(seed=0)
+    _run_linear(X, W, b, 8, False)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,K,N", [(1, 16, 16), (77, 336, 200), (300, 320, 328), (129, 1040, 136), (256, 2048, 24)])
+def test_linear_ragged_tiles(bits, M, K, N):
+    g = synth.normal_f16((M, K), 1.0, seed=M + K)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 1)
+    b = synth.normal_f16((N,), 0.01, seed=N)
+    _run_linear(g, W, b, bits, False)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,K,N", [(256, 5120, 320), (130, 1280, 200), (512, 4096, 136)])
+def test_linear_split_reduction(bits, M, K, N):
+    g = synth.normal_f16((M, K), 1.0, seed=M + K + 7)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 8)
+    _run_linear(g, W, None, bits, True)
+    _run_linear(g, W, None, bits, True)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_linear_corner_shapes_plain_kernel(bits):
+    # reduction length not a multiple of 16, and fewer than 16 output channels
+    _run_linear(synth.normal_f16((50, 36), 1.0, 1), synth.normal_f16((40, 36), 0.02, 2), None, bits, False)
+    _run_linear(synth.normal_f16((70, 64), 1.0, 3), synth.normal_f16((4, 64), 0.02, 4),
+                synth.normal_f16((4,), 0.01, 5), bits, False)
+
+
+def test_ffn_outlier_channels():
+    X = synth.ffn_input(1, seed=3000, K=1280)
+    W = synth.normal_f16((384, 1280), 0.02, seed=3001)
+    _run_linear(X, W, None, 4, True)
+    _run_linear(X, W, None, 8, True)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,N", [(1, 64), (3, 200)])
+def test_bos_aware_kv(bits, B, N):
+    E = synth.text_embedding(B, seed=4000)
+    W = synth.kv_weight(N, seed=4100 + N)
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    bos = orc.bos_row(E[0, 0], W)
+    sx_ref = orc.crossattn_act_scale(E)
+    acc_ref, y_ref = orc.crossattn_kv(E, codes, s_ref, sx_ref, bos)
+
+    Ed = dev(E)
+    s, _, packed = device_weights(W, bits, True)
+    sx = mixdq.act_scale(Ed.reshape(-1, E.shape[-1]), skip_rows_mod=77)
+    assert host(sx)[0] == sx_ref
+    st = status_word()
+    ws = workspace_for(B * 76, N, 2048, bits)
+    acc = mixdq.crossattn_kv_acc_i32(Ed, packed, N, bits, sx, workspace=ws, status=st)
+    y = mixdq.crossattn_kv(Ed, packed, N, bits, s, sx, dev(bos), workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    yh = host(y)
+    for b in range(B):
+        assert np.array_equal(yh[b, 0].view(np.uint16), bos.view(np.uint16))
+    assert_close(yh, y_ref)
+    # what token 0 holds changes nothing in rows >= 1
+    E2 = E.copy()
+    E2[:, 0, :] = np.float16(-777.0)
+    y2 = mixdq.crossattn_kv(dev(E2), packed, N, bits, s, sx, dev(bos), workspace=ws, status=st)
+    assert np.array_equal(host(y2).view(np.uint16), yh.view(np.uint16))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,W,Cin,Cout,stride", [(1, 8, 8, 16, 16, 1), (2, 12, 10, 32, 48, 1),
+                                                    (2, 12, 10, 32, 48, 2), (1, 16, 16, 320, 136, 1),
+                                                    (3, 9, 7, 48, 24, 2)])
+def test_conv3x3(bits, B, H, W, Cin, Cout, stride):
+    X = synth.normal_f16((B, H, W, Cin), 1.0, seed=H * W + Cin)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin)
+    b = synth.normal_f16((Cout,), 0.01, seed=Cout)
+    s_ref, _, codes = oracle_weights(Wt.reshape(Cout, -1), bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.conv3x3_a8(X, codes.reshape(Cout, 3, 3, Cin), s_ref, sx_ref, b, stride)
+
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt.reshape(Cout, -1), bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    ws = workspace_for(acc_ref.size // Cout, Cout, 9 * Cin, bits)
+    acc = mixdq.conv3x3_acc_i32(Xd, packed, Cout, bits, sx, stride, workspace=ws, status=st)
+    y = mixdq.conv3x3(Xd, packed, Cout, bits, s, None, 8, sx, dev(b), stride, workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+
+
+def test_conv_corner_shapes_plain_kernel():
+    # conv_in-like (4 input channels) and conv_out-like (4 output channels)
+    for Cin, Cout in ((4, 32), (32, 4)):
+        X = synth.normal_f16((1, 10, 10, Cin), 1.0, seed=Cin)
+        Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout)
+        s_ref, _, codes = oracle_weights(Wt.reshape(Cout, -1), 8, True)
+        sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+        acc_ref, y_ref = orc.conv3x3_a8(X, codes.reshape(Cout, 3, 3, Cin), s_ref, sx_ref, None, 1)
+        Xd = dev(X)
+        s, _, packed = device_weights(Wt.reshape(Cout, -1), 8, True)
+        sx = mixdq.act_scale(Xd)
+        acc = mixdq.conv3x3_acc_i32(Xd, packed, Cout, 8, sx, 1)
+        y = mixdq.conv3x3(Xd, packed, Cout, 8, s, None, 8, sx, None, 1)
+        assert np.array_equal(host(acc), acc_ref)
+        assert_close(host(y), y_ref)
+
+
+def test_conv1x1_equals_linear():
+    X = synth.normal_f16((2, 8, 8, 64), 1.0, seed=11)
+    Wt = synth.normal_f16((48, 64), 0.02, seed=12)
+    s_ref, _, codes = oracle_weights(Wt, 4, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    _, y_ref = orc.linear_a8(X.reshape(-1, 64), codes, s_ref, sx_ref, None)
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt, 4, True)
+    y = mixdq.conv1x1(Xd, packed, 48, 4, s, None, 8, mixdq.act_scale(Xd), None)
+    assert_close(host(y).reshape(-1, 48), y_ref)
