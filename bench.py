@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized UNet layer sweep (one JSON line on stdout).
+
+A step is one pass over every quantizable layer of the SDXL-turbo-shaped 512px UNet
+(794 layers) at image batch B, each layer at the widths its bit table assigns
+(default: W4A8 with 10% of the layers at W8A8).  Weights are distinct per layer
+(1.3 GB packed, far larger than L2); inputs are seeded and synthetic.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--batch B] [--table w4a8|a16]
+  python bench.py --impl reference ...    # the CPU oracle on a bounded sample
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same sweep on its own
+images: independent replicas, no data-path collective, weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "unet_layer_sweep_throughput"
+UNIT = "TOP/s"
+INT8_TO_BF16_NOMINAL = 2.0  # dense int8 : bf16 tensor throughput of the part (4.5 : 2.25 POP/s)
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=4)
+    ap.add_argument("--table", default="w4a8", choices=["w4a8", "a16"])
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(args):
+    return f"unet_sweep_sdxl512_{args.table}_b{args.batch}"
+
+
+# ----------------------------------------------------------------------------- peaks
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+
+def oracle_sample_layers(table: str, batch: int, mac_budget: float):
+    """A bounded sample of the sweep for the CPU oracle: layers of distinct shapes, in census
+    order, until the MAC budget is spent (at least one layer)."""
+    from paper_2405_17873_b200 import synth
+    layers = synth.unet_layers()
+    (synth.assign_bits_w4a8 if table == "w4a8" else synth.assign_bits_weight_only)(layers)
+    seen, picked, macs = set(), [], 0.0
+    # cheapest distinct shapes first, so that a small budget still covers several kinds
+    order = sorted(layers, key=lambda l: l.ops(batch))
+    for l in order:
+        key = (l.kind, l.M, l.N, l.K, l.stride, l.w_bits, l.a_bits)
+        if key in seen:
+            continue
+        m = l.ops(batch) / 2
+        if picked and macs + m > mac_budget:
+            continue
+        seen.add(key)
+        picked.append(l)
+        macs += m
+    return picked
+
+
+def oracle_run_layers(picked, batch: int, prepared=None):
+    """One oracle pass over the sample; returns (seconds, ops, prepared inputs)."""
+    from oracle import mixdq_oracle as orc
+    from paper_2405_17873_b200 import synth
+    if prepared is None:
+        prepared = []
+        for l in picked:
+            X, W, b = synth.layer_inputs(l, batch, seed=5000 + l.index)
+            W2 = W.reshape(l.N, -1)
+            sym = l.a_bits == 8
+            s, z = orc.weight_minmax_params(W2, l.w_bits, sym)
+            codes = orc.quantize_weights(W2, l.w_bits, s, None if sym else z)
+            extra = {}
+            if l.a_bits == 8:
+                if l.kind == "bos_kv":
+                    extra["sx"] = orc.crossattn_act_scale(X)
+                    extra["bos"] = orc.bos_row(X[0, 0], W2)
+                else:
+                    extra["sx"] = orc.act_scale(orc.act_absmax(X), 8)
+            prepared.append((l, X, codes, s, None if sym else z, b, extra))
+    t0 = time.perf_counter()
+    ops = 0
+    for l, X, codes, s, z, b, extra in prepared:
+        if l.a_bits == 8:
+            if l.kind == "conv3x3":
+                orc.conv3x3_a8(X, codes.reshape(l.N, 3, 3, l.Cin), s, extra["sx"], b, l.stride)
+            elif l.kind == "bos_kv":
+                orc.crossattn_kv(X, codes, s, extra["sx"], extra["bos"])
+            else:
+                orc.linear_a8(X.reshape(-1, l.K), codes, s, extra["sx"], b)
+        else:
+            if l.kind == "conv3x3":
+                orc.conv3x3_a16(X, codes.reshape(l.N, 3, 3, l.Cin), s, z, b, l.stride)
+            else:
+                orc.linear_a16(X.reshape(-1, l.K), codes, s, z, None if l.kind == "bos_kv" else b)
+        ops += l.ops(batch)
+    return time.perf_counter() - t0, ops, prepared
+
+
+def oracle_rate_estimate(table: str) -> float:
+    """MAC/s of the oracle on this host, from one small layer."""
+    from oracle import mixdq_oracle as orc
+    import numpy as np
+    rng = np.random.default_rng(0)
+    M, N, K = 128, 320, 640
+    X = rng.normal(size=(M, K)).astype(np.float16)
+    codes = rng.integers(0, 8, size=(N, K)).astype(np.int16)
+    s = np.ones(N, np.float32)
+    t0 = time.perf_counter()
+    if table == "w4a8":
+        orc.linear_a8(X, codes, s, np.float32(0.03), None)
+    else:
+        orc.linear_a16(X, codes, s, np.zeros(N, np.int32), None)
+    return M * N * K / (time.perf_counter() - t0)
+
+
+def cpu_baseline(table: str, batch: int, seconds: float):
+    from oracle import mixdq_oracle as orc
+    rate = oracle_rate_estimate(table)
+    picked = oracle_sample_layers(table, batch, rate * seconds)
+    dt, ops, _ = oracle_run_layers(picked, batch)
+    return {"value": ops / dt / 1e12, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{len(picked)} layers of distinct shapes of the sweep ({ops / 2e9:.1f} GMAC), one pass, "
+                      f"{dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import mixdq_oracle as orc
+    total = args.steps + args.warmup
+    rate = oracle_rate_estimate(args.table)
+    per_step_s = max(0.02, min(5.0, 120.0 / max(total, 1)))
+    picked = oracle_sample_layers(args.table, args.batch, rate * per_step_s)
+    prepared = None
+    for _ in range(args.warmup):
+        _, _, prepared = oracle_run_layers(picked, args.batch, prepared)
+    t, ops = 0.0, 0
+    for _ in range(args.steps):
+        dt, o, prepared = oracle_run_layers(picked, args.batch, prepared)
+        t += dt
+        ops += o
+    value = ops / t / 1e12
+    sample = f"{len(picked)} layers of distinct shapes per step ({ops / args.steps / 2e9:.2f} GMAC per step)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8" if args.table == "w4a8" else "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args), "table": args.table, "batch": args.batch},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2405_17873_b200 import build, mixdq
+    from paper_2405_17873_b200.unet_sweep import UNetSweep
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    build.build()
+    mixdq.lib()  # fail here, loudly, if the CUDA library is missing
+
+    sweep = UNetSweep(args.batch, args.table, seed=5 + rank)
+    tc_layers = [pl for pl in sweep.layers if sweep.uses_tensor_int8(pl)]
+    other_layers = [pl for pl in sweep.layers if not sweep.uses_tensor_int8(pl)]
+    if args.table == "a16":
+        tc_layers, other_layers = [], list(sweep.layers)  # all on the weight-only engine
+
+    # warm-up outside the graphs (also sets kernel attributes), then capture one step as two graphs
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            sweep.step()
+    torch.cuda.synchronize()
+    graphs = []
+    for group in (tc_layers, other_layers):
+        if not group:
+            graphs.append(None)
+            continue
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            sweep.step(group)
+        graphs.append(g)
+    g_tc, g_other = graphs
+    launches_per_step = len(sweep.layers)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            if g_tc is not None:
+                g_tc.replay()
+            if g_other is not None:
+                g_other.replay()
+        torch.cuda.synchronize()
+
+        # ---------------- timed region: inputs resident in HBM
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        time.sleep(0.3)
+        marks = []
+        barrier()
+        torch.cuda.synchronize()
+        start, end = ev(), ev()
+        start.record()
+        for _ in range(args.steps):
+            a, b, c = ev(), ev(), ev()
+            a.record()
+            if g_tc is not None:
+                g_tc.replay()
+            b.record()
+            if g_other is not None:
+                g_other.replay()
+            c.record()
+            marks.append((a, b, c))
+        end.record()
+        torch.cuda.synchronize()
+        barrier()
+        total_ms = start.elapsed_time(end)
+        clocks = sampler.stop()
+        tc_ms = sum(a.elapsed_time(b) for a, b, _ in marks) / args.steps
+        other_ms = sum(b.elapsed_time(c) for _, b, c in marks) / args.steps
+        status = int(sweep.status.item())
+
+        # ---------------- end to end: host buffers in, host buffers out, every step
+        x_host = {k: torch.empty_like(v, device="cpu").pin_memory().copy_(v) for k, v in sweep.x.items()}
+        y_host = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in sweep.y.items()}
+        h2d = sum(v.numel() * 2 for v in x_host.values())
+        d2h = sum(v.numel() * 2 for v in y_host.values())
+
+        def e2e_step():
+            for k, v in x_host.items():
+                sweep.x[k].copy_(v, non_blocking=True)
+            if g_tc is not None:
+                g_tc.replay()
+            if g_other is not None:
+                g_other.replay()
+            for k, v in y_host.items():
+                v.copy_(sweep.y[k], non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        torch.cuda.synchronize()
+        s2, e2 = ev(), ev()
+        s2.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e2.record()
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = s2.elapsed_time(e2) / args.e2e_steps
+
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_per_step, e2e_ms, tc_ms, other_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, e2e_ms, tc_ms, other_ms = t.tolist()
+
+    ops_step = sweep.total_ops()
+    peaks = measured_peaks()
+    if args.table == "w4a8":
+        tc_ops = sweep.total_ops(tc_layers)
+        achieved = tc_ops / (tc_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
+                    "traffic": None, "kernel": "i8::gemm_kernel (tcgen05 kind::i8)",
+                    "peak_source": f"{peaks['source']} bf16 sustained x {INT8_TO_BF16_NOMINAL:g} (nominal int8:bf16)",
+                    "launches_per_step": len(tc_layers), "ms_per_step": tc_ms}
+    else:
+        alg = sum(sweep.algorithmic_bytes(pl) for pl in sweep.layers)
+        achieved = alg / (other_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "wo::wo_kernel (mma.sync f16)",
+                    "peak_source": f"{peaks['source']} copy bandwidth", "launches_per_step": len(other_layers),
+                    "ms_per_step": other_ms}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": world * ops_step / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8" if args.table == "w4a8" else "f16",
+            "data": "synthetic",
+            "config": {"workload": workload_name(args), "table": args.table, "batch": args.batch,
+                       "layers": len(sweep.layers), "ops_per_step": ops_step,
+                       "packed_weight_bytes": sweep.packed_weight_bytes(),
+                       "l2": "weights (distinct per layer) are larger than L2", "launch": "CUDA graph replay"},
+            "clocks": clocks,
+            "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline,
+            "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
+            "device_status": status,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

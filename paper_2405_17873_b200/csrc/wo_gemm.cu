@@ -137,16 +137,31 @@ __device__ __forceinline__ uint4 load_x8(const Params& p, int amode, int m, int 
         const int hw = p.Ho * p.Wo;
         const int b = m / hw, rem = m - b * hw;
         const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+        const long long img = static_cast<long long>(b) * p.H * p.W * p.Cin;
+        if (p.Cin % 8 != 0) {
+            // a run of eight may straddle filter taps: gather element by element
+            __align__(16) __half tmp[8];
+            for (int j = 0; j < 8; ++j) {
+                tmp[j] = __float2half(0.f);
+                const int kk = k + j;
+                if (kk >= p.K) continue;
+                const int tap = kk / p.Cin, c = kk - tap * p.Cin;
+                const int hi = ho * p.stride - 1 + tap / 3, wi = wo * p.stride - 1 + tap % 3;
+                if (hi < 0 || hi >= p.H || wi < 0 || wi >= p.W) continue;
+                tmp[j] = p.X[img + (static_cast<long long>(hi) * p.W + wi) * p.Cin + c];
+            }
+            return *reinterpret_cast<uint4*>(tmp);
+        }
         const int tap = k / p.Cin, c = k - tap * p.Cin;
         const int hi = ho * p.stride - 1 + tap / 3, wi = wo * p.stride - 1 + tap % 3;
         if (hi < 0 || hi >= p.H || wi < 0 || wi >= p.W) return make_uint4(0, 0, 0, 0);
-        src = p.X + ((static_cast<long long>(b) * p.H + hi) * p.W + wi) * p.Cin + c;
+        src = p.X + img + (static_cast<long long>(hi) * p.W + wi) * p.Cin + c;
     } else {
         src = p.X + static_cast<long long>(m) * p.ldx + k;
     }
     if (k + 8 <= p.K) return __ldg(reinterpret_cast<const uint4*>(src));
     // ragged end of the reduction (only when K is not a multiple of 8)
-    __half tmp[8];
+    __align__(16) __half tmp[8];
     for (int j = 0; j < 8; ++j) tmp[j] = (k + j < p.K) ? src[j] : __float2half(0.f);
     return *reinterpret_cast<uint4*>(tmp);
 }
@@ -310,7 +325,6 @@ int launch_nt(const Params& p, int amode, const void* packed, long long pitch, c
 int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream)
 {
     if (amode != A_LINEAR && amode != A_CONV3) return MIXDQ_ERR_INVALID_ARG;
-    if (amode == A_CONV3 && p.Cin % 8 != 0) return MIXDQ_ERR_UNSUPPORTED;
     if (amode == A_LINEAR && ((p.ldx % 8 != 0) || (reinterpret_cast<uintptr_t>(p.X) & 15)))
         return MIXDQ_ERR_ALIGNMENT;
     const long long pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);

@@ -1,0 +1,144 @@
+"""Layer sweep over the SDXL-turbo-shaped UNet: every quantizable layer once, each with the
+weight / activation widths its bit table assigns (the granularity of mixed precision is
+the layer, paper Sec. 5 "Hardware Friendly").
+
+The sweep owns device buffers only; each layer is one call into the C-ABI library, which
+picks the engine from the widths.  Weights are distinct per layer (as in the real model);
+layers with the same input shape read the same activation buffer.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional
+
+import torch
+
+from . import mixdq, synth
+
+
+@dataclass
+class PackedLayer:
+    spec: synth.LayerSpec
+    packed: torch.Tensor
+    w_scale: torch.Tensor
+    w_zero: Optional[torch.Tensor]
+    bias: Optional[torch.Tensor]
+    bos_out: Optional[torch.Tensor]
+    x_key: tuple
+    y_key: tuple
+
+
+class UNetSweep:
+    def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
+                 layers: Optional[List[synth.LayerSpec]] = None):
+        assert table in ("w4a8", "a16")
+        self.batch = batch
+        self.table = table
+        self.device = device
+        self.specs = layers if layers is not None else synth.unet_layers()
+        if layers is None:
+            if table == "w4a8":
+                synth.assign_bits_w4a8(self.specs, seed)
+            else:
+                synth.assign_bits_weight_only(self.specs, seed)
+        self.x: Dict[tuple, torch.Tensor] = {}
+        self.y: Dict[tuple, torch.Tensor] = {}
+        self.x_scale: Dict[tuple, torch.Tensor] = {}
+        self.layers: List[PackedLayer] = []
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self._build(seed)
+
+    # ------------------------------------------------------------------ setup (untimed)
+    def _x_shape(self, l: synth.LayerSpec):
+        B = self.batch
+        if l.kind in ("conv3x3", "conv1x1"):
+            return ("nhwc", B, l.H, l.H, l.Cin)
+        if l.kind == "bos_kv":
+            return ("text", B, synth.TOKENS_PER_PROMPT, l.K)
+        return ("rows", l.M * B, l.K)
+
+    def _y_shape(self, l: synth.LayerSpec):
+        B = self.batch
+        if l.kind == "conv3x3":
+            Ho = (l.H - 1) // l.stride + 1
+            return (B, Ho, Ho, l.N)
+        if l.kind == "conv1x1":
+            return (B, l.H, l.H, l.N)
+        if l.kind == "bos_kv":
+            return (B, synth.TOKENS_PER_PROMPT, l.N)
+        return (l.M * B, l.N)
+
+    def _build(self, seed: int):
+        g = torch.Generator(device=self.device).manual_seed(seed)
+        max_ws = 0
+        for l in self.specs:
+            xk, yk = self._x_shape(l), self._y_shape(l)
+            if xk not in self.x:
+                if xk[0] == "text":
+                    x = torch.from_numpy(synth.text_embedding(self.batch, seed=seed * 1000)).to(self.device)
+                else:
+                    x = torch.randn(xk[1:], generator=g, device=self.device, dtype=torch.float32).to(torch.float16)
+                self.x[xk] = x.contiguous()
+                if l.a_bits == 8 or self.table == "w4a8":
+                    skip = synth.TOKENS_PER_PROMPT if xk[0] == "text" else 0
+                    self.x_scale[xk] = mixdq.act_scale(self.x[xk].reshape(-1, xk[-1]), skip)
+            if yk not in self.y:
+                self.y[yk] = torch.empty(yk, dtype=torch.float16, device=self.device)
+            W = (torch.randn((l.N, l.K), generator=g, device=self.device, dtype=torch.float32) * 0.02).to(torch.float16)
+            bias = (torch.randn((l.N,), generator=g, device=self.device, dtype=torch.float32) * 0.01).to(torch.float16)
+            symmetric = l.a_bits == 8
+            s, z = mixdq.weight_minmax_params(W, l.w_bits, symmetric)
+            packed = mixdq.pack_weights(W, l.w_bits, s, None if symmetric else z)
+            bos = None
+            if l.kind == "bos_kv":
+                bias = None
+                if l.a_bits == 8:
+                    e0 = self.x[xk][0, 0].to(torch.float32)
+                    bos = (W.to(torch.float32) @ e0).to(torch.float16).contiguous()
+            self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk))
+            rows = yk[0] * (yk[1] if len(yk) > 2 else 1) * (yk[2] if len(yk) > 3 else 1)
+            max_ws = max(max_ws, mixdq.workspace_bytes(rows, l.N, l.K, l.w_bits, l.a_bits))
+        self.workspace = mixdq.new_workspace(max_ws, self.device)
+        torch.cuda.synchronize()
+
+    # ------------------------------------------------------------------ the timed pass
+    def run_layer(self, pl: PackedLayer, workspace=None):
+        l = pl.spec
+        x, y = self.x[pl.x_key], self.y[pl.y_key]
+        sx = self.x_scale.get(pl.x_key) if l.a_bits == 8 else None
+        ws = workspace if workspace is not None else self.workspace
+        if l.kind == "conv3x3":
+            return mixdq.conv3x3(x, pl.packed, l.N, l.w_bits, pl.w_scale, pl.w_zero, l.a_bits, sx, pl.bias,
+                                 l.stride, ws, self.status, out=y)
+        if l.kind == "bos_kv" and l.a_bits == 8:
+            return mixdq.crossattn_kv(x, pl.packed, l.N, l.w_bits, pl.w_scale, sx, pl.bos_out, ws, self.status,
+                                      out=y)
+        x2 = x.reshape(-1, x.shape[-1])
+        return mixdq.linear(x2, pl.packed, l.N, l.w_bits, pl.w_scale, pl.w_zero, l.a_bits, sx, pl.bias, ws,
+                            self.status, out=y.reshape(-1, l.N))
+
+    def step(self, subset=None):
+        for pl in (self.layers if subset is None else subset):
+            self.run_layer(pl)
+
+    # ------------------------------------------------------------------ accounting
+    def total_ops(self, subset=None) -> int:
+        return sum(pl.spec.ops(self.batch) for pl in (self.layers if subset is None else subset))
+
+    def packed_weight_bytes(self) -> int:
+        return sum(pl.packed.numel() for pl in self.layers)
+
+    def algorithmic_bytes(self, pl: PackedLayer) -> int:
+        """Packed weights + per-channel params + input once + output once + bias."""
+        l = pl.spec
+        x, y = self.x[pl.x_key], self.y[pl.y_key]
+        params = l.N * (4 if pl.w_zero is None else 8)
+        return pl.packed.numel() + params + x.numel() * 2 + y.numel() * 2 + (0 if pl.bias is None else l.N * 2)
+
+    def uses_tensor_int8(self, pl: PackedLayer) -> bool:
+        """True when the layer runs on the tcgen05 int8 engine (not the plain corner kernel)."""
+        l = pl.spec
+        if l.a_bits != 8:
+            return False
+        unit = l.Cin if l.kind == "conv3x3" else l.K
+        return unit % 16 == 0 and l.N >= 16
