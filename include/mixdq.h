@@ -180,6 +180,28 @@ int mixdq_crossattn_kv_acc_i32(const void* text_emb, int64_t B, int64_t Kt, cons
                                void* workspace, size_t workspace_bytes, int32_t* status,
                                void* stream);
 
+/*
+ * (No counterpart in the paper: an addition for hosts that cannot allocate.)
+ * mixdq_linear with act_bits = 8 for callers that have no device memory to give as a
+ * workspace -- a process whose memory manager owns the whole GPU, code embedded in another
+ * framework's allocator, or a loop that cannot afford the device-wide synchronization of
+ * cudaMalloc.  The split-reduction scratch is a fixed array of
+ * mixdq_static_scratch_bytes() bytes (8 MiB) inside the library image; every GPU that loads
+ * the library holds it until the process exits.  The call allocates and frees nothing.
+ *   - A problem whose scratch need (mixdq_workspace_bytes) exceeds the array is rejected with
+ *     MIXDQ_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls share the one array and each call clears the part it uses first, so two
+ *     calls that can overlap on the GPU (different streams) race: serialize them.
+ * Arguments as in mixdq_linear; weights symmetric, w_bits in {4, 8}.
+ */
+size_t mixdq_static_scratch_bytes(void);
+int mixdq_linear_a8_static_scratch(const void* X, int64_t M, int64_t K, int64_t ldx,
+                                   const void* packed_W, int64_t N, int w_bits, const float* w_scale,
+                                   const float* act_scale, const void* bias, void* Y, int32_t* status,
+                                   void* stream);
+
 #ifdef __cplusplus
 }
 #endif

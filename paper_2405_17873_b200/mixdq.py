@@ -42,6 +42,9 @@ _SIGNATURES = {
                              _sz, _vp, _vp]),
     "mixdq_crossattn_kv": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "mixdq_crossattn_kv_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_static_scratch_bytes": (_sz, []),
+    "mixdq_linear_a8_static_scratch": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp,
+                                              _vp]),
 }
 
 EXPORTS = tuple(_SIGNATURES)
@@ -236,3 +239,19 @@ def crossattn_kv_acc_i32(text_emb, packed_W, N: int, w_bits: int, act_scale, wor
                                           _ptr(acc), wp, wb, _ptr(status), _stream()),
          "mixdq_crossattn_kv_acc_i32")
     return acc
+
+
+def static_scratch_bytes() -> int:
+    return lib().mixdq_static_scratch_bytes()
+
+
+def linear_a8_static_scratch(X, packed_W, N: int, w_bits: int, w_scale, act_scale, bias=None, status=None,
+                             out=None):
+    """W8A8 / W4A8 linear whose scratch is the library's built-in array: for callers that cannot
+    allocate device memory.  The output tensor is still the caller's (``out``, or a fresh one here)."""
+    M, K = X.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=X.device)
+    _chk(lib().mixdq_linear_a8_static_scratch(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits,
+                                              _ptr(w_scale), _ptr(act_scale), _ptr(bias), _ptr(Y), _ptr(status),
+                                              _stream()), "mixdq_linear_a8_static_scratch")
+    return Y
