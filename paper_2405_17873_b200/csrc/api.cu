@@ -100,6 +100,7 @@ int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, cons
         p.Ho = static_cast<int>(Ho);
         p.Wo = static_cast<int>(Wo);
         p.stride = stride;
+        p.batch = static_cast<int>(B);
         p.act_scale = act_scale;
         p.w_scale = w_scale;
         p.bias = static_cast<const __half*>(bias);
@@ -181,7 +182,19 @@ extern "C" int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_b
     if (!out || rows <= 0 || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
     if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
-    *out = (act_bits == 8) ? i8::workspace_bytes(rows, N) : 0;
+    *out = (act_bits == 8) ? i8::workspace_bytes(rows, N, rows, K) : 0;
+    return MIXDQ_OK;
+}
+
+extern "C" int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int stride,
+                                             int w_bits, int act_bits, size_t* out)
+{
+    if (!out || B <= 0 || H <= 0 || W <= 0 || Cin <= 0 || Cout <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (stride != 1 && stride != 2) return MIXDQ_ERR_INVALID_ARG;
+    if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * H * W, Cin) : 0;
     return MIXDQ_OK;
 }
 

@@ -49,6 +49,10 @@ int encode_tmap_2d_u8(CUtensorMap* map, const void* base, uint64_t row_bytes, ui
 int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows,
                        uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows);
 
+// 4-D byte tensor map with the 128-byte swizzle (NHWC int8 image: dims {C, W, H, B}).
+int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
+                      const uint32_t box[4]);
+
 #ifdef __CUDACC__
 
 // ---------------------------------------------------------------- device helpers
@@ -126,6 +130,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
         "%3}], [%4];" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
+        "%3, %4, %5}], [%6];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
 }
 

@@ -36,9 +36,17 @@ struct Params {
     int force_splits = 0;           // > 0: use exactly this many reduction splits
 };
 
-size_t workspace_bytes(int64_t rows, int64_t N);
+// Scratch of the fused kernel's split reduction (tickets + int32 partial sums).
+size_t split_scratch_bytes(int64_t rows, int64_t N);
+// Scratch of the two-kernel path: the int8 copy of the activations.
+size_t tma_scratch_bytes(int64_t in_rows, int64_t row_len);
+// Whole workspace of a linear layer (conv: pass the input pixel count and Cin).
+size_t workspace_bytes(int64_t out_rows, int64_t N, int64_t in_rows, int64_t row_len);
 int run(Params p, int amode, const void* packed, int w_bits, void* workspace, size_t ws_bytes,
         cudaStream_t stream);
+// Two-kernel path (quantize once, then a TMA-fed GEMM); see i8_tma.cu.
+bool tma_path_ok(const Params& p, int amode, int w_bits);
+int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream);
 
 }  // namespace i8
 

@@ -15,6 +15,9 @@
 //
 // int4 weights are expanded to (16 * q) by placing the nibble in the high half of the
 // byte, which needs no sign extension; the factor 16 is divided out exactly afterwards.
+#include <cstdlib>
+#include <cstring>
+
 #include "common.cuh"
 #include "engines.h"
 
@@ -519,10 +522,29 @@ int launch_mode(const Params& p, const void* packed, int64_t pitch, int splits, 
     return launch_tc<128, 4, W4, AMODE>(p, packed, pitch, splits, stream);
 }
 
-size_t workspace_bytes(int64_t rows, int64_t N)
+size_t split_scratch_bytes(int64_t rows, int64_t N)
 {
     const int64_t tiles = ceil_div(rows, BM) * ceil_div(N, 128);
     return static_cast<size_t>(round_up(tiles * 4, 256) + round_up(rows, BM) * round_up(N, 128) * 4);
+}
+
+size_t workspace_bytes(int64_t out_rows, int64_t N, int64_t in_rows, int64_t row_len)
+{
+    return split_scratch_bytes(out_rows, N) + tma_scratch_bytes(in_rows, row_len);
+}
+
+// MIXDQ_I8_PATH=fused|tma overrides the choice between the fused single kernel and the
+// quantize-then-GEMM pair (diagnostics and tuning; unset = automatic).
+static int path_override()
+{
+    static int v = -1;
+    if (v < 0) {
+        const char* e = getenv("MIXDQ_I8_PATH");
+        v = 0;
+        if (e && !strcmp(e, "fused")) v = 1;
+        if (e && !strcmp(e, "tma")) v = 2;
+    }
+    return v;
 }
 
 int run(Params p, int amode, const void* packed, int w_bits, void* workspace, size_t ws_bytes,
@@ -533,6 +555,18 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     p.k_blocks = static_cast<int>(ceil_div(p.K, BK));
     const bool tc_ok = (amode == A_CONV3 ? (p.Cin % 16 == 0) : (p.K % 16 == 0)) && p.N >= 16 &&
                        (p.ldx % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 15) == 0);
+
+    // two-kernel path: needs room for the int8 activations behind the split-reduction scratch
+    const size_t split_bytes = split_scratch_bytes(p.M, p.N);
+    const int64_t in_rows = amode == A_CONV3 ? static_cast<int64_t>(p.batch) * p.H * p.W : p.M;
+    const int64_t row_len = amode == A_CONV3 ? p.Cin : p.K;
+    const bool tma_room = workspace && ws_bytes >= split_bytes + tma_scratch_bytes(in_rows, row_len);
+    if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1) {
+        const bool big = amode == A_CONV3 || p.M >= 64;
+        if (big || path_override() == 2)
+            return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
+    }
+
     if (!tc_ok) {
         const long long total = static_cast<long long>(p.M) * p.N;
         const unsigned grid = static_cast<unsigned>(ceil_div(total, 128));
@@ -545,13 +579,13 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     // split the reduction across CTAs when the output tiles alone cannot fill the GPU
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, 128);
     int splits = 1;
-    if (workspace && ws_bytes >= workspace_bytes(p.M, p.N) && tiles < 96 && p.k_blocks >= 8) {
+    if (workspace && ws_bytes >= split_bytes && tiles < 96 && p.k_blocks >= 8) {
         splits = static_cast<int>(148 / tiles);
         if (splits > p.k_blocks / 4) splits = p.k_blocks / 4;
         if (splits < 1) splits = 1;
     }
     if (p.force_splits > 0) {
-        if (p.force_splits > 1 && !(workspace && ws_bytes >= workspace_bytes(p.M, p.N))) return MIXDQ_ERR_WORKSPACE;
+        if (p.force_splits > 1 && !(workspace && ws_bytes >= split_bytes)) return MIXDQ_ERR_WORKSPACE;
         splits = p.force_splits > p.k_blocks ? p.k_blocks : p.force_splits;
     }
     if (splits > 1) {

@@ -1,0 +1,522 @@
+// Two-kernel form of the W8A8 / W4A8 engine for layers large enough to be bound by the
+// tensor cores or by on-chip bandwidth rather than by launch latency:
+//   1. quant_kernel: the per-tensor fp16 -> int8 activation quantization, once per layer
+//      (the fused engine in i8_gemm.cu repeats it for every tile column and, for a 3x3 conv,
+//      for every filter tap);
+//   2. tma_gemm_kernel: both operands arrive by TMA in the 128-byte-swizzled layout that
+//      tcgen05.mma reads, so the main loop does no arithmetic of its own for int8 weights and
+//      only the nibble expansion for int4 weights.  A 3x3 convolution is an implicit GEMM:
+//      the A tile of filter tap (kh, kw) is a 4-D box of the int8 NHWC image shifted by
+//      (kh - 1, kw - 1), and the zero padding is TMA's out-of-bounds fill.
+// Output tile 128 x BN (BN = 128 or 256), 128-wide k-blocks, accumulators in tensor memory.
+#include "common.cuh"
+#include "engines.h"
+
+namespace mixdq {
+namespace i8 {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 128;
+constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: fma(x, inv, magic) rounds x * inv to nearest even
+
+__device__ __forceinline__ uint32_t q4(float a, float b, float c, float d, float inv)
+{
+    const float lo = kMagic - 127.f, hi = kMagic + 127.f;
+    const uint32_t qa = __float_as_uint(fminf(fmaxf(fmaf(a, inv, kMagic), lo), hi));
+    const uint32_t qb = __float_as_uint(fminf(fmaxf(fmaf(b, inv, kMagic), lo), hi));
+    const uint32_t qc = __float_as_uint(fminf(fmaxf(fmaf(c, inv, kMagic), lo), hi));
+    const uint32_t qd = __float_as_uint(fminf(fmaxf(fmaf(d, inv, kMagic), lo), hi));
+    return __byte_perm(__byte_perm(qa, qb, 0x0040), __byte_perm(qc, qd, 0x0040), 0x5410);
+}
+
+// One thread per 16 consecutive elements of a row.  bos != 0: output row r reads input row
+// (r / 76) * 77 + r % 76 + 1, i.e. the BOS token of every prompt is left out.
+__global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long long rows, int K, int bos,
+                             const float* __restrict__ act_scale, int8_t* __restrict__ out)
+{
+    const int cpr = K >> 4;
+    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    if (idx >= rows * cpr) return;
+    const long long r = idx / cpr;
+    const int c = static_cast<int>(idx - r * cpr);
+    long long src_row = r;
+    if (bos) {
+        const long long prompt = r / (MIXDQ_TOKENS_PER_PROMPT - 1);
+        src_row = prompt * MIXDQ_TOKENS_PER_PROMPT + (r - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1)) + 1;
+    }
+    const float inv = __fdiv_rn(1.f, __ldg(act_scale));
+    const uint4* src = reinterpret_cast<const uint4*>(X + src_row * ldx + c * 16);
+    const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
+    const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
+    const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
+    float2 f[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[j] = __half22float2(h0[j]);
+        f[4 + j] = __half22float2(h1[j]);
+    }
+    uint4 o;
+    o.x = q4(f[0].x, f[0].y, f[1].x, f[1].y, inv);
+    o.y = q4(f[2].x, f[2].y, f[3].x, f[3].y, inv);
+    o.z = q4(f[4].x, f[4].y, f[5].x, f[5].y, inv);
+    o.w = q4(f[6].x, f[6].y, f[7].x, f[7].y, inv);
+    *reinterpret_cast<uint4*>(out + r * K + c * 16) = o;
+}
+
+// Barrier over all threads of all CTAs of the cluster (hardware barrier, not a spin).
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// 16 bytes from the shared memory of CTA `cta_rank` of this cluster, at this CTA's offset `addr`.
+__device__ __forceinline__ int4 ld_cluster_v4(uint32_t addr, int cta_rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(cta_rank));
+    int4 v;
+    asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(remote)
+                 : "memory");
+    return v;
+}
+
+struct TmaParams {
+    int M, N, k_blocks;
+    int conv;     // 0: A is a [M, K] int8 matrix; 1: A is an int8 NHWC image gathered per filter tap
+    int cblocks;  // conv: k-blocks per filter tap = ceil(Cin / 128)
+    int Cin, HoWo, Wo;
+    int bos;      // output row m maps to row (m / 76) * 77 + m % 76 + 1 of Y
+    int batch;
+    const float* act_scale;
+    const float* w_scale;
+    const __half* bias;
+    const __half* bos_out;
+    __half* Y;
+    long long ldy;
+    int32_t* acc_out;
+    int32_t* status;
+};
+
+template <int BN, int STAGES, bool W4>
+struct TmaSmem {
+    static constexpr int A_BYTES = BM * BK;
+    static constexpr int B_BYTES = BN * BK;
+    static constexpr int STG_BYTES = W4 ? BN * (BK / 2) : 0;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+    static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
+    static constexpr int OFF_BARS = OFF_STG + STAGES * STG_BYTES;
+    static constexpr int NUM_BARS = 3 * STAGES + 1;
+    static constexpr int OFF_COMB = OFF_BARS + NUM_BARS * 8;
+    static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
+    static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
+    static constexpr int TOTAL = OFF_MISC + 64 + 1024;
+    static constexpr int THREADS = W4 ? 320 : 192;
+};
+
+template <int BN, int STAGES, bool W4>
+__global__ void __launch_bounds__(TmaSmem<BN, STAGES, W4>::THREADS, 1)
+tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                const TmaParams p)
+{
+    using L = TmaSmem<BN, STAGES, W4>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    uint8_t* sA = smem + L::OFF_A;
+    uint8_t* sB = smem + L::OFF_B;
+    uint8_t* sStg = smem + L::OFF_STG;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
+    float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
+    float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM;
+    // the CTAs of a cluster (gridDim.z of them) share one output tile and split the reduction
+    const int splits = gridDim.z, rank = blockIdx.z;
+    const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * rank) / splits);
+    const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (rank + 1)) / splits);
+    const int nkb = kb_end - kb_begin;
+
+    const uint32_t bar_full = smem_u32(bars);                 // TMA bytes of the stage have landed
+    const uint32_t bar_unpacked = smem_u32(bars + STAGES);    // W4: nibbles expanded into the B tile
+    const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);   // MMAs reading the stage have finished
+    const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_unpacked + 8 * s, 4);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_accum, 1);
+        *s_abort = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(s_tmem), BN);
+        tmem_relinquish();
+    }
+    if (warp >= 2 && warp < 6) {
+        const float sx = __ldg(p.act_scale);
+        for (int j = tid - 64; j < BN; j += 128) {
+            const int n = n0 + j;
+            float comb = 0.f, b = 0.f;
+            if (n < p.N && p.w_scale) {
+                comb = sx * __ldg(p.w_scale + n);
+                if (W4) comb *= 0.0625f;
+                if (p.bias) b = __half2float(p.bias[n]);
+            }
+            s_comb[j] = comb;
+            s_bias[j] = b;
+        }
+        if (p.bos && p.Y && blockIdx.y == 0) {
+            // row 0 of every prompt: the stored floating-point BOS projection, copied as is
+            for (int idx = tid - 64; idx < p.batch * BN; idx += 128) {
+                const int b = idx / BN, j = idx - b * BN;
+                if (n0 + j < p.N)
+                    p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            int img_b = 0, ho0 = 0, wo0 = 0;
+            if (p.conv) {
+                img_b = m0 / p.HoWo;
+                const int rem = m0 - img_b * p.HoWo;
+                ho0 = rem / p.Wo;
+                wo0 = rem - ho0 * p.Wo;
+            }
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % STAGES;
+                const uint32_t round = static_cast<uint32_t>(i / STAGES);
+                if (!mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort)) break;
+                mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
+                const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
+                const uint32_t dst_b = W4 ? smem_u32(sStg + s * L::STG_BYTES) : smem_u32(sB + s * L::B_BYTES);
+                const int kb = kb_begin + i;
+                if (p.conv) {
+                    const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+                    const int kh = tap / 3, kw = tap - 3 * kh;
+                    tma_load_4d(dst_a, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, bar_full + 8 * s);
+                    const int kx = tap * p.Cin + cb * BK;
+                    tma_load_2d(dst_b, &tmap_w, W4 ? kx / 2 : kx, n0, bar_full + 8 * s);
+                } else {
+                    tma_load_2d(dst_a, &tmap_a, kb * BK, m0, bar_full + 8 * s);
+                    tma_load_2d(dst_b, &tmap_w, kb * ROW_BYTES, n0, bar_full + 8 * s);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
+            bool ok = true;
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % STAGES;
+                const uint32_t round = static_cast<uint32_t>(i / STAGES);
+                ok = mbar_wait(bar_full + 8 * s, round & 1, s_abort);
+                if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, round & 1, s_abort);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint64_t a_desc = smem_desc_sw128(smem_u32(sA + s * L::A_BYTES));
+                const uint64_t b_desc = smem_desc_sw128(smem_u32(sB + s * L::B_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / 32; ++k)
+                    mma_i8_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0);
+                tc_commit(bar_empty + 8 * s);
+            }
+            if (ok) tc_commit(bar_accum);
+        }
+        __syncwarp();
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue, part 1
+        // accumulators: tensor memory -> registers -> shared memory (the pipeline buffers are
+        // free once the last MMA has completed), 16-byte chunks XOR-swizzled by row
+        bool ok = mbar_wait(bar_accum, 0, s_abort);
+        tc_fence_after_sync();
+        const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        if (go) {
+            uint8_t* prow = smem + row * (BN * 4);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int chunk = (c0 >> 2) + j;
+                    *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
+                        make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                }
+            }
+        }
+    } else if (W4) {
+        // ------------------------------------------------------------ int4 -> int8 (x16) expansion
+        const int ut = tid - 192;
+        for (int i = 0; i < nkb; ++i) {
+            const int s = i % STAGES;
+            const uint32_t round = static_cast<uint32_t>(i / STAGES);
+            if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
+            const uint8_t* stg = sStg + s * L::STG_BYTES;
+            uint8_t* b_stage = sB + s * L::B_BYTES;
+#pragma unroll 4
+            for (int t = 0; t < (BN * 4) / 128; ++t) {
+                const int task = ut + t * 128;
+                const int r = task >> 2, j = task & 3;
+                const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
+                uint4 c0, c1;
+                c0.x = (w.x << 4) & 0xF0F0F0F0u;
+                c0.y = w.x & 0xF0F0F0F0u;
+                c0.z = (w.y << 4) & 0xF0F0F0F0u;
+                c0.w = w.y & 0xF0F0F0F0u;
+                c1.x = (w.z << 4) & 0xF0F0F0F0u;
+                c1.y = w.z & 0xF0F0F0F0u;
+                c1.z = (w.w << 4) & 0xF0F0F0F0u;
+                c1.w = w.w & 0xF0F0F0F0u;
+                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
+                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
+        }
+    }
+
+    // ---------------------------------------------------------------- epilogue, part 2
+    // Every CTA of the cluster holds partial sums of the same tile in its shared memory.  CTA
+    // `rank` adds up rows [rank * 128 / splits, ...) over all of them (integer adds: exact,
+    // order-free), dequantizes and stores; threads run along a row so stores coalesce.
+    __syncthreads();
+    if (splits > 1) cluster_sync_all();
+    if (warp >= 2 && warp < 6 && !*s_abort) {
+        const int et = tid - 64;
+        const int rows_per = BM / splits;
+        constexpr int CHUNKS = BN / 4;
+        const bool vec = ((p.ldy & 3) == 0);
+        for (int item = et; item < rows_per * CHUNKS; item += 128) {
+            const int rl = item / CHUNKS, chunk = item - rl * CHUNKS;
+            const int row = rank * rows_per + rl;
+            const int m = m0 + row, n = n0 + chunk * 4;
+            if (m >= p.M || n >= p.N) continue;
+            const uint32_t off = smem_u32(smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4));
+            int4 acc = make_int4(0, 0, 0, 0);
+            if (splits == 1) {
+                acc = *reinterpret_cast<const int4*>(smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4));
+            } else {
+                for (int q = 0; q < splits; ++q) {
+                    const int4 v = ld_cluster_v4(off, q);
+                    acc.x += v.x;
+                    acc.y += v.y;
+                    acc.z += v.z;
+                    acc.w += v.w;
+                }
+            }
+            if (p.acc_out) {
+                int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
+                const int a[4] = {acc.x, acc.y, acc.z, acc.w};
+                for (int j = 0; j < 4; ++j)
+                    if (n + j < p.N) dst[j] = W4 ? (a[j] >> 4) : a[j];
+            }
+            if (p.Y) {
+                long long out_row = m;
+                if (p.bos) {
+                    const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                    out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                              (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+                }
+                const int c = chunk * 4;
+                const float4 cb = *reinterpret_cast<const float4*>(s_comb + c);
+                const float4 bb = *reinterpret_cast<const float4*>(s_bias + c);
+                __half2 h[2];
+                h[0] = __floats2half2_rn(fmaf(static_cast<float>(acc.x), cb.x, bb.x),
+                                         fmaf(static_cast<float>(acc.y), cb.y, bb.y));
+                h[1] = __floats2half2_rn(fmaf(static_cast<float>(acc.z), cb.z, bb.z),
+                                         fmaf(static_cast<float>(acc.w), cb.w, bb.w));
+                __half* dst = p.Y + out_row * p.ldy + n;
+                if (vec && n + 4 <= p.N) {
+                    *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
+                } else {
+                    const __half* hs = reinterpret_cast<const __half*>(h);
+                    for (int j = 0; j < 4; ++j)
+                        if (n + j < p.N) dst[j] = hs[j];
+                }
+            }
+        }
+    }
+    if (*s_abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (tid == 0 && p.status) atomicExch(p.status, MIXDQ_ERR_TIMEOUT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's shared memory
+    if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+template <int BN, int STAGES, bool W4>
+int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp, int splits, cudaStream_t stream)
+{
+    using L = TmaSmem<BN, STAGES, W4>;
+    auto kernel = tma_gemm_kernel<BN, STAGES, W4>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
+                       static_cast<unsigned>(splits));
+    cfg.blockDim = dim3(L::THREADS);
+    cfg.dynamicSmemBytes = L::TOTAL;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = static_cast<unsigned>(splits);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MIXDQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tw, tp));
+    return MIXDQ_OK;
+}
+
+// Reduction splits (cluster size): enough CTAs to cover the SMs, at least 4 k-blocks each.
+int pick_splits(int64_t tiles, int k_blocks)
+{
+    int s = 1;
+    while (s < 8 && tiles * (2 * s) <= 160 && k_blocks / (2 * s) >= 4) s *= 2;
+    return s;
+}
+
+}  // namespace
+
+size_t tma_scratch_bytes(int64_t in_rows, int64_t K_row) { return static_cast<size_t>(round_up(in_rows * K_row, 256)); }
+
+// Box of 128 consecutive output pixels as (Wb, Hb, Bb) in image coordinates; false when the
+// image size does not tile that way.
+static bool conv_box(int Ho, int Wo, int* Wb, int* Hb, int* Bb)
+{
+    if (Wo >= BM) {
+        if (Wo % BM) return false;
+        *Wb = BM; *Hb = 1; *Bb = 1;
+        return true;
+    }
+    if (BM % Wo) return false;
+    const int rows = BM / Wo;
+    if (Ho >= rows) {
+        if (Ho % rows) return false;
+        *Wb = Wo; *Hb = rows; *Bb = 1;
+        return true;
+    }
+    if (rows % Ho) return false;
+    *Wb = Wo; *Hb = Ho; *Bb = rows / Ho;
+    return true;
+}
+
+bool tma_path_ok(const Params& p, int amode, int w_bits)
+{
+    if (p.N < 16) return false;
+    if (amode == A_CONV3) {
+        int a, b, c;
+        if (p.stride != 1 || p.Cin % 32 != 0) return false;
+        return conv_box(p.Ho, p.Wo, &a, &b, &c);
+    }
+    (void)w_bits;
+    return p.K % 16 == 0 && p.ldx % 8 == 0 && (reinterpret_cast<uintptr_t>(p.X) & 15) == 0;
+}
+
+int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream)
+{
+    const bool w4 = w_bits == 4;
+    const int64_t pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
+    int8_t* aq = static_cast<int8_t*>(scratch);
+
+    // 1. quantize the activations once
+    const bool conv = amode == A_CONV3;
+    const long long in_rows = conv ? static_cast<long long>(p.batch) * p.H * p.W : p.M;
+    const int row_len = conv ? p.Cin : p.K;
+    const long long ldx = conv ? p.Cin : p.ldx;
+    const long long tasks = in_rows * (row_len / 16);
+    quant_kernel<<<static_cast<unsigned>(ceil_div(tasks, 256)), 256, 0, stream>>>(
+        p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, aq);
+    int rc = check_launch();
+    if (rc != MIXDQ_OK) return rc;
+
+    // 2. tensor maps
+    CUtensorMap ta, tw;
+    TmaParams tp{};
+    tp.M = p.M;
+    tp.N = p.N;
+    tp.bos = amode == A_BOS;
+    tp.batch = p.batch;
+    tp.act_scale = p.act_scale;
+    tp.w_scale = p.w_scale;
+    tp.bias = p.bias;
+    tp.bos_out = p.bos_out;
+    tp.Y = p.Y;
+    tp.ldy = p.ldy;
+    tp.acc_out = p.acc_out;
+    tp.status = p.status;
+    if (conv) {
+        int Wb, Hb, Bb;
+        if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
+        const uint64_t dims[4] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.W),
+                                  static_cast<uint64_t>(p.H), static_cast<uint64_t>(p.batch)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.Cin) * p.W,
+                                     static_cast<uint64_t>(p.Cin) * p.W * p.H};
+        const uint32_t box[4] = {BK, static_cast<uint32_t>(Wb), static_cast<uint32_t>(Hb), static_cast<uint32_t>(Bb)};
+        rc = encode_tmap_4d_u8(&ta, aq, dims, strides, box);
+        tp.conv = 1;
+        tp.cblocks = static_cast<int>(ceil_div(p.Cin, BK));
+        tp.Cin = p.Cin;
+        tp.HoWo = p.Ho * p.Wo;
+        tp.Wo = p.Wo;
+        tp.k_blocks = 9 * tp.cblocks;
+    } else {
+        rc = encode_tmap_2d_u8(&ta, aq, static_cast<uint64_t>(p.K), static_cast<uint64_t>(p.M),
+                               static_cast<uint64_t>(p.K), BK, BM, true);
+        tp.k_blocks = static_cast<int>(ceil_div(p.K, BK));
+    }
+    if (rc != MIXDQ_OK) return rc;
+    const bool wide = p.N >= 1024 || p.N % 256 == 0;
+    const uint32_t bn = wide ? 256 : 128;
+    if (w4)
+        rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, bn, false);
+    else
+        rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(p.K), p.N, pitch, BK, bn, true);
+    if (rc != MIXDQ_OK) return rc;
+
+    int splits = pick_splits(ceil_div(p.M, BM) * ceil_div(p.N, bn), tp.k_blocks);
+    if (p.force_splits > 0) {
+        splits = 1;
+        while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;
+    }
+    if (wide)
+        return w4 ? launch_tma<256, 3, true>(ta, tw, tp, splits, stream)
+                  : launch_tma<256, 4, false>(ta, tw, tp, splits, stream);
+    return w4 ? launch_tma<128, 4, true>(ta, tw, tp, splits, stream)
+              : launch_tma<128, 4, false>(ta, tw, tp, splits, stream);
+}
+
+}  // namespace i8
+}  // namespace mixdq

@@ -54,7 +54,7 @@ extern "C" int mixdq_linear_a8_static_scratch(const void* X, int64_t M, int64_t 
         return MIXDQ_ERR_INVALID_ARG;
     if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(packed_W) & 15) return MIXDQ_ERR_ALIGNMENT;
-    const size_t need = i8::workspace_bytes(M, N);
+    const size_t need = i8::workspace_bytes(M, N, M, K);
     if (need > kStaticScratchBytes) return MIXDQ_ERR_WORKSPACE;  // problem too large for the fixed array
     void* scratch = nullptr;
     int rc = scratch_address(&scratch);

@@ -65,4 +65,27 @@ int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64
     return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;
 }
 
+
+int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
+                      const uint32_t box[4])
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return MIXDQ_ERR_CUDA;
+    if (reinterpret_cast<uintptr_t>(base) & 15) return MIXDQ_ERR_ALIGNMENT;
+    cuuint64_t d[4], st[3];
+    cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
+    for (int i = 0; i < 4; ++i) {
+        d[i] = dims[i];
+        b[i] = box[i];
+    }
+    for (int i = 0; i < 3; ++i) {
+        if (strides_bytes[i] & 15) return MIXDQ_ERR_ALIGNMENT;
+        st[i] = strides_bytes[i];
+    }
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), d, st, b, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;
+}
+
 }  // namespace mixdq

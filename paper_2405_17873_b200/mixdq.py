@@ -31,6 +31,7 @@ _SIGNATURES = {
     "mixdq_act_absmax": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp]),
     "mixdq_act_scale_from_absmax": (_int, [_vp, _vp, _vp]),
     "mixdq_workspace_bytes": (_int, [_i64, _i64, _i64, _int, _int, C.POINTER(_sz)]),
+    "mixdq_conv3x3_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, _int, _int, _int, C.POINTER(_sz)]),
     "mixdq_linear": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp, _sz,
                             _vp, _vp]),
     "mixdq_linear_acc_i32": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _sz, _vp, _vp]),
@@ -100,6 +101,14 @@ def packed_bytes(N: int, K: int, bits: int, layout: int = LAYOUT_DEVICE) -> int:
 def workspace_bytes(rows: int, N: int, K: int, w_bits: int, act_bits: int) -> int:
     out = _sz(0)
     _chk(lib().mixdq_workspace_bytes(rows, N, K, w_bits, act_bits, C.byref(out)), "mixdq_workspace_bytes")
+    return out.value
+
+
+def conv3x3_workspace_bytes(B: int, H: int, W: int, Cin: int, Cout: int, stride: int, w_bits: int,
+                            act_bits: int) -> int:
+    out = _sz(0)
+    _chk(lib().mixdq_conv3x3_workspace_bytes(B, H, W, Cin, Cout, stride, w_bits, act_bits, C.byref(out)),
+         "mixdq_conv3x3_workspace_bytes")
     return out.value
 
 

@@ -96,8 +96,14 @@ class UNetSweep:
                     e0 = self.x[xk][0, 0].to(torch.float32)
                     bos = (W.to(torch.float32) @ e0).to(torch.float16).contiguous()
             self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk))
-            rows = yk[0] * (yk[1] if len(yk) > 2 else 1) * (yk[2] if len(yk) > 3 else 1)
-            max_ws = max(max_ws, mixdq.workspace_bytes(rows, l.N, l.K, l.w_bits, l.a_bits))
+            if l.kind == "conv3x3":
+                need = mixdq.conv3x3_workspace_bytes(self.batch, l.H, l.H, l.Cin, l.N, l.stride, l.w_bits, l.a_bits)
+            else:
+                rows = yk[0] * (yk[1] if len(yk) > 2 else 1) * (yk[2] if len(yk) > 3 else 1)
+                if l.kind == "bos_kv" and l.a_bits == 8:
+                    rows = self.batch * (synth.TOKENS_PER_PROMPT - 1)
+                need = mixdq.workspace_bytes(rows, l.N, l.K, l.w_bits, l.a_bits)
+            max_ws = max(max_ws, need)
         self.workspace = mixdq.new_workspace(max_ws, self.device)
         torch.cuda.synchronize()
 

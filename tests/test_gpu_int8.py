@@ -31,25 +31,33 @@ def _run_linear(X, W, b, bits, use_ws):
     assert np.array_equal(host(acc), acc_ref)
     assert_close(host(y), y_ref)
     if ws is not None:
-        assert not bool(ws.any())          # the scratch is left zero-filled
+        # the part of the scratch that must be zero on entry is left zero-filled
+        n_zero = ws.numel() - (M * K + 255) // 256 * 256
+        assert n_zero > 0 and not bool(ws[:n_zero].any())
 
 
-def test_single_linear_w8a8_seed0():
+@pytest.mark.parametrize("use_ws", [False, True])
+def test_single_linear_w8a8_seed0(use_ws):
     X, W, b = synth.single_linear(seed=0)
-    _run_linear(X, W, b, 8, False)
+    _run_linear(X, W, b, 8, use_ws)
 
 
+# without a workspace the fused kernel runs; with one, layers of 64 rows or more take the
+# quantize-once + TMA-fed GEMM pair (128- or 256-wide tiles, cluster split of the reduction)
+@pytest.mark.parametrize("use_ws", [False, True])
 @pytest.mark.parametrize("bits", [8, 4])
-@pytest.mark.parametrize("M,K,N", [(1, 16, 16), (77, 336, 200), (300, 320, 328), (129, 1040, 136), (256, 2048, 24)])
-def test_linear_ragged_tiles(bits, M, K, N):
+@pytest.mark.parametrize("M,K,N", [(1, 16, 16), (77, 336, 200), (300, 320, 328), (129, 1040, 136), (256, 2048, 24),
+                                   (200, 272, 1032), (136, 2064, 520)])
+def test_linear_ragged_tiles(bits, M, K, N, use_ws):
     g = synth.normal_f16((M, K), 1.0, seed=M + K)
     W = synth.normal_f16((N, K), 0.02, seed=N + K + 1)
     b = synth.normal_f16((N,), 0.01, seed=N)
-    _run_linear(g, W, b, bits, False)
+    _run_linear(g, W, b, bits, use_ws)
 
 
 @pytest.mark.parametrize("bits", [8, 4])
-@pytest.mark.parametrize("M,K,N", [(256, 5120, 320), (130, 1280, 200), (512, 4096, 136)])
+@pytest.mark.parametrize("M,K,N", [(256, 5120, 320), (130, 1280, 200), (512, 4096, 136), (40, 4096, 136),
+                                   (16, 2560, 1300), (256, 5120, 1280)])
 def test_linear_split_reduction(bits, M, K, N):
     g = synth.normal_f16((M, K), 1.0, seed=M + K + 7)
     W = synth.normal_f16((N, K), 0.02, seed=N + K + 8)
@@ -72,9 +80,10 @@ def test_ffn_outlier_channels():
     _run_linear(X, W, None, 8, True)
 
 
+@pytest.mark.parametrize("use_ws", [False, True])
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("B,N", [(1, 64), (3, 200)])
-def test_bos_aware_kv(bits, B, N):
+def test_bos_aware_kv(bits, B, N, use_ws):
     E = synth.text_embedding(B, seed=4000)
     W = synth.kv_weight(N, seed=4100 + N)
     s_ref, _, codes = oracle_weights(W, bits, True)
@@ -87,7 +96,7 @@ def test_bos_aware_kv(bits, B, N):
     sx = mixdq.act_scale(Ed.reshape(-1, E.shape[-1]), skip_rows_mod=77)
     assert host(sx)[0] == sx_ref
     st = status_word()
-    ws = workspace_for(B * 76, N, 2048, bits)
+    ws = workspace_for(B * 76, N, 2048, bits) if use_ws else None
     acc = mixdq.crossattn_kv_acc_i32(Ed, packed, N, bits, sx, workspace=ws, status=st)
     y = mixdq.crossattn_kv(Ed, packed, N, bits, s, sx, dev(bos), workspace=ws, status=st)
     torch.cuda.synchronize()
@@ -105,10 +114,13 @@ def test_bos_aware_kv(bits, B, N):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("use_ws", [False, True])
 @pytest.mark.parametrize("B,H,W,Cin,Cout,stride", [(1, 8, 8, 16, 16, 1), (2, 12, 10, 32, 48, 1),
                                                     (2, 12, 10, 32, 48, 2), (1, 16, 16, 320, 136, 1),
-                                                    (3, 9, 7, 48, 24, 2)])
-def test_conv3x3(bits, B, H, W, Cin, Cout, stride):
+                                                    (3, 9, 7, 48, 24, 2), (3, 8, 8, 32, 40, 1),
+                                                    (2, 32, 32, 160, 136, 1), (1, 64, 64, 32, 24, 1),
+                                                    (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2)])
+def test_conv3x3(bits, B, H, W, Cin, Cout, stride, use_ws):
     X = synth.normal_f16((B, H, W, Cin), 1.0, seed=H * W + Cin)
     Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin)
     b = synth.normal_f16((Cout,), 0.01, seed=Cout)
@@ -120,7 +132,7 @@ def test_conv3x3(bits, B, H, W, Cin, Cout, stride):
     s, _, packed = device_weights(Wt.reshape(Cout, -1), bits, True)
     sx = mixdq.act_scale(Xd)
     st = status_word()
-    ws = workspace_for(acc_ref.size // Cout, Cout, 9 * Cin, bits)
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, W, Cin, Cout, stride, bits, 8)) if use_ws else None
     acc = mixdq.conv3x3_acc_i32(Xd, packed, Cout, bits, sx, stride, workspace=ws, status=st)
     y = mixdq.conv3x3(Xd, packed, Cout, bits, s, None, 8, sx, dev(b), stride, workspace=ws, status=st)
     torch.cuda.synchronize()
