@@ -112,7 +112,7 @@ struct TmaSmem {
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
     static constexpr int OFF_BARS = OFF_STG + STAGES * STG_BYTES;
     static constexpr int NUM_BARS = 3 * STAGES + 1;
-    static constexpr int OFF_COMB = OFF_BARS + NUM_BARS * 8;
+    static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // read as float4
     static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
     static constexpr int TOTAL = OFF_MISC + 64 + 1024;
