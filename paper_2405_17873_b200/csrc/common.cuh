@@ -55,7 +55,51 @@ int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4]
 
 #ifdef __CUDACC__
 
+// Launch with programmatic dependent launch enabled (and an optional cluster along z): the
+// grid may start while the previous kernel of the stream is still draining, so its set-up
+// (barrier init, tensor-memory allocation, descriptor prefetch) overlaps that tail.  Every
+// kernel launched this way calls pdl_wait() before it touches global memory.
+template <typename... KArgs, typename... Args>
+inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                      unsigned cluster_z, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = cluster_z;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MIXDQ_ERR_CUDA;
+    }
+    return MIXDQ_OK;
+}
+
 // ---------------------------------------------------------------- device helpers
+
+// Let the next kernel of the stream begin launching (it still waits for this grid to finish
+// before reading memory).
+__device__ __forceinline__ void pdl_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Wait until every kernel this grid depends on has completed and its writes are visible.
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 
 // Spin budget of every bounded wait, in SM clock cycles (a few hundred ms).
 constexpr long long kWaitBudgetCycles = 400000000LL;

@@ -118,6 +118,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const Params p)
     const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);
     const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
 
+    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full_a + 8 * s, kFeedWarps);
@@ -134,6 +135,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const Params p)
         tmem_alloc(smem_u32(s_tmem), BN);
         tmem_relinquish();
     }
+    pdl_wait();  // set-up above overlaps the previous kernel; global memory is touched only from here
     const float sx = __ldg(p.act_scale);
     if (tid >= 64) {
         // per-column epilogue factors of this tile
@@ -435,6 +437,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const Params p)
 template <bool W4>
 __global__ void simple_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, int amode)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
     if (idx >= static_cast<long long>(p.M) * p.N) return;
     const int m = static_cast<int>(idx / p.N);
@@ -512,8 +516,7 @@ int launch_tc(const Params& p, const void* packed, int64_t pitch, int splits, cu
     }
     dim3 grid(static_cast<unsigned>(ceil_div(p.N, BN)), static_cast<unsigned>(ceil_div(p.M, BM)),
               static_cast<unsigned>(splits));
-    kernel<<<grid, kThreads, L::TOTAL, stream>>>(tmap, p);
-    return check_launch();
+    return launch_pdl(kernel, grid, dim3(kThreads), L::TOTAL, stream, 1, tmap, p);
 }
 
 template <bool W4, int AMODE>
@@ -561,20 +564,18 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     const int64_t in_rows = amode == A_CONV3 ? static_cast<int64_t>(p.batch) * p.H * p.W : p.M;
     const int64_t row_len = amode == A_CONV3 ? p.Cin : p.K;
     const bool tma_room = workspace && ws_bytes >= split_bytes + tma_scratch_bytes(in_rows, row_len);
-    if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1) {
-        const bool big = amode == A_CONV3 || p.M >= 64;
-        if (big || path_override() == 2)
-            return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
-    }
+    if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1)
+        return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
 
     if (!tc_ok) {
         const long long total = static_cast<long long>(p.M) * p.N;
         const unsigned grid = static_cast<unsigned>(ceil_div(total, 128));
+        const long long pitch_ll = pitch;
         if (w4)
-            simple_kernel<true><<<grid, 128, 0, stream>>>(static_cast<const uint8_t*>(packed), pitch, p, amode);
-        else
-            simple_kernel<false><<<grid, 128, 0, stream>>>(static_cast<const uint8_t*>(packed), pitch, p, amode);
-        return check_launch();
+            return launch_pdl(simple_kernel<true>, dim3(grid), dim3(128), 0, stream, 1,
+                              static_cast<const uint8_t*>(packed), pitch_ll, p, amode);
+        return launch_pdl(simple_kernel<false>, dim3(grid), dim3(128), 0, stream, 1,
+                          static_cast<const uint8_t*>(packed), pitch_ll, p, amode);
     }
     // split the reduction across CTAs when the output tiles alone cannot fill the GPU
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, 128);

@@ -36,6 +36,8 @@ __device__ __forceinline__ uint32_t q4(float a, float b, float c, float d, float
 __global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long long rows, int K, int bos,
                              const float* __restrict__ act_scale, int8_t* __restrict__ out)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int cpr = K >> 4;
     const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
     if (idx >= rows * cpr) return;
@@ -75,13 +77,14 @@ __device__ __forceinline__ void cluster_sync_all()
 // 16 bytes from the shared memory of CTA `cta_rank` of this cluster, at this CTA's offset `addr`.
 __device__ __forceinline__ int4 ld_cluster_v4(uint32_t addr, int cta_rank)
 {
+    // not volatile and no memory clobber: the data was published by the cluster barrier before,
+    // and the compiler may then keep several of these loads in flight
     uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(cta_rank));
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(cta_rank));
     int4 v;
-    asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "r"(remote)
-                 : "memory");
+    asm("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "r"(remote));
     return v;
 }
 
@@ -150,6 +153,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);   // MMAs reading the stage have finished
     const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
 
+    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -166,6 +170,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         tmem_alloc(smem_u32(s_tmem), BN);
         tmem_relinquish();
     }
+    pdl_wait();  // everything above is independent of earlier kernels; global memory is not
     if (warp >= 2 && warp < 6) {
         const float sx = __ldg(p.act_scale);
         for (int j = tid - 64; j < BN; j += 128) {
@@ -308,12 +313,11 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // order-free), dequantizes and stores; threads run along a row so stores coalesce.
     __syncthreads();
     if (splits > 1) cluster_sync_all();
-    if (warp >= 2 && warp < 6 && !*s_abort) {
-        const int et = tid - 64;
+    if (!*s_abort) {
         const int rows_per = BM / splits;
         constexpr int CHUNKS = BN / 4;
         const bool vec = ((p.ldy & 3) == 0);
-        for (int item = et; item < rows_per * CHUNKS; item += 128) {
+        for (int item = tid; item < rows_per * CHUNKS; item += L::THREADS) {
             const int rl = item / CHUNKS, chunk = item - rl * CHUNKS;
             const int row = rank * rows_per + rl;
             const int m = m0 + row, n = n0 + chunk * 4;
@@ -323,12 +327,15 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (splits == 1) {
                 acc = *reinterpret_cast<const int4*>(smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4));
             } else {
-                for (int q = 0; q < splits; ++q) {
-                    const int4 v = ld_cluster_v4(off, q);
-                    acc.x += v.x;
-                    acc.y += v.y;
-                    acc.z += v.z;
-                    acc.w += v.w;
+                int4 v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = (q < splits) ? ld_cluster_v4(off, q) : make_int4(0, 0, 0, 0);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    acc.x += v[q].x;
+                    acc.y += v[q].y;
+                    acc.z += v[q].z;
+                    acc.w += v[q].w;
                 }
             }
             if (p.acc_out) {
@@ -383,28 +390,16 @@ int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp
         MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
         attr_set = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
-                       static_cast<unsigned>(splits));
-    cfg.blockDim = dim3(L::THREADS);
-    cfg.dynamicSmemBytes = L::TOTAL;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = static_cast<unsigned>(splits);
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    MIXDQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ta, tw, tp));
-    return MIXDQ_OK;
+    const dim3 grid(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
+                    static_cast<unsigned>(splits));
+    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, static_cast<unsigned>(splits), ta, tw, tp);
 }
 
 // Reduction splits (cluster size): enough CTAs to cover the SMs, at least 4 k-blocks each.
 int pick_splits(int64_t tiles, int k_blocks)
 {
     int s = 1;
-    while (s < 8 && tiles * (2 * s) <= 160 && k_blocks / (2 * s) >= 4) s *= 2;
+    while (s < 8 && tiles * (2 * s) <= 160 && k_blocks / (2 * s) >= 2) s *= 2;
     return s;
 }
 
@@ -435,7 +430,6 @@ static bool conv_box(int Ho, int Wo, int* Wb, int* Hb, int* Bb)
 
 bool tma_path_ok(const Params& p, int amode, int w_bits)
 {
-    if (p.N < 16) return false;
     if (amode == A_CONV3) {
         int a, b, c;
         if (p.stride != 1 || p.Cin % 32 != 0) return false;
@@ -457,9 +451,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     const int row_len = conv ? p.Cin : p.K;
     const long long ldx = conv ? p.Cin : p.ldx;
     const long long tasks = in_rows * (row_len / 16);
-    quant_kernel<<<static_cast<unsigned>(ceil_div(tasks, 256)), 256, 0, stream>>>(
-        p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, aq);
-    int rc = check_launch();
+    int rc = launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
+                        p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, aq);
     if (rc != MIXDQ_OK) return rc;
 
     // 2. tensor maps

@@ -170,6 +170,8 @@ template <int BITS, bool SIGNED, int NT>
 __global__ void __launch_bounds__(kThreads)
 wo_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, int amode, int chunk_len)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int MB = 8 * NT;                       // tokens per CTA
     const int x_stride = chunk_len * 2 + 64;         // bytes per token row (64 mod 128: no bank conflicts)
@@ -310,8 +312,8 @@ int launch(const Params& p, int amode, const void* packed, long long pitch, cuda
         attr_set = true;
     }
     dim3 grid(static_cast<unsigned>(ceil_div(p.N, kChanPerCta)), static_cast<unsigned>(ceil_div(p.M, MB)));
-    kernel<<<grid, kThreads, smem, stream>>>(static_cast<const uint8_t*>(packed), pitch, p, amode, chunk_len);
-    return check_launch();
+    return launch_pdl(kernel, grid, dim3(kThreads), smem, stream, 1, static_cast<const uint8_t*>(packed), pitch, p,
+                      amode, chunk_len);
 }
 
 template <int BITS, bool SIGNED>

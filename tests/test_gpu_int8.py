@@ -66,6 +66,13 @@ def test_linear_split_reduction(bits, M, K, N):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+def test_few_output_channels_with_workspace(bits):
+    # 4 output channels (conv_out-like): the weight tile is mostly out-of-bounds fill
+    _run_linear(synth.normal_f16((200, 2880), 1.0, 6), synth.normal_f16((4, 2880), 0.02, 7),
+                synth.normal_f16((4,), 0.01, 8), bits, True)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
 def test_linear_corner_shapes_plain_kernel(bits):
     # reduction length not a multiple of 16, and fewer than 16 output channels
     _run_linear(synth.normal_f16((50, 36), 1.0, 1), synth.normal_f16((40, 36), 0.02, 2), None, bits, False)
@@ -119,7 +126,8 @@ def test_bos_aware_kv(bits, B, N, use_ws):
                                                     (2, 12, 10, 32, 48, 2), (1, 16, 16, 320, 136, 1),
                                                     (3, 9, 7, 48, 24, 2), (3, 8, 8, 32, 40, 1),
                                                     (2, 32, 32, 160, 136, 1), (1, 64, 64, 32, 24, 1),
-                                                    (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2)])
+                                                    (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2),
+                                                    (1, 12, 12, 256, 32, 1)])
 def test_conv3x3(bits, B, H, W, Cin, Cout, stride, use_ws):
     X = synth.normal_f16((B, H, W, Cin), 1.0, seed=H * W + Cin)
     Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin)
