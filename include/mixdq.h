@@ -189,6 +189,16 @@ int mixdq_crossattn_kv_acc_i32(const void* text_emb, int64_t B, int64_t Kt, cons
                                void* stream);
 
 /*
+ * Measurement aid (the paper reports no kernel-level throughput): every SM issues
+ * `batches` x 128 back-to-back 128x256 tensor-core MMAs on operands resident in shared
+ * memory, with no loads and no epilogue.  kind 1 = int8 -> int32 (the W8A8 / W4A8 engine's
+ * instruction), kind 0 = fp16 -> fp32.  *ops_out (HOST) receives 2 * multiply-adds issued by
+ * the whole grid; dividing by the time of the call, measured by the caller with CUDA events,
+ * gives the MMA-loop peak that benchmark fractions are quoted against.
+ */
+int mixdq_probe_mma_loop(int kind, int batches, double* ops_out, int32_t* status, void* stream);
+
+/*
  * (No counterpart in the paper: an addition for hosts that cannot allocate.)
  * mixdq_linear with act_bits = 8 for callers that have no device memory to give as a
  * workspace -- a process whose memory manager owns the whole GPU, code embedded in another

@@ -170,32 +170,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         tmem_alloc(smem_u32(s_tmem), BN);
         tmem_relinquish();
     }
-    pdl_wait();  // everything above is independent of earlier kernels; global memory is not
-    if (warp >= 2 && warp < 6) {
-        const float sx = __ldg(p.act_scale);
-        for (int j = tid - 64; j < BN; j += 128) {
-            const int n = n0 + j;
-            float comb = 0.f, b = 0.f;
-            if (n < p.N && p.w_scale) {
-                comb = sx * __ldg(p.w_scale + n);
-                if (W4) comb *= 0.0625f;
-                if (p.bias) b = __half2float(p.bias[n]);
-            }
-            s_comb[j] = comb;
-            s_bias[j] = b;
-        }
-        if (p.bos && p.Y && blockIdx.y == 0) {
-            // row 0 of every prompt: the stored floating-point BOS projection, copied as is
-            for (int idx = tid - 64; idx < p.batch * BN; idx += 128) {
-                const int b = idx / BN, j = idx - b * BN;
-                if (n0 + j < p.N)
-                    p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
-            }
-        }
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_wait();  // everything above is independent of earlier kernels; global memory is not
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
@@ -253,6 +231,31 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
         __syncwarp();
     } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue warps
+        // while the main loop runs: per-column dequantization factors of this tile, and the
+        // stored BOS rows
+        {
+            const float sx = __ldg(p.act_scale);
+            for (int j = tid - 64; j < BN; j += 128) {
+                const int n = n0 + j;
+                float comb = 0.f, b = 0.f;
+                if (n < p.N && p.w_scale) {
+                    comb = sx * __ldg(p.w_scale + n);
+                    if (W4) comb *= 0.0625f;
+                    if (p.bias) b = __half2float(p.bias[n]);
+                }
+                s_comb[j] = comb;
+                s_bias[j] = b;
+            }
+            if (p.bos && p.Y && blockIdx.y == 0 && rank == 0) {
+                // row 0 of every prompt: the stored floating-point BOS projection, copied as is
+                for (int idx = tid - 64; idx < p.batch * BN; idx += 128) {
+                    const int b = idx / BN, j = idx - b * BN;
+                    if (n0 + j < p.N)
+                        p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
+                }
+            }
+        }
         // ------------------------------------------------------------ epilogue, part 1
         // accumulators: tensor memory -> registers -> shared memory (the pipeline buffers are
         // free once the last MMA has completed), 16-byte chunks XOR-swizzled by row
@@ -399,7 +402,7 @@ int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp
 int pick_splits(int64_t tiles, int k_blocks)
 {
     int s = 1;
-    while (s < 8 && tiles * (2 * s) <= 160 && k_blocks / (2 * s) >= 2) s *= 2;
+    while (s < 8 && tiles * (2 * s) <= 148 && k_blocks / (2 * s) >= 2) s *= 2;
     return s;
 }
 
@@ -491,7 +494,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         tp.k_blocks = static_cast<int>(ceil_div(p.K, BK));
     }
     if (rc != MIXDQ_OK) return rc;
-    const bool wide = p.N >= 1024 || p.N % 256 == 0;
+    // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
+    const bool wide = (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
     const uint32_t bn = wide ? 256 : 128;
     if (w4)
         rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, bn, false);
@@ -507,8 +511,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     if (wide)
         return w4 ? launch_tma<256, 3, true>(ta, tw, tp, splits, stream)
                   : launch_tma<256, 4, false>(ta, tw, tp, splits, stream);
-    return w4 ? launch_tma<128, 4, true>(ta, tw, tp, splits, stream)
-              : launch_tma<128, 4, false>(ta, tw, tp, splits, stream);
+    return w4 ? launch_tma<128, 5, true>(ta, tw, tp, splits, stream)
+              : launch_tma<128, 6, false>(ta, tw, tp, splits, stream);
 }
 
 }  // namespace i8

@@ -43,6 +43,7 @@ _SIGNATURES = {
                              _sz, _vp, _vp]),
     "mixdq_crossattn_kv": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "mixdq_crossattn_kv_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_probe_mma_loop": (_int, [_int, _int, C.POINTER(C.c_double), _vp, _vp]),
     "mixdq_static_scratch_bytes": (_sz, []),
     "mixdq_linear_a8_static_scratch": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp,
                                               _vp]),
@@ -264,3 +265,20 @@ def linear_a8_static_scratch(X, packed_W, N: int, w_bits: int, w_scale, act_scal
                                               _ptr(w_scale), _ptr(act_scale), _ptr(bias), _ptr(Y), _ptr(status),
                                               _stream()), "mixdq_linear_a8_static_scratch")
     return Y
+
+
+def probe_mma_loop(kind: int, batches: int, repeats: int = 3) -> float:
+    """Tensor-core MMA-loop peak in TOP/s (kind 1: int8, kind 0: fp16), best of ``repeats``."""
+    ops = C.c_double(0.0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    best = 0.0
+    for _ in range(repeats + 1):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        _chk(lib().mixdq_probe_mma_loop(kind, batches, C.byref(ops), _ptr(status), _stream()), "mixdq_probe_mma_loop")
+        b.record()
+        torch.cuda.synchronize()
+        if int(status.item()) != 0:
+            raise MixdqError("mixdq_probe_mma_loop: device-side wait timed out")
+        best = max(best, ops.value / (a.elapsed_time(b) * 1e-3) / 1e12)
+    return best
