@@ -383,6 +383,301 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (warp == 1) tmem_dealloc(tmem_base, BN);
 }
 
+// Persistent form for problems with at least as many output tiles as SMs: one CTA per SM
+// walks over tiles (tile = blockIdx.x + i * gridDim.x, column-fastest so that concurrent CTAs
+// share operands in L2).  Two accumulators in tensor memory alternate, so the epilogue of one
+// tile (tensor memory -> registers -> fp16 stores) runs while the MMAs of the next tile are
+// already being issued, and the TMA pipeline never drains between tiles.
+template <int BN, int STAGES, bool W4>
+struct PersistSmem {
+    static constexpr int A_BYTES = BM * BK;
+    static constexpr int B_BYTES = BN * BK;
+    static constexpr int STG_BYTES = W4 ? BN * (BK / 2) : 0;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+    static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
+    static constexpr int OFF_BARS = OFF_STG + STAGES * STG_BYTES;
+    static constexpr int NUM_BARS = 3 * STAGES + 4;
+    static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] floats
+    static constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;
+    static constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
+    static constexpr int TOTAL = OFF_MISC + 64 + 1024;
+    static constexpr int THREADS = W4 ? 320 : 192;
+};
+
+template <int BN, int STAGES, bool W4>
+__global__ void __launch_bounds__(PersistSmem<BN, STAGES, W4>::THREADS, 1)
+tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                           const TmaParams p, int n_tiles, int total_tiles)
+{
+    using L = PersistSmem<BN, STAGES, W4>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    uint8_t* sA = smem + L::OFF_A;
+    uint8_t* sB = smem + L::OFF_B;
+    uint8_t* sStg = smem + L::OFF_STG;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
+    float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
+    float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nkb = p.k_blocks;
+    const int my_tiles = (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                         static_cast<int>(gridDim.x);
+
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_unpacked = smem_u32(bars + STAGES);
+    const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);
+    const uint32_t bar_acc_full = smem_u32(bars + 3 * STAGES);       // [2]: accumulator complete
+    const uint32_t bar_acc_empty = smem_u32(bars + 3 * STAGES + 2);  // [2]: accumulator drained
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_unpacked + 8 * s, 4);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, 4);
+        }
+        *s_abort = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(s_tmem), 2 * BN);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            int it = 0;  // k-blocks issued so far, over all tiles
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = blockIdx.x + t * gridDim.x;
+                const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+                int img_b = 0, ho0 = 0, wo0 = 0;
+                if (p.conv) {
+                    img_b = m0 / p.HoWo;
+                    const int rem = m0 - img_b * p.HoWo;
+                    ho0 = rem / p.Wo;
+                    wo0 = rem - ho0 * p.Wo;
+                }
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t round = static_cast<uint32_t>(it / STAGES);
+                    ok = mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
+                    const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
+                    const uint32_t dst_b = W4 ? smem_u32(sStg + s * L::STG_BYTES) : smem_u32(sB + s * L::B_BYTES);
+                    if (p.conv) {
+                        const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
+                        const int kh = tap / 3, kw = tap - 3 * kh;
+                        tma_load_4d(dst_a, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, bar_full + 8 * s);
+                        const int kx = tap * p.Cin + cb * BK;
+                        tma_load_2d(dst_b, &tmap_w, W4 ? kx / 2 : kx, n0, bar_full + 8 * s);
+                    } else {
+                        tma_load_2d(dst_a, &tmap_a, kb * BK, m0, bar_full + 8 * s);
+                        tma_load_2d(dst_b, &tmap_w, kb * ROW_BYTES, n0, bar_full + 8 * s);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
+            int it = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int buf = t & 1;
+                const uint32_t use = static_cast<uint32_t>(t >> 1);  // how often this accumulator was used before
+                ok = mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, s_abort);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t acc = tmem_base + buf * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t round = static_cast<uint32_t>(it / STAGES);
+                    ok = mbar_wait(bar_full + 8 * s, round & 1, s_abort);
+                    if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, round & 1, s_abort);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint64_t a_desc = smem_desc_sw128(smem_u32(sA + s * L::A_BYTES));
+                    const uint64_t b_desc = smem_desc_sw128(smem_u32(sB + s * L::B_BYTES));
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    tc_commit(bar_empty + 8 * s);
+                }
+                if (ok) tc_commit(bar_acc_full + 8 * buf);
+            }
+        }
+        __syncwarp();
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue warps
+        const int lg = warp & 3;
+        const int et = tid - 64;
+        const float sx = __ldg(p.act_scale);
+        const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
+        bool ok = true;
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = blockIdx.x + t * gridDim.x;
+            const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+            const int buf = t & 1;
+            const uint32_t use = static_cast<uint32_t>(t >> 1);
+            float* comb = s_comb + buf * BN;
+            float* bias = s_bias + buf * BN;
+            // this tile's per-column factors (the buffer was last read two tiles ago)
+            for (int j = et; j < BN; j += 128) {
+                const int n = n0 + j;
+                float c = 0.f, b = 0.f;
+                if (n < p.N && p.w_scale) {
+                    c = sx * __ldg(p.w_scale + n);
+                    if (W4) c *= 0.0625f;
+                    if (p.bias) b = __half2float(p.bias[n]);
+                }
+                comb[j] = c;
+                bias[j] = b;
+            }
+            if (p.bos && p.Y && m0 == 0) {
+                for (int idx = et; idx < p.batch * BN; idx += 128) {
+                    const int b = idx / BN, j = idx - b * BN;
+                    if (n0 + j < p.N)
+                        p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ok) ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, s_abort);
+            tc_fence_after_sync();
+            const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
+            if (!go) {
+                ok = false;
+                continue;
+            }
+            const int m = m0 + lg * 32 + lane;
+            const bool m_ok = m < p.M;
+            long long out_row = m;
+            if (p.bos && m_ok) {
+                const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                          (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+            }
+            const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (n0 + c0 >= p.N) break;  // uniform across the warp
+                uint32_t r[32];
+                tmem_ld_32x32(acc + c0, r);
+                tmem_ld_wait();
+                if (!m_ok) continue;
+                const int n = n0 + c0;
+                if (p.acc_out) {
+                    int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n + j < p.N) dst[j] = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
+                }
+                if (p.Y) {
+                    __half* dst = p.Y + out_row * p.ldy + n;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        __half2 h[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int c = c0 + j + 2 * q;
+                            h[q] = __floats2half2_rn(
+                                fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2 * q])), comb[c], bias[c]),
+                                fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2 * q + 1])), comb[c + 1], bias[c + 1]));
+                        }
+                        if (vec && n + j + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(dst + j) = *reinterpret_cast<const uint4*>(h);
+                        } else {
+                            const __half* hs = reinterpret_cast<const __half*>(h);
+                            for (int q = 0; q < 8; ++q)
+                                if (n + j + q < p.N) dst[j + q] = hs[q];
+                        }
+                    }
+                }
+            }
+            // the accumulator may be overwritten once every epilogue warp has read it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+        }
+    } else if (W4) {
+        // ------------------------------------------------------------ int4 -> int8 (x16) expansion
+        const int ut = tid - 192;
+        const int total_kb = my_tiles * nkb;
+        for (int it = 0; it < total_kb; ++it) {
+            const int s = it % STAGES;
+            const uint32_t round = static_cast<uint32_t>(it / STAGES);
+            if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
+            const uint8_t* stg = sStg + s * L::STG_BYTES;
+            uint8_t* b_stage = sB + s * L::B_BYTES;
+#pragma unroll 4
+            for (int t = 0; t < (BN * 4) / 128; ++t) {
+                const int task = ut + t * 128;
+                const int r = task >> 2, j = task & 3;
+                const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
+                uint4 c0, c1;
+                c0.x = (w.x << 4) & 0xF0F0F0F0u;
+                c0.y = w.x & 0xF0F0F0F0u;
+                c0.z = (w.y << 4) & 0xF0F0F0F0u;
+                c0.w = w.y & 0xF0F0F0F0u;
+                c1.x = (w.z << 4) & 0xF0F0F0F0u;
+                c1.y = w.z & 0xF0F0F0F0u;
+                c1.z = (w.w << 4) & 0xF0F0F0F0u;
+                c1.w = w.w & 0xF0F0F0F0u;
+                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
+                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
+        }
+    }
+
+    if (*s_abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (tid == 0 && p.status) atomicExch(p.status, MIXDQ_ERR_TIMEOUT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
+}
+
+template <int BN, int STAGES, bool W4>
+int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp, int num_sms,
+                      cudaStream_t stream)
+{
+    using L = PersistSmem<BN, STAGES, W4>;
+    auto kernel = tma_gemm_persistent_kernel<BN, STAGES, W4>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
+        attr_set = true;
+    }
+    const int n_tiles = static_cast<int>(ceil_div(tp.N, BN));
+    const int total = n_tiles * static_cast<int>(ceil_div(tp.M, BM));
+    const dim3 grid(static_cast<unsigned>(total < num_sms ? total : num_sms));
+    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, tp, n_tiles, total);
+}
+
 template <int BN, int STAGES, bool W4>
 int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp, int splits, cudaStream_t stream)
 {
@@ -503,7 +798,21 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(p.K), p.N, pitch, BK, bn, true);
     if (rc != MIXDQ_OK) return rc;
 
-    int splits = pick_splits(ceil_div(p.M, BM) * ceil_div(p.N, bn), tp.k_blocks);
+    const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, bn);
+    static int num_sms = 0;
+    if (!num_sms) {
+        int dev = 0;
+        MIXDQ_CUDA_TRY(cudaGetDevice(&dev));
+        MIXDQ_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if (tiles >= num_sms && p.force_splits <= 0) {
+        if (wide)
+            return w4 ? launch_persistent<256, 3, true>(ta, tw, tp, num_sms, stream)
+                      : launch_persistent<256, 4, false>(ta, tw, tp, num_sms, stream);
+        return w4 ? launch_persistent<128, 5, true>(ta, tw, tp, num_sms, stream)
+                  : launch_persistent<128, 6, false>(ta, tw, tp, num_sms, stream);
+    }
+    int splits = pick_splits(tiles, tp.k_blocks);
     if (p.force_splits > 0) {
         splits = 1;
         while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;

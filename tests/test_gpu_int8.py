@@ -66,6 +66,16 @@ def test_linear_split_reduction(bits, M, K, N):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,K,N", [(2048, 272, 1288), (4100, 144, 1290), (2500, 1040, 1032)])
+def test_linear_persistent_tiles(bits, M, K, N):
+    # at least as many output tiles as SMs: the persistent kernel walks several tiles per CTA
+    g = synth.normal_f16((M, K), 1.0, seed=M + K + 3)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 4)
+    b = synth.normal_f16((N,), 0.01, seed=N + 1)
+    _run_linear(g, W, b, bits, True)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
 def test_few_output_channels_with_workspace(bits):
     # 4 output channels (conv_out-like): the weight tile is mostly out-of-bounds fill
     _run_linear(synth.normal_f16((200, 2880), 1.0, 6), synth.normal_f16((4, 2880), 0.02, 7),
@@ -89,7 +99,7 @@ def test_ffn_outlier_channels():
 
 @pytest.mark.parametrize("use_ws", [False, True])
 @pytest.mark.parametrize("bits", [8, 4])
-@pytest.mark.parametrize("B,N", [(1, 64), (3, 200)])
+@pytest.mark.parametrize("B,N", [(1, 64), (3, 200), (30, 1280)])
 def test_bos_aware_kv(bits, B, N, use_ws):
     E = synth.text_embedding(B, seed=4000)
     W = synth.kv_weight(N, seed=4100 + N)
@@ -127,7 +137,7 @@ def test_bos_aware_kv(bits, B, N, use_ws):
                                                     (3, 9, 7, 48, 24, 2), (3, 8, 8, 32, 40, 1),
                                                     (2, 32, 32, 160, 136, 1), (1, 64, 64, 32, 24, 1),
                                                     (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2),
-                                                    (1, 12, 12, 256, 32, 1)])
+                                                    (1, 12, 12, 256, 32, 1), (1, 64, 64, 32, 648, 1)])
 def test_conv3x3(bits, B, H, W, Cin, Cout, stride, use_ws):
     X = synth.normal_f16((B, H, W, Cin), 1.0, seed=H * W + Cin)
     Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin)
