@@ -24,6 +24,7 @@ constexpr int kSlices = 4;
 constexpr int kChanPerCta = 16 * kTilesPerCta;
 constexpr int kUnit = 128;       // reduction elements per unit: 32 codes per thread of a quad
 constexpr int kChunkMax = 2048;  // reduction elements staged in shared memory at a time
+constexpr int kSmallKMax = 5120; // longest reduction the small-token kernel keeps in shared memory
 
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
@@ -225,18 +226,34 @@ wo_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, i
 
         if (kc0 > 0) __syncthreads();  // everyone is done reading the previous chunk
         // stage X[m_base .. m_base+MB) x [kc0, kc0+len) in decode order
-        for (int idx = tid; idx < MB * (len / 8); idx += kThreads) {
-            const int r = idx / (len / 8), j = idx - r * (len / 8);
-            uint4 v = load_x8(p, amode, m_base + r, kc0 + j * 8);
-            if (BITS != 8) {
-                // decode order inside each run of four: (0, 2, 1, 3)
-                const uint32_t a = __byte_perm(v.x, v.y, 0x5410), b = __byte_perm(v.x, v.y, 0x7632);
-                const uint32_t c = __byte_perm(v.z, v.w, 0x5410), d = __byte_perm(v.z, v.w, 0x7632);
-                v = make_uint4(a, b, c, d);
+        // (loads are issued eight at a time so that their latencies overlap)
+        const int per_row = len / 8, total16 = MB * per_row;
+        for (int base = tid; base < total16; base += kThreads * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int idx = base + i * kThreads;
+                if (idx < total16) {
+                    const int r = idx / per_row, j = idx - r * per_row;
+                    v[i] = load_x8(p, amode, m_base + r, kc0 + j * 8);
+                }
             }
-            // 16-byte slot of (unit U, quad thread tt, sub-step s): 16 U + 4 s + tt
-            const int U = j >> 4, tt = (j >> 2) & 3, s = j & 3;
-            *reinterpret_cast<uint4*>(sX + r * x_stride + (16 * U + 4 * s + tt) * 16) = v;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int idx = base + i * kThreads;
+                if (idx >= total16) break;
+                const int r = idx / per_row, j = idx - r * per_row;
+                uint4 x = v[i];
+                if (BITS != 8) {
+                    // decode order inside each run of four: (0, 2, 1, 3)
+                    const uint32_t a = __byte_perm(x.x, x.y, 0x5410), b = __byte_perm(x.x, x.y, 0x7632);
+                    const uint32_t c = __byte_perm(x.z, x.w, 0x5410), d = __byte_perm(x.z, x.w, 0x7632);
+                    x = make_uint4(a, b, c, d);
+                }
+                // 16-byte slot of (unit U, quad thread tt, sub-step s): 16 U + 4 s + tt
+                const int U = j >> 4, tt = (j >> 2) & 3, sub = j & 3;
+                *reinterpret_cast<uint4*>(sX + r * x_stride + (16 * U + 4 * sub + tt) * 16) = x;
+            }
         }
         __syncthreads();
 
@@ -298,6 +315,185 @@ wo_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, i
     }
 }
 
+// Small-token form (linear layers, at most 16 tokens): the layer is a single stream over the
+// packed weights, so the kernel is built around that stream.  The first weight loads go out
+// before the wait on the previous kernel -- weights and their parameters are constants of the
+// layer, only the activations can come from the kernel before -- so consecutive layers keep
+// the memory system busy across the kernel boundary.  The few activation rows are read
+// straight from global memory (they stay in L1) instead of being staged in shared memory.
+// CTA = 8 warps = TILES channel tiles x (8 / TILES) slices of the reduction.
+template <int BITS, bool SIGNED, int NT, int TILES>
+__global__ void __launch_bounds__(kThreads, 3)
+wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, int groups, int k_pad)
+{
+    constexpr int SLICES = 8 / TILES;
+    constexpr int MB = 8 * NT;
+    constexpr int GROUP = BITS == 8 ? 2 : 4;
+    extern __shared__ __align__(16) uint8_t smem[];
+    const int x_stride = k_pad * 2 + 64;  // 64 mod 128 bytes: quad reads of two token rows do not collide
+    uint8_t* sX = smem;
+    float* sRed = reinterpret_cast<float*>(smem + MB * x_stride);  // [SLICES][TILES * 16][MB]
+
+    pdl_launch_dependents();
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int tile = warp % TILES, slice = warp / TILES;
+    const int units = k_pad / kUnit;
+    const int u_begin = (units * slice) / SLICES, u_end = (units * (slice + 1)) / SLICES;
+
+    // state of the channel-tile group being worked on (a CTA walks groups blockIdx.x,
+    // blockIdx.x + gridDim.x, ...)
+    const uint8_t *row_lo, *row_hi;
+    bool lo_ok, hi_ok;
+    float z_a, z_b;
+    UnitRegs<BITS> ra[GROUP], rb[GROUP];
+
+    auto load_group_units = [&](int u0) {
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i) {
+            const bool in = u0 + i < u_end;
+            load_unit<BITS>(ra[i], row_lo, pitch, u0 + i, t, lo_ok && in);
+            load_unit<BITS>(rb[i], row_hi, pitch, u0 + i, t, hi_ok && in);
+        }
+    };
+    // weight side of a group: zero-points and the first packed words of this warp's slice
+    auto begin_group = [&](int grp) {
+        const int n_lo = (grp * TILES + tile) * 16 + g, n_hi = n_lo + 8;
+        lo_ok = n_lo < p.N;
+        hi_ok = n_hi < p.N;
+        row_lo = packed + static_cast<long long>(lo_ok ? n_lo : 0) * pitch;
+        row_hi = packed + static_cast<long long>(hi_ok ? n_hi : 0) * pitch;
+        z_a = z_b = SIGNED ? (BITS == 8 ? 128.f : 8.f) : 0.f;
+        if (!SIGNED && p.w_zero) {
+            if (lo_ok) z_a = static_cast<float>(__ldg(p.w_zero + n_lo));
+            if (hi_ok) z_b = static_cast<float>(__ldg(p.w_zero + n_hi));
+        }
+        load_group_units(u_begin);
+    };
+
+    int grp = blockIdx.x;
+    if (grp < groups) begin_group(grp);  // issued before the wait: weights are constants of the layer
+    pdl_wait();                          // the activations may be the previous kernel's output
+
+    // the token rows, once per CTA, in the order in which the decode produces the weights
+    {
+        const int per_row = k_pad / 8, total16 = MB * per_row;
+        for (int base = tid; base < total16; base += kThreads * 10) {
+            uint4 v[10];
+#pragma unroll
+            for (int i = 0; i < 10; ++i) {
+                const int idx = base + i * kThreads;
+                const int r = idx / per_row, k = (idx - r * per_row) * 8;
+                v[i] = (idx < total16 && r < p.M && k < p.K)
+                           ? __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<long long>(r) * p.ldx + k))
+                           : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int i = 0; i < 10; ++i) {
+                const int idx = base + i * kThreads;
+                if (idx >= total16) break;
+                const int r = idx / per_row, j = idx - r * per_row;
+                uint4 x = v[i];
+                if (BITS != 8)  // the decode yields pairs (0, 2), (1, 3) of each run of four
+                    x = make_uint4(__byte_perm(x.x, x.y, 0x5410), __byte_perm(x.x, x.y, 0x7632),
+                                   __byte_perm(x.z, x.w, 0x5410), __byte_perm(x.z, x.w, 0x7632));
+                const int U = j >> 4, tt = (j >> 2) & 3, sub = j & 3;
+                *reinterpret_cast<uint4*>(sX + r * x_stride + (16 * U + 4 * sub + tt) * 16) = x;
+            }
+        }
+    }
+    __syncthreads();
+
+    for (; grp < groups; grp += gridDim.x) {
+        const __half2 zlo_a = __float2half2_rn(1024.f + z_a), zhi_a = __float2half2_rn(-(64.f + z_a));
+        const __half2 zlo_b = __float2half2_rn(1024.f + z_b), zhi_b = __float2half2_rn(-(64.f + z_b));
+        float acc[NT][4];
+#pragma unroll
+        for (int i = 0; i < NT; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+        for (int u0 = u_begin; u0 < u_end; u0 += GROUP) {
+            if (u0 != u_begin) load_group_units(u0);
+#pragma unroll
+            for (int i = 0; i < GROUP; ++i) {
+                if (u0 + i >= u_end) break;
+#pragma unroll
+                for (int sub = 0; sub < 4; ++sub) {
+                    uint32_t fa[4], fb[4];
+                    decode_substep<BITS, SIGNED>(ra[i], sub, zlo_a, zhi_a, fa);
+                    decode_substep<BITS, SIGNED>(rb[i], sub, zlo_b, zhi_b, fb);
+                    const uint32_t a1[4] = {fa[0], fb[0], fa[1], fb[1]};
+                    const uint32_t a2[4] = {fa[2], fb[2], fa[3], fb[3]};
+                    const int slot = (16 * (u0 + i) + 4 * sub + t) * 16;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(sX + (g + 8 * nt) * x_stride + slot);
+                        mma_16816(acc[nt], a1, x.x, x.y);
+                        mma_16816(acc[nt], a2, x.z, x.w);
+                    }
+                }
+            }
+        }
+
+        // the next group's weights start streaming while this one is reduced and stored
+        const int out_grp = grp;
+        if (grp + static_cast<int>(gridDim.x) < groups) begin_group(grp + gridDim.x);
+
+        // sum the reduction slices: sRed[slice][channel][token]
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float* base = sRed + (slice * TILES * 16 + tile * 16) * MB + nt * 8 + 2 * t;
+            base[g * MB] = acc[nt][0];
+            base[g * MB + 1] = acc[nt][1];
+            base[(g + 8) * MB] = acc[nt][2];
+            base[(g + 8) * MB + 1] = acc[nt][3];
+        }
+        __syncthreads();
+        for (int idx = tid; idx < TILES * 16 * MB; idx += kThreads) {
+            const int ch = idx % (TILES * 16), tok = idx / (TILES * 16);
+            const int n = out_grp * TILES * 16 + ch;
+            if (n >= p.N || tok >= p.M) continue;
+            float sum = 0.f;
+#pragma unroll
+            for (int sl = 0; sl < SLICES; ++sl) sum += sRed[(sl * TILES * 16 + ch) * MB + tok];
+            const float b = p.bias ? __half2float(p.bias[n]) : 0.f;
+            p.Y[static_cast<long long>(tok) * p.ldy + n] = __float2half_rn(fmaf(__ldg(p.w_scale + n), sum, b));
+        }
+        __syncthreads();  // sRed is reused by the next group
+    }
+}
+
+template <int BITS, bool SIGNED, int NT, int TILES>
+int launch_small_tiles(const Params& p, const void* packed, long long pitch, cudaStream_t stream)
+{
+    constexpr int MB = 8 * NT;
+    const int k_pad = static_cast<int>(round_up(p.K, kUnit));
+    const size_t smem = static_cast<size_t>(MB) * (k_pad * 2 + 64) + 8 * 16 * MB * sizeof(float);
+    auto kernel = wo_small_kernel<BITS, SIGNED, NT, TILES>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            16 * (kSmallKMax * 2 + 64) + 8 * 16 * 16 * 4));
+        attr_set = true;
+    }
+    // groups of TILES channel tiles are dealt to CTAs in equal rounds of at most three CTAs per SM
+    const int groups = static_cast<int>(ceil_div(p.N, 16 * TILES));
+    const int rounds = static_cast<int>(ceil_div(groups, 444));
+    const dim3 grid(static_cast<unsigned>(ceil_div(groups, rounds)));
+    return launch_pdl(kernel, grid, dim3(kThreads), smem, stream, 1, static_cast<const uint8_t*>(packed), pitch, p,
+                      groups, k_pad);
+}
+
+template <int BITS, bool SIGNED, int NT>
+int launch_small(const Params& p, const void* packed, long long pitch, cudaStream_t stream)
+{
+    // one channel tile per CTA (more reduction slices) when two per CTA would leave SMs idle
+    if (ceil_div(p.N, 32) < 148) return launch_small_tiles<BITS, SIGNED, NT, 1>(p, packed, pitch, stream);
+    return launch_small_tiles<BITS, SIGNED, NT, 2>(p, packed, pitch, stream);
+}
+
 template <int BITS, bool SIGNED, int NT>
 int launch(const Params& p, int amode, const void* packed, long long pitch, cudaStream_t stream)
 {
@@ -319,6 +515,10 @@ int launch(const Params& p, int amode, const void* packed, long long pitch, cuda
 template <int BITS, bool SIGNED>
 int launch_nt(const Params& p, int amode, const void* packed, long long pitch, cudaStream_t stream)
 {
+    if (amode == A_LINEAR && p.M <= 16 && p.K % 8 == 0 && p.K <= kSmallKMax) {
+        if (p.M <= 8) return launch_small<BITS, SIGNED, 1>(p, packed, pitch, stream);
+        return launch_small<BITS, SIGNED, 2>(p, packed, pitch, stream);
+    }
     if (p.M <= 8) return launch<BITS, SIGNED, 1>(p, amode, packed, pitch, stream);
     if (p.M <= 16) return launch<BITS, SIGNED, 2>(p, amode, packed, pitch, stream);
     return launch<BITS, SIGNED, 4>(p, amode, packed, pitch, stream);
