@@ -379,10 +379,10 @@ wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Param
     // the token rows, once per CTA, in the order in which the decode produces the weights
     {
         const int per_row = k_pad / 8, total16 = MB * per_row;
-        for (int base = tid; base < total16; base += kThreads * 10) {
-            uint4 v[10];
+        for (int base = tid; base < total16; base += kThreads * 6) {
+            uint4 v[6];
 #pragma unroll
-            for (int i = 0; i < 10; ++i) {
+            for (int i = 0; i < 6; ++i) {
                 const int idx = base + i * kThreads;
                 const int r = idx / per_row, k = (idx - r * per_row) * 8;
                 v[i] = (idx < total16 && r < p.M && k < p.K)
@@ -390,7 +390,7 @@ wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Param
                            : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
-            for (int i = 0; i < 10; ++i) {
+            for (int i = 0; i < 6; ++i) {
                 const int idx = base + i * kThreads;
                 if (idx >= total16) break;
                 const int r = idx / per_row, j = idx - r * per_row;
