@@ -123,6 +123,7 @@ int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, cons
     p.Ho = static_cast<int>(Ho);
     p.Wo = static_cast<int>(Wo);
     p.stride = stride;
+    p.batch = static_cast<int>(B);
     p.w_scale = w_scale;
     p.w_zero = w_zero;
     p.bias = static_cast<const __half*>(bias);

@@ -52,6 +52,9 @@ int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64
 // 4-D byte tensor map with the 128-byte swizzle (NHWC int8 image: dims {C, W, H, B}).
 int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
                       const uint32_t box[4]);
+// The same for an fp16 NHWC image (box extents in elements, strides in bytes).
+int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
+                       const uint32_t box[4]);
 
 #ifdef __CUDACC__
 

@@ -57,6 +57,7 @@ struct Params {
     long long ldx = 0;
     int M = 0, N = 0, K = 0;
     int H = 0, W = 0, Cin = 0, Ho = 0, Wo = 0, stride = 1;
+    int batch = 0;  // images (conv)
     const float* w_scale = nullptr;
     const int32_t* w_zero = nullptr;  // nullptr: signed codes, zero-point 0
     const __half* bias = nullptr;
@@ -66,6 +67,9 @@ struct Params {
 };
 
 int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream);
+// Many-token path on tcgen05 (fp16 MMA, weights expanded into shared memory); see wo_tc.cu.
+bool tc_path_ok(const Params& p, int amode, int w_bits);
+int run_tc(const Params& p, int amode, const void* packed, int w_bits, int batch, cudaStream_t stream);
 
 }  // namespace wo
 

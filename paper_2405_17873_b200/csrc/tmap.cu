@@ -66,8 +66,23 @@ int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64
 }
 
 
+static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, const uint64_t dims[4],
+                          const uint64_t strides_bytes[3], const uint32_t box[4]);
+
 int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
                       const uint32_t box[4])
+{
+    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, dims, strides_bytes, box);
+}
+
+int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
+                       const uint32_t box[4])
+{
+    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, base, dims, strides_bytes, box);
+}
+
+static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, const uint64_t dims[4],
+                          const uint64_t strides_bytes[3], const uint32_t box[4])
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return MIXDQ_ERR_CUDA;
@@ -82,7 +97,7 @@ int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4]
         if (strides_bytes[i] & 15) return MIXDQ_ERR_ALIGNMENT;
         st[i] = strides_bytes[i];
     }
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), d, st, b, estr,
+    CUresult r = fn(map, dtype, 4, const_cast<void*>(base), d, st, b, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;

@@ -37,6 +37,23 @@ def test_ragged_shapes(bits, M, K, N):
     _run(X, W, b, bits)
 
 
+# 64 tokens or more: the tensor-memory (tcgen05) form of the engine, one or several tiles per CTA
+@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("M,K,N", [(64, 64, 16), (300, 2880, 136), (2100, 320, 1300), (130, 200, 264), (4096, 320, 320)])
+def test_many_token_shapes(bits, M, K, N):
+    X = synth.normal_f16((M, K), 1.0, seed=M * 7 + K)
+    W = synth.normal_f16((N, K), 0.02, seed=N * 11 + K)
+    b = synth.normal_f16((N,), 0.01, seed=N + 2)
+    _run(X, W, b, bits)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_symmetric_codes_many_tokens(bits):
+    X = synth.normal_f16((256, 640), 1.0, seed=3)
+    W = synth.normal_f16((72, 640), 0.02, seed=4)
+    _run(X, W, None, bits, symmetric=True)
+
+
 @pytest.mark.parametrize("bits", [4, 8])
 def test_symmetric_codes_at_a16(bits):
     X = synth.normal_f16((16, 640), 1.0, seed=1)
@@ -45,9 +62,10 @@ def test_symmetric_codes_at_a16(bits):
 
 
 @pytest.mark.parametrize("bits", [3, 4, 8])
-@pytest.mark.parametrize("stride", [1, 2])
-def test_weight_only_conv3x3(bits, stride):
-    B, H, Wd, Cin, Cout = 2, 6, 5, 32, 40
+@pytest.mark.parametrize("geom", [(2, 6, 5, 32, 40, 1), (2, 6, 5, 32, 40, 2), (2, 16, 16, 64, 40, 1),
+                                  (1, 8, 8, 128, 48, 1), (3, 32, 32, 192, 136, 1)])
+def test_weight_only_conv3x3(bits, geom):
+    B, H, Wd, Cin, Cout, stride = geom
     X = synth.normal_f16((B, H, Wd, Cin), 1.0, seed=7)
     Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=8)
     b = synth.normal_f16((Cout,), 0.01, seed=9)
