@@ -5,7 +5,7 @@
 //               convolution reads a 4-D box of the NHWC image shifted by the filter tap
 //   warp 1      tensor-memory owner and MMA issuer (128 x 128 x 16 per instruction)
 //   warps 2..5  epilogue: tensor memory -> registers -> y = fp16(scale[n] * acc + bias[n])
-//   warps 6..9  weight feeders: packed codes straight from global memory into registers,
+//   warps 6..13 weight feeders: packed codes straight from global memory into registers,
 //               expanded to the exact fp16 integers (q - z) and written as the swizzled
 //               K-major B tile
 // One CTA per SM walks over output tiles; two accumulators alternate so that the epilogue of
@@ -32,7 +32,8 @@ constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] scale
 constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;                 // [2][BN] biases
 constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
 constexpr int SMEM_TOTAL = OFF_MISC + 64 + 1024;
-constexpr int THREADS = 320;
+constexpr int THREADS = 448;
+constexpr int kFeedWarps = 8;
 
 struct TcParams {
     int M, N, K, k_blocks;
@@ -164,7 +165,7 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full_a + 8 * s, 1);
-            mbar_init(bar_full_b + 8 * s, 4);
+            mbar_init(bar_full_b + 8 * s, kFeedWarps);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -313,25 +314,17 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
         // thread -> (row of the tile, which 32-code half of the 64-wide k-block)
         const int ft = tid - 192;
         const int half = ft & 1;
-        const int r0 = ft >> 1;  // rows r0 and r0 + 64
+        const int r = ft >> 1;
         int it = 0;
         bool ok = true;
         for (int t = 0; t < my_tiles && ok; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
-            const int n0 = (tile % n_tiles) * BN;
-            const uint8_t* rows[2];
-            bool row_ok[2];
-            __half2 z_lo[2], z_hi[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const int n = n0 + r0 + 64 * i;
-                row_ok[i] = n < p.N;
-                rows[i] = p.packed + static_cast<long long>(row_ok[i] ? n : 0) * p.pitch;
-                float z = SIGNED ? (BITS == 8 ? 128.f : 8.f) : 0.f;
-                if (!SIGNED && p.w_zero && row_ok[i]) z = static_cast<float>(__ldg(p.w_zero + n));
-                z_lo[i] = __float2half2_rn(1024.f + z);
-                z_hi[i] = __float2half2_rn(-(64.f + z));
-            }
+            const int n = (tile % n_tiles) * BN + r;
+            const bool row_ok = n < p.N;
+            const uint8_t* row = p.packed + static_cast<long long>(row_ok ? n : 0) * p.pitch;
+            float z = SIGNED ? (BITS == 8 ? 128.f : 8.f) : 0.f;
+            if (!SIGNED && p.w_zero && row_ok) z = static_cast<float>(__ldg(p.w_zero + n));
+            const __half2 z_lo = __float2half2_rn(1024.f + z), z_hi = __float2half2_rn(-(64.f + z));
             // reduction index (in 32-code runs) of k-block kb: conv k-blocks restart per filter tap
             auto k32_of = [&](int kb) {
                 if (p.conv) {
@@ -340,32 +333,26 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
                 }
                 return kb * 2 + half;
             };
-            Codes32<BITS> cur[2], nxt[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) load_codes32<BITS>(cur[i], rows[i], p.pitch, k32_of(0), row_ok[i]);
+            // packed words two k-blocks ahead of the one being expanded
+            Codes32<BITS> c0, c1, c2;
+            load_codes32<BITS>(c0, row, p.pitch, k32_of(0), row_ok);
+            load_codes32<BITS>(c1, row, p.pitch, k32_of(nkb > 1 ? 1 : 0), row_ok && nkb > 1);
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % STAGES;
                 const uint32_t round = static_cast<uint32_t>(it / STAGES);
-                if (kb + 1 < nkb) {
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) load_codes32<BITS>(nxt[i], rows[i], p.pitch, k32_of(kb + 1), row_ok[i]);
-                }
+                load_codes32<BITS>(c2, row, p.pitch, k32_of(kb + 2 < nkb ? kb + 2 : 0), row_ok && kb + 2 < nkb);
                 ok = mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort);
                 if (!ok) break;
                 uint8_t* b_stage = sB + s * B_BYTES;
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int r = r0 + 64 * i;
-#pragma unroll
-                    for (int sub = 0; sub < 4; ++sub)
-                        *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 4 * half + sub)) =
-                            decode8<BITS, SIGNED>(cur[i], sub, z_lo[i], z_hi[i]);
-                }
+                for (int sub = 0; sub < 4; ++sub)
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 4 * half + sub)) =
+                        decode8<BITS, SIGNED>(c0, sub, z_lo, z_hi);
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full_b + 8 * s);
-#pragma unroll
-                for (int i = 0; i < 2; ++i) cur[i] = nxt[i];
+                c0 = c1;
+                c1 = c2;
             }
         }
     }
