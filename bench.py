@@ -235,7 +235,7 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2405_17873_b200 import build, mixdq
+    from paper_2405_17873_b200 import build, mixdq, replicas
     from paper_2405_17873_b200.unet_sweep import UNetSweep
 
     rank = int(os.environ.get("RANK", "0"))
@@ -259,21 +259,22 @@ def run_ours(args):
         for _ in range(2):
             sweep.step()
     torch.cuda.synchronize()
-    graphs = []
+    graphs, group_launches = [], []
     for group in (tc_layers, other_layers):
         if not group:
             graphs.append(None)
+            group_launches.append(0)
             continue
         g = torch.cuda.CUDAGraph()
+        before = mixdq.kernel_launches()
         with torch.cuda.graph(g, stream=stream):
             sweep.step(group)
+        group_launches.append(mixdq.kernel_launches() - before)   # kernels recorded into the graph
         graphs.append(g)
     g_tc, g_other = graphs
-    launches_per_step = len(sweep.layers)
+    launches_per_step = sum(group_launches)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    barrier = replicas.barrier
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -343,10 +344,7 @@ def run_ours(args):
         e2e_ms = s2.elapsed_time(e2) / args.e2e_steps
 
     ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step, e2e_ms, tc_ms, other_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms, tc_ms, other_ms = t.tolist()
+    ms_per_step, e2e_ms, tc_ms, other_ms = replicas.max_over_ranks([ms_per_step, e2e_ms, tc_ms, other_ms], "cuda")
 
     ops_step = sweep.total_ops()
     peaks = measured_peaks()
@@ -355,20 +353,22 @@ def run_ours(args):
         achieved = tc_ops / (tc_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
-                    "traffic": None, "kernel": "i8::gemm_kernel (tcgen05 kind::i8)",
+                    "traffic": None,
+                    "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
+                              "their quant_kernel pre-pass, all tensor-core int8 layers of the step",
                     "peak_source": f"{peaks['source']} bf16 sustained x {INT8_TO_BF16_NOMINAL:g} (nominal int8:bf16)",
-                    "launches_per_step": len(tc_layers), "ms_per_step": tc_ms}
+                    "launches_per_step": group_launches[0], "layers": len(tc_layers), "ms_per_step": tc_ms}
     else:
         alg = sum(sweep.algorithmic_bytes(pl) for pl in sweep.layers)
         achieved = alg / (other_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "wo::wo_kernel (mma.sync f16)",
-                    "peak_source": f"{peaks['source']} copy bandwidth", "launches_per_step": len(other_layers),
+                    "peak_source": f"{peaks['source']} copy bandwidth", "launches_per_step": group_launches[1],
                     "ms_per_step": other_ms}
 
     if rank == 0:
         out = {
-            "metric": METRIC, "value": world * ops_step / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": replicas.whole_job_rate(ops_step, ms_per_step) / 1e12, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8" if args.table == "w4a8" else "f16",
             "data": "synthetic",
@@ -377,7 +377,7 @@ def run_ours(args):
                        "packed_weight_bytes": sweep.packed_weight_bytes(),
                        "l2": "weights (distinct per layer) are larger than L2", "launch": "CUDA graph replay"},
             "clocks": clocks,
-            "e2e": {"value": world * ops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": replicas.whole_job_rate(ops_step, e2e_ms) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline,

@@ -51,6 +51,11 @@ extern "C" {
 /* Library version as major*10000 + minor*100 + patch. */
 int mixdq_version(void);
 
+/* Number of kernels the layer calls (mixdq_linear, mixdq_conv3x3, mixdq_conv1x1,
+ * mixdq_crossattn_kv and their variants) have launched, or recorded into a stream capture, in
+ * this process so far: a measurement aid for counting launches per step. */
+unsigned long long mixdq_kernel_launches(void);
+
 /* Static, NUL-terminated description of an error code (host pointer, never NULL). */
 const char* mixdq_strerror(int code);
 

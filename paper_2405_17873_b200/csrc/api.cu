@@ -164,6 +164,11 @@ int kv_impl(const void* text_emb, int64_t B, int64_t Kt, const void* packed_W, i
 
 extern "C" int mixdq_version(void) { return 100; }
 
+extern "C" unsigned long long mixdq_kernel_launches(void)
+{
+    return g_layer_kernel_launches.load(std::memory_order_relaxed);
+}
+
 extern "C" const char* mixdq_strerror(int code)
 {
     switch (code) {

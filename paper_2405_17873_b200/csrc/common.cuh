@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/mixdq.h"
 
 namespace mixdq {
@@ -39,6 +41,9 @@ inline int64_t row_pitch_bytes(int64_t K, int bits, int layout)
             return MIXDQ_ERR_CUDA;          \
         }                                   \
     } while (0)
+
+// Kernels of the layer calls launched (or captured into a graph) by this process so far.
+inline std::atomic<unsigned long long> g_layer_kernel_launches{0};
 
 inline int check_launch() { return cudaGetLastError() == cudaSuccess ? MIXDQ_OK : MIXDQ_ERR_CUDA; }
 
@@ -80,6 +85,7 @@ inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     attr[1].val.clusterDim.z = cluster_z;
     cfg.attrs = attr;
     cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    g_layer_kernel_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();

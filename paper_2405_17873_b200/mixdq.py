@@ -24,6 +24,7 @@ _i64, _int, _vp, _sz = C.c_int64, C.c_int, C.c_void_p, C.c_size_t
 _SIGNATURES = {
     "mixdq_version": (C.c_int, []),
     "mixdq_strerror": (C.c_char_p, [_int]),
+    "mixdq_kernel_launches": (C.c_ulonglong, []),
     "mixdq_packed_bytes": (_int, [_i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_weight_minmax_params": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp, _vp]),
     "mixdq_pack_weights": (_int, [_vp, _i64, _i64, _int, _vp, _vp, _int, _vp, _vp]),
@@ -91,6 +92,10 @@ def _stream():
 
 def version() -> int:
     return lib().mixdq_version()
+
+
+def kernel_launches() -> int:
+    return int(lib().mixdq_kernel_launches())
 
 
 def packed_bytes(N: int, K: int, bits: int, layout: int = LAYOUT_DEVICE) -> int:

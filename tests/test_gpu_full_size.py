@@ -1,0 +1,140 @@
+"""Parity at the full layer sizes of the SDXL-turbo-shaped UNet sweep (image batch 4), through
+the same entry points and with the same workspace the benchmark uses.  The oracle computes a
+sample of output rows one by one (a 3x3 conv output pixel is a dot product over its gathered
+window, which the CPU suite pins against the direct convolution); int32 accumulators of the
+sampled rows must match bit for bit, fp16 outputs within the path's tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mixdq_oracle as orc
+from paper_2405_17873_b200 import mixdq, synth
+from helpers import dev, host, status_word
+
+pytestmark = pytest.mark.gpu
+
+B = 4
+_SPECS = {l.name: l for l in synth.unet_layers()}
+
+
+def _sample_rows(total, n=10, seed=0):
+    rng = np.random.default_rng(seed)
+    rows = set(rng.integers(0, total, size=n).tolist()) | {0, total - 1, min(127, total - 1), min(128, total - 1)}
+    return np.array(sorted(rows))
+
+
+def _window_rows(X, rows, stride):
+    """Gathered 3x3 windows (zero padding 1) of the sampled output pixels: [len(rows), 9*C]."""
+    Bn, H, W, C = X.shape
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    out = np.zeros((len(rows), 3, 3, C), X.dtype)
+    for i, m in enumerate(rows):
+        b, rem = divmod(int(m), Ho * Wo)
+        ho, wo = divmod(rem, Wo)
+        for kh in range(3):
+            for kw in range(3):
+                hi, wi = ho * stride + kh - 1, wo * stride + kw - 1
+                if 0 <= hi < H and 0 <= wi < W:
+                    out[i, kh, kw] = X[b, hi, wi]
+    return out.reshape(len(rows), 9 * C)
+
+
+def _close(y, y_ref):
+    d = np.abs(y.astype(np.float64) - y_ref.astype(np.float64)).max()
+    assert d <= 1e-3 * np.abs(y_ref.astype(np.float64)).max() + 1e-3, d
+
+
+def _check_layer(name, w_bits, a_bits, rows_override=None):
+    l = _SPECS[name]
+    X, W, b = synth.layer_inputs(l, B, seed=7000 + l.index)
+    if rows_override:                      # the weight-bound regime: a few tokens only
+        X = np.ascontiguousarray(X[:rows_override])
+    W2 = np.ascontiguousarray(W.reshape(l.N, -1))
+    sym = a_bits == 8
+    s_ref, z_ref = orc.weight_minmax_params(W2, w_bits, sym)
+    codes = orc.quantize_weights(W2, w_bits, s_ref, None if sym else z_ref)
+
+    Xd, Wd = dev(X), dev(W2)
+    s, z = mixdq.weight_minmax_params(Wd, w_bits, sym)
+    packed = mixdq.pack_weights(Wd, w_bits, s, None if sym else z)
+    zd = None if sym else z
+    st = status_word()
+    conv = l.kind == "conv3x3"
+    if conv:
+        ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, l.H, l.H, l.Cin, l.N, l.stride, w_bits, a_bits))
+    else:
+        rows_total = X.reshape(-1, X.shape[-1]).shape[0]
+        ws = mixdq.new_workspace(mixdq.workspace_bytes(rows_total, l.N, l.K, w_bits, a_bits))
+
+    if a_bits == 8:
+        if l.kind == "bos_kv":
+            sx_ref = orc.crossattn_act_scale(X)
+            sx = mixdq.act_scale(Xd.reshape(-1, l.K), 77)
+            bos = orc.bos_row(X[0, 0], W2)
+            y = host(mixdq.crossattn_kv(Xd, packed, l.N, w_bits, s, sx, dev(bos), ws, st))
+            acc = host(mixdq.crossattn_kv_acc_i32(Xd, packed, l.N, w_bits, sx, ws, st)).reshape(-1, l.N)
+            rest = np.ascontiguousarray(X[:, 1:, :]).reshape(-1, l.K)
+            rows = _sample_rows(rest.shape[0], seed=l.index)
+            a_rows = rest[rows]
+            y_rows = y[:, 1:, :].reshape(-1, l.N)[rows]
+            assert np.array_equal(y[:, 0, :].view(np.uint16), np.broadcast_to(bos, (B, l.N)).copy().view(np.uint16))
+            bias = None
+        elif conv:
+            sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+            sx = mixdq.act_scale(Xd)
+            y = host(mixdq.conv3x3(Xd, packed, l.N, w_bits, s, None, 8, sx, dev(b), l.stride, ws, st)).reshape(-1, l.N)
+            acc = host(mixdq.conv3x3_acc_i32(Xd, packed, l.N, w_bits, sx, l.stride, ws, st)).reshape(-1, l.N)
+            rows = _sample_rows(y.shape[0], seed=l.index)
+            a_rows = _window_rows(X, rows, l.stride)
+            y_rows, bias = y[rows], b
+        else:
+            X2 = X.reshape(-1, l.K)
+            sx_ref = orc.act_scale(orc.act_absmax(X2), 8)
+            sx = mixdq.act_scale(Xd.reshape(-1, l.K))
+            y = host(mixdq.linear(Xd.reshape(-1, l.K), packed, l.N, w_bits, s, None, 8, sx, dev(b), ws, st))
+            acc = host(mixdq.linear_acc_i32(Xd.reshape(-1, l.K), packed, l.N, w_bits, sx, ws, st))
+            rows = _sample_rows(X2.shape[0], seed=l.index)
+            a_rows, y_rows, bias = X2[rows], y[rows], b
+        assert host(sx)[0] == sx_ref
+        acc_ref, y_ref = orc.linear_a8(np.ascontiguousarray(a_rows), codes, s_ref, sx_ref, bias)
+        torch.cuda.synchronize()
+        assert int(host(st)[0]) == 0
+        assert np.array_equal(acc[rows], acc_ref)
+        _close(y_rows, y_ref)
+    else:
+        if conv:
+            y = host(mixdq.conv3x3(Xd, packed, l.N, w_bits, s, zd, 16, None, dev(b), l.stride, ws, st)).reshape(-1, l.N)
+            rows = _sample_rows(y.shape[0], seed=l.index)
+            a_rows = _window_rows(X, rows, l.stride)
+        else:
+            X2 = X.reshape(-1, l.K)
+            y = host(mixdq.linear(Xd.reshape(-1, l.K), packed, l.N, w_bits, s, zd, 16, None, dev(b), ws, st))
+            rows = _sample_rows(X2.shape[0], seed=l.index)
+            a_rows = X2[rows]
+        y_ref = orc.linear_a16(np.ascontiguousarray(a_rows), codes, s_ref, z_ref, b)
+        torch.cuda.synchronize()
+        assert int(host(st)[0]) == 0
+        _close(y[rows], y_ref)
+
+
+@pytest.mark.parametrize("name,w_bits", [
+    ("ffn1_1280#0", 4), ("ffn1_1280#1", 8), ("ffn2_1280#0", 4), ("attn_1280#0", 4), ("attn_640#0", 8),
+    ("ffn1_640#0", 4), ("kv_1280#0", 8), ("kv_640#0", 4), ("up64_640#0", 4), ("res64_320_320#0", 8),
+    ("res32_1920_640#0", 4), ("res16_2560_1280#0", 4), ("down64_320#0", 4), ("sc64_960#0", 4),
+    ("conv_in#0", 8), ("conv_out#0", 8), ("time_emb1#0", 4), ("add_emb1#0", 8)])
+def test_int8_layers_full_size(name, w_bits):
+    _check_layer(name, w_bits, 8)
+
+
+@pytest.mark.parametrize("name,w_bits", [
+    ("ffn1_1280#0", 3), ("ffn1_1280#1", 4), ("ffn2_1280#0", 8), ("attn_1280#0", 3), ("kv_1280#0", 4),
+    ("res64_320_320#0", 3), ("up32_1280#0", 4), ("res16_2560_1280#0", 8), ("down32_640#0", 3),
+    ("conv_in#0", 8), ("conv_out#0", 8), ("res_time_640#0", 4)])
+def test_weight_only_layers_full_size(name, w_bits):
+    _check_layer(name, w_bits, 16)
+
+
+@pytest.mark.parametrize("name,w_bits", [("ffn1_1280#0", 3), ("ffn1_1280#0", 4), ("ffn2_1280#0", 4),
+                                         ("attn_1280#0", 8)])
+def test_weight_only_sixteen_tokens_full_width(name, w_bits):
+    _check_layer(name, w_bits, 16, rows_override=16)
