@@ -119,7 +119,7 @@ struct TmaSmem {
     static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
     static constexpr int TOTAL = OFF_MISC + 64 + 1024;
-    static constexpr int THREADS = W4 ? 320 : 192;
+    static constexpr int THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
 };
 
 template <int BN, int STAGES, bool W4>
@@ -157,7 +157,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_unpacked + 8 * s, 4);
+            mbar_init(bar_unpacked + 8 * s, 8);
             mbar_init(bar_empty + 8 * s, 1);
         }
         mbar_init(bar_accum, 1);
@@ -287,9 +287,9 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
             const uint8_t* stg = sStg + s * L::STG_BYTES;
             uint8_t* b_stage = sB + s * L::B_BYTES;
-#pragma unroll 4
-            for (int t = 0; t < (BN * 4) / 128; ++t) {
-                const int task = ut + t * 128;
+#pragma unroll
+            for (int t = 0; t < (BN * 4) / 256; ++t) {
+                const int task = ut + t * 256;
                 const int r = task >> 2, j = task & 3;
                 const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
                 uint4 c0, c1;
@@ -401,8 +401,11 @@ struct PersistSmem {
     static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] floats
     static constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
-    static constexpr int TOTAL = OFF_MISC + 64 + 1024;
-    static constexpr int THREADS = W4 ? 320 : 192;
+    static constexpr int OFF_EPI = OFF_MISC + 64;  // per epilogue warp: 32 rows x 64 fp16, rows 144 bytes apart
+    static constexpr int EPI_ROW = 144;
+    static constexpr int EPI_WARP_BYTES = 32 * EPI_ROW;
+    static constexpr int TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
+    static constexpr int THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
 };
 
 template <int BN, int STAGES, bool W4>
@@ -438,7 +441,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_unpacked + 8 * s, 4);
+            mbar_init(bar_unpacked + 8 * s, 8);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -572,46 +575,78 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             }
             const int m = m0 + lg * 32 + lane;
             const bool m_ok = m < p.M;
-            long long out_row = m;
-            if (p.bos && m_ok) {
-                const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
-                out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
-                          (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
-            }
             const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;  // uniform across the warp
-                uint32_t r[32];
-                tmem_ld_32x32(acc + c0, r);
-                tmem_ld_wait();
-                if (!m_ok) continue;
-                const int n = n0 + c0;
-                if (p.acc_out) {
+            if (p.acc_out) {
+                // parity hook: raw accumulators, one row per thread
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (n0 + c0 >= p.N) break;  // uniform across the warp
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc + c0, r);
+                    tmem_ld_wait();
+                    if (!m_ok) continue;
+                    const int n = n0 + c0;
                     int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
                         if (n + j < p.N) dst[j] = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
                 }
-                if (p.Y) {
-                    __half* dst = p.Y + out_row * p.ldy + n;
+            }
+            if (p.Y) {
+                // 64 columns at a time: dequantize in registers (one row per thread), pass through a
+                // small shared-memory tile, and store with eight lanes along each row so that
+                // every store instruction writes whole 128-byte lines
+                uint8_t* stage = smem + L::OFF_EPI + (warp - 2) * L::EPI_WARP_BYTES;
+                for (int c0 = 0; c0 < BN; c0 += 64) {
+                    if (n0 + c0 >= p.N) break;  // uniform across the warp
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        __half2 h[4];
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(acc + c0 + 32 * h, r);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int c = c0 + j + 2 * q;
-                            h[q] = __floats2half2_rn(
-                                fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2 * q])), comb[c], bias[c]),
-                                fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2 * q + 1])), comb[c + 1], bias[c + 1]));
-                        }
-                        if (vec && n + j + 8 <= p.N) {
-                            *reinterpret_cast<uint4*>(dst + j) = *reinterpret_cast<const uint4*>(h);
-                        } else {
-                            const __half* hs = reinterpret_cast<const __half*>(h);
-                            for (int q = 0; q < 8; ++q)
-                                if (n + j + q < p.N) dst[j + q] = hs[q];
+                        for (int j = 0; j < 32; j += 8) {
+                            const int c = c0 + 32 * h + j;
+                            const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+                            const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+                            const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+                            const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+                            __half2 hv[4];
+                            hv[0] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j])), ca.x, ba.x),
+                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 1])), ca.y, ba.y));
+                            hv[1] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2])), ca.z, ba.z),
+                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 3])), ca.w, ba.w));
+                            hv[2] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 4])), cb.x, bb.x),
+                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 5])), cb.y, bb.y));
+                            hv[3] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 6])), cb.z, bb.z),
+                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 7])), cb.w, bb.w));
+                            *reinterpret_cast<uint4*>(stage + lane * L::EPI_ROW + (32 * h + j) * 2) =
+                                *reinterpret_cast<const uint4*>(hv);
                         }
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int it8 = 0; it8 < 8; ++it8) {
+                        const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
+                        const int mm = m0 + lg * 32 + rl;
+                        const int n = n0 + c0 + seg * 8;
+                        if (mm >= p.M || n >= p.N) continue;
+                        long long orow = mm;
+                        if (p.bos) {
+                            const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                            orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                                   (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+                        }
+                        const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * L::EPI_ROW + seg * 16);
+                        __half* dst = p.Y + orow * p.ldy + n;
+                        if (vec && n + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(dst) = v;
+                        } else {
+                            const __half* hs = reinterpret_cast<const __half*>(&v);
+                            for (int q = 0; q < 8; ++q)
+                                if (n + q < p.N) dst[q] = hs[q];
+                        }
+                    }
+                    __syncwarp();
                 }
             }
             // the accumulator may be overwritten once every epilogue warp has read it
@@ -629,9 +664,9 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
             const uint8_t* stg = sStg + s * L::STG_BYTES;
             uint8_t* b_stage = sB + s * L::B_BYTES;
-#pragma unroll 4
-            for (int t = 0; t < (BN * 4) / 128; ++t) {
-                const int task = ut + t * 128;
+#pragma unroll
+            for (int t = 0; t < (BN * 4) / 256; ++t) {
+                const int task = ut + t * 256;
                 const int r = task >> 2, j = task & 3;
                 const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
                 uint4 c0, c1;

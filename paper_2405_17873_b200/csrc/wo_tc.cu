@@ -31,7 +31,10 @@ constexpr int NUM_BARS = 3 * STAGES + 4;
 constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] scales
 constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;                 // [2][BN] biases
 constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
-constexpr int SMEM_TOTAL = OFF_MISC + 64 + 1024;
+constexpr int OFF_EPI = OFF_MISC + 64;  // per epilogue warp: 32 rows x 64 fp16, rows 144 bytes apart
+constexpr int EPI_ROW = 144;
+constexpr int EPI_WARP_BYTES = 32 * EPI_ROW;
+constexpr int SMEM_TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
 constexpr int THREADS = 448;
 constexpr int kFeedWarps = 8;
 
@@ -276,34 +279,56 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
                 ok = false;
                 continue;
             }
-            const int m = m0 + lg * 32 + lane;
-            const bool m_ok = m < p.M;
             const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;
-                uint32_t r[32];
-                tmem_ld_32x32(acc + c0, r);
-                tmem_ld_wait();
-                if (!m_ok) continue;
-                const int n = n0 + c0;
-                __half* dst = p.Y + static_cast<long long>(m) * p.ldy + n;
+            // 64 columns at a time: scale in registers (one row per thread), pass through a small
+            // shared-memory tile, and store with eight lanes along each row so that every store
+            // instruction writes whole 128-byte lines
+            uint8_t* stage = smem + OFF_EPI + (warp - 2) * EPI_WARP_BYTES;
+            for (int c0 = 0; c0 < BN; c0 += 64) {
+                if (n0 + c0 >= p.N) break;  // uniform across the warp
 #pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    __half2 h[4];
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc + c0 + 32 * h, r);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int c = c0 + j + 2 * q;
-                        h[q] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 2 * q]), comb[c], bias[c]),
-                                                 fmaf(__uint_as_float(r[j + 2 * q + 1]), comb[c + 1], bias[c + 1]));
-                    }
-                    if (vec && n + j + 8 <= p.N) {
-                        *reinterpret_cast<uint4*>(dst + j) = *reinterpret_cast<const uint4*>(h);
-                    } else {
-                        const __half* hs = reinterpret_cast<const __half*>(h);
-                        for (int q = 0; q < 8; ++q)
-                            if (n + j + q < p.N) dst[j + q] = hs[q];
+                    for (int j = 0; j < 32; j += 8) {
+                        const int c = c0 + 32 * h + j;
+                        const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+                        const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+                        const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+                        const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+                        __half2 hv[4];
+                        hv[0] = __floats2half2_rn(fmaf(__uint_as_float(r[j]), ca.x, ba.x),
+                                                  fmaf(__uint_as_float(r[j + 1]), ca.y, ba.y));
+                        hv[1] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 2]), ca.z, ba.z),
+                                                  fmaf(__uint_as_float(r[j + 3]), ca.w, ba.w));
+                        hv[2] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 4]), cb.x, bb.x),
+                                                  fmaf(__uint_as_float(r[j + 5]), cb.y, bb.y));
+                        hv[3] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 6]), cb.z, bb.z),
+                                                  fmaf(__uint_as_float(r[j + 7]), cb.w, bb.w));
+                        *reinterpret_cast<uint4*>(stage + lane * EPI_ROW + (32 * h + j) * 2) =
+                            *reinterpret_cast<const uint4*>(hv);
                     }
                 }
+                __syncwarp();
+#pragma unroll
+                for (int it8 = 0; it8 < 8; ++it8) {
+                    const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
+                    const int mm = m0 + lg * 32 + rl;
+                    const int n = n0 + c0 + seg * 8;
+                    if (mm >= p.M || n >= p.N) continue;
+                    const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI_ROW + seg * 16);
+                    __half* dst = p.Y + static_cast<long long>(mm) * p.ldy + n;
+                    if (vec && n + 8 <= p.N) {
+                        *reinterpret_cast<uint4*>(dst) = v;
+                    } else {
+                        const __half* hs = reinterpret_cast<const __half*>(&v);
+                        for (int q = 0; q < 8; ++q)
+                            if (n + q < p.N) dst[q] = hs[q];
+                    }
+                }
+                __syncwarp();
             }
             tc_fence_before_sync();
             __syncwarp();
