@@ -4,8 +4,8 @@
 //   warp 0      TMA producer: fp16 activation tiles (128 rows x 64 k), 128-byte swizzle; a 3x3
 //               convolution reads a 4-D box of the NHWC image shifted by the filter tap
 //   warp 1      tensor-memory owner and MMA issuer (128 x 128 x 16 per instruction)
-//   warps 2..5  epilogue: tensor memory -> registers -> y = fp16(scale[n] * acc + bias[n])
-//   warps 6..13 weight feeders: packed codes straight from global memory into registers,
+//   warps 2..9  epilogue: tensor memory -> registers -> y = fp16(scale[n] * acc + bias[n])
+//   warps 10..17 weight feeders: packed codes straight from global memory into registers,
 //               expanded to the exact fp16 integers (q - z) and written as the swizzled
 //               K-major B tile
 // One CTA per SM walks over output tiles; two accumulators alternate so that the epilogue of
@@ -31,11 +31,11 @@ constexpr int NUM_BARS = 3 * STAGES + 4;
 constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] scales
 constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;                 // [2][BN] biases
 constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
-constexpr int OFF_EPI = OFF_MISC + 64;  // per epilogue warp: 32 rows x 64 fp16, rows 144 bytes apart
-constexpr int EPI_ROW = 144;
+constexpr int OFF_EPI = OFF_MISC + 64;  // per epilogue warp: 32 rows x 32 fp16, rows 80 bytes apart
+constexpr int EPI_ROW = 80;
 constexpr int EPI_WARP_BYTES = 32 * EPI_ROW;
-constexpr int SMEM_TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
-constexpr int THREADS = 448;
+constexpr int SMEM_TOTAL = OFF_EPI + 8 * EPI_WARP_BYTES + 1024;
+constexpr int THREADS = 576;
 constexpr int kFeedWarps = 8;
 
 struct TcParams {
@@ -173,7 +173,7 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, 4);
+            mbar_init(bar_acc_empty + 8 * b, 8);
         }
         *s_abort = 0;
         fence_barrier_init();
@@ -253,9 +253,10 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
             }
         }
         __syncwarp();
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // ------------------------------------------------------------ epilogue
         const int lg = warp & 3;
+        const int chalf = (warp - 2) >> 2;  // which half of the tile's columns this warp handles
         const int et = tid - 64;
         const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
         bool ok = true;
@@ -266,12 +267,12 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
             const uint32_t use = static_cast<uint32_t>(t >> 1);
             float* comb = s_comb + buf * BN;
             float* bias = s_bias + buf * BN;
-            {
+            if (et < BN) {
                 const int n = n0 + et;
                 comb[et] = n < p.N ? __ldg(p.w_scale + n) : 0.f;
                 bias[et] = (n < p.N && p.bias) ? __half2float(p.bias[n]) : 0.f;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (ok) ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, s_abort);
             tc_fence_after_sync();
             const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
@@ -280,43 +281,41 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
                 continue;
             }
             const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
-            // 64 columns at a time: scale in registers (one row per thread), pass through a small
-            // shared-memory tile, and store with eight lanes along each row so that every store
-            // instruction writes whole 128-byte lines
+            // 32 columns at a time: scale in registers (one row per thread), pass through a small
+            // shared-memory tile, and store with four lanes along each row so that every store
+            // instruction writes whole 32-byte sectors of eight rows
             uint8_t* stage = smem + OFF_EPI + (warp - 2) * EPI_WARP_BYTES;
-            for (int c0 = 0; c0 < BN; c0 += 64) {
+            const int row_base = m0 + lg * 32;
+            for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
                 if (n0 + c0 >= p.N) break;  // uniform across the warp
+                uint32_t r[32];
+                tmem_ld_32x32(acc + c0, r);
+                tmem_ld_wait();
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r[32];
-                    tmem_ld_32x32(acc + c0 + 32 * h, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        const int c = c0 + 32 * h + j;
-                        const float4 ca = *reinterpret_cast<const float4*>(comb + c);
-                        const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
-                        const float4 ba = *reinterpret_cast<const float4*>(bias + c);
-                        const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
-                        __half2 hv[4];
-                        hv[0] = __floats2half2_rn(fmaf(__uint_as_float(r[j]), ca.x, ba.x),
-                                                  fmaf(__uint_as_float(r[j + 1]), ca.y, ba.y));
-                        hv[1] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 2]), ca.z, ba.z),
-                                                  fmaf(__uint_as_float(r[j + 3]), ca.w, ba.w));
-                        hv[2] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 4]), cb.x, bb.x),
-                                                  fmaf(__uint_as_float(r[j + 5]), cb.y, bb.y));
-                        hv[3] = __floats2half2_rn(fmaf(__uint_as_float(r[j + 6]), cb.z, bb.z),
-                                                  fmaf(__uint_as_float(r[j + 7]), cb.w, bb.w));
-                        *reinterpret_cast<uint4*>(stage + lane * EPI_ROW + (32 * h + j) * 2) =
-                            *reinterpret_cast<const uint4*>(hv);
-                    }
+                for (int j = 0; j < 32; j += 8) {
+                    const int c = c0 + j;
+                    const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+                    const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+                    const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+                    const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+                    uint4 o;
+                    o.x = h2u(__floats2half2_rn(fmaf(__uint_as_float(r[j]), ca.x, ba.x),
+                                                fmaf(__uint_as_float(r[j + 1]), ca.y, ba.y)));
+                    o.y = h2u(__floats2half2_rn(fmaf(__uint_as_float(r[j + 2]), ca.z, ba.z),
+                                                fmaf(__uint_as_float(r[j + 3]), ca.w, ba.w)));
+                    o.z = h2u(__floats2half2_rn(fmaf(__uint_as_float(r[j + 4]), cb.x, bb.x),
+                                                fmaf(__uint_as_float(r[j + 5]), cb.y, bb.y)));
+                    o.w = h2u(__floats2half2_rn(fmaf(__uint_as_float(r[j + 6]), cb.z, bb.z),
+                                                fmaf(__uint_as_float(r[j + 7]), cb.w, bb.w)));
+                    *reinterpret_cast<uint4*>(stage + lane * EPI_ROW + j * 2) = o;
                 }
                 __syncwarp();
+                const int seg = lane & 3;
+                const int n = n0 + c0 + seg * 8;
 #pragma unroll
-                for (int it8 = 0; it8 < 8; ++it8) {
-                    const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
-                    const int mm = m0 + lg * 32 + rl;
-                    const int n = n0 + c0 + seg * 8;
+                for (int it4 = 0; it4 < 4; ++it4) {
+                    const int rl = it4 * 8 + (lane >> 2);
+                    const int mm = row_base + rl;
                     if (mm >= p.M || n >= p.N) continue;
                     const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI_ROW + seg * 16);
                     __half* dst = p.Y + static_cast<long long>(mm) * p.ldy + n;
@@ -337,7 +336,7 @@ wo_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const TcParams p, int n
     } else {
         // ------------------------------------------------------------ weight feeders
         // thread -> (row of the tile, which 32-code half of the 64-wide k-block)
-        const int ft = tid - 192;
+        const int ft = tid - 320;
         const int half = ft & 1;
         const int r = ft >> 1;
         int it = 0;
