@@ -109,7 +109,9 @@ template <int BN, int STAGES, bool W4>
 struct TmaSmem {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
-    static constexpr int STG_BYTES = W4 ? BN * (BK / 2) : 0;
+    // packed int4 rows land in the last half of the B slot and are expanded in place
+    static constexpr int STG_BYTES = 0;
+    static constexpr int STG_OFFSET = BN * (BK / 2);
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
@@ -133,7 +135,6 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                                                ~static_cast<uintptr_t>(1023));
     uint8_t* sA = smem + L::OFF_A;
     uint8_t* sB = smem + L::OFF_B;
-    uint8_t* sStg = smem + L::OFF_STG;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
     float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
     float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
@@ -193,7 +194,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 if (!mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort)) break;
                 mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
                 const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
-                const uint32_t dst_b = W4 ? smem_u32(sStg + s * L::STG_BYTES) : smem_u32(sB + s * L::B_BYTES);
+                const uint32_t dst_b = smem_u32(sB + s * L::B_BYTES + (W4 ? L::STG_OFFSET : 0));
                 const int kb = kb_begin + i;
                 if (p.conv) {
                     const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
@@ -285,13 +286,21 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             const int s = i % STAGES;
             const uint32_t round = static_cast<uint32_t>(i / STAGES);
             if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
-            const uint8_t* stg = sStg + s * L::STG_BYTES;
+            const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
             uint8_t* b_stage = sB + s * L::B_BYTES;
+            // in place: every thread first reads its packed runs, then (after all have) writes
+            uint4 wv[(BN * 4) / 256];
+#pragma unroll
+            for (int t = 0; t < (BN * 4) / 256; ++t) {
+                const int task = ut + t * 256;
+                wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
+            }
+            asm volatile("bar.sync 2, 256;" ::: "memory");
 #pragma unroll
             for (int t = 0; t < (BN * 4) / 256; ++t) {
                 const int task = ut + t * 256;
                 const int r = task >> 2, j = task & 3;
-                const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
+                const uint4 w = wv[t];
                 uint4 c0, c1;
                 c0.x = (w.x << 4) & 0xF0F0F0F0u;
                 c0.y = w.x & 0xF0F0F0F0u;
@@ -392,7 +401,9 @@ template <int BN, int STAGES, bool W4>
 struct PersistSmem {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
-    static constexpr int STG_BYTES = W4 ? BN * (BK / 2) : 0;
+    // packed int4 rows land in the last half of the B slot and are expanded in place
+    static constexpr int STG_BYTES = 0;
+    static constexpr int STG_OFFSET = BN * (BK / 2);
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
@@ -419,7 +430,6 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                                                ~static_cast<uintptr_t>(1023));
     uint8_t* sA = smem + L::OFF_A;
     uint8_t* sB = smem + L::OFF_B;
-    uint8_t* sStg = smem + L::OFF_STG;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
     float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
     float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
@@ -486,7 +496,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     if (!ok) break;
                     mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
                     const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
-                    const uint32_t dst_b = W4 ? smem_u32(sStg + s * L::STG_BYTES) : smem_u32(sB + s * L::B_BYTES);
+                    const uint32_t dst_b = smem_u32(sB + s * L::B_BYTES + (W4 ? L::STG_OFFSET : 0));
                     if (p.conv) {
                         const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
                         const int kh = tap / 3, kw = tap - 3 * kh;
@@ -662,13 +672,21 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             const int s = it % STAGES;
             const uint32_t round = static_cast<uint32_t>(it / STAGES);
             if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
-            const uint8_t* stg = sStg + s * L::STG_BYTES;
+            const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
             uint8_t* b_stage = sB + s * L::B_BYTES;
+            // in place: every thread first reads its packed runs, then (after all have) writes
+            uint4 wv[(BN * 4) / 256];
+#pragma unroll
+            for (int t = 0; t < (BN * 4) / 256; ++t) {
+                const int task = ut + t * 256;
+                wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
+            }
+            asm volatile("bar.sync 2, 256;" ::: "memory");
 #pragma unroll
             for (int t = 0; t < (BN * 4) / 256; ++t) {
                 const int task = ut + t * 256;
                 const int r = task >> 2, j = task & 3;
-                const uint4 w = *reinterpret_cast<const uint4*>(stg + r * (BK / 2) + j * 16);
+                const uint4 w = wv[t];
                 uint4 c0, c1;
                 c0.x = (w.x << 4) & 0xF0F0F0F0u;
                 c0.y = w.x & 0xF0F0F0F0u;
@@ -842,9 +860,9 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     }
     if (tiles >= num_sms && p.force_splits <= 0) {
         if (wide)
-            return w4 ? launch_persistent<256, 3, true>(ta, tw, tp, num_sms, stream)
+            return w4 ? launch_persistent<256, 4, true>(ta, tw, tp, num_sms, stream)
                       : launch_persistent<256, 4, false>(ta, tw, tp, num_sms, stream);
-        return w4 ? launch_persistent<128, 5, true>(ta, tw, tp, num_sms, stream)
+        return w4 ? launch_persistent<128, 6, true>(ta, tw, tp, num_sms, stream)
                   : launch_persistent<128, 6, false>(ta, tw, tp, num_sms, stream);
     }
     int splits = pick_splits(tiles, tp.k_blocks);
@@ -853,9 +871,9 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;
     }
     if (wide)
-        return w4 ? launch_tma<256, 3, true>(ta, tw, tp, splits, stream)
+        return w4 ? launch_tma<256, 4, true>(ta, tw, tp, splits, stream)
                   : launch_tma<256, 4, false>(ta, tw, tp, splits, stream);
-    return w4 ? launch_tma<128, 5, true>(ta, tw, tp, splits, stream)
+    return w4 ? launch_tma<128, 6, true>(ta, tw, tp, splits, stream)
               : launch_tma<128, 6, false>(ta, tw, tp, splits, stream);
 }
 
