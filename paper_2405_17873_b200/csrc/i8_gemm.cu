@@ -497,6 +497,102 @@ __global__ void simple_kernel(const uint8_t* __restrict__ packed, long long pitc
         p.Y[static_cast<long long>(m) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n] = p.bos_out[n];
 }
 
+// Short reductions (K <= 64, int8 weights): the first convolution of the UNet has 4 input
+// channels, i.e. K = 36.  A CTA quantizes the gathered inputs of 32 output rows into shared
+// memory once; each thread then keeps one weight row in registers and produces that channel
+// for all 32 rows with dp4a, so the stores of a row are contiguous across threads.
+constexpr int kSmallKRows = 32;
+
+__global__ void __launch_bounds__(128)
+small_k_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, int amode)
+{
+    __shared__ __align__(16) int8_t xq[kSmallKRows][64];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.x * kSmallKRows;
+    const float sx = __ldg(p.act_scale);
+    const float inv = __fdiv_rn(1.f, sx);
+    for (int idx = tid; idx < kSmallKRows * 64; idx += 128) {
+        const int r = idx >> 6, k = idx & 63;
+        const int m = m0 + r;
+        int q = 0;
+        if (m < p.M && k < p.K) {
+            float x = 0.f;
+            bool in = true;
+            if (amode == A_CONV3) {
+                const int hw = p.Ho * p.Wo;
+                const int b = m / hw, rem = m - b * hw;
+                const int ho = rem / p.Wo, wo = rem - ho * p.Wo;
+                const int tap = k / p.Cin, c = k - tap * p.Cin;
+                const int hi = ho * p.stride - 1 + tap / 3, wi = wo * p.stride - 1 + tap % 3;
+                in = hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                if (in) x = __half2float(p.X[((static_cast<long long>(b) * p.H + hi) * p.W + wi) * p.Cin + c]);
+            } else {
+                long long row = m;
+                if (amode == A_BOS) {
+                    const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                    row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                          (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+                }
+                x = __half2float(p.X[row * p.ldx + k]);
+            }
+            if (in) {
+                const float y = fminf(fmaxf(fmaf(x, inv, kMagic), kMagic - 127.f), kMagic + 127.f);
+                q = static_cast<int>(__float_as_uint(y)) - 0x4B400000;
+            }
+        }
+        xq[r][k] = static_cast<int8_t>(q);
+    }
+    __syncthreads();
+    const int words = (p.K + 3) >> 2;
+    for (int n = tid; n < p.N; n += 128) {
+        int w[16];
+        const uint8_t* wrow = packed + static_cast<long long>(n) * pitch;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            w[j] = 0;
+            if (j < words) {
+                // bytes beyond K inside the last word are padding of the packed row (zero codes)
+                const int byte0 = 4 * j;
+                uint32_t v = 0;
+                for (int b = 0; b < 4; ++b)
+                    if (byte0 + b < p.K) v |= static_cast<uint32_t>(wrow[byte0 + b]) << (8 * b);
+                w[j] = static_cast<int>(v);
+            }
+        }
+        const float comb = p.w_scale ? sx * __ldg(p.w_scale + n) : 0.f;
+        const float bias = p.bias ? __half2float(p.bias[n]) : 0.f;
+        for (int r = 0; r < kSmallKRows; ++r) {
+            const int m = m0 + r;
+            if (m >= p.M) break;
+            const int4* xr = reinterpret_cast<const int4*>(xq[r]);
+            int acc = 0;
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+                const int4 xv = xr[j4];
+                acc = __dp4a(xv.x, w[4 * j4], acc);
+                acc = __dp4a(xv.y, w[4 * j4 + 1], acc);
+                acc = __dp4a(xv.z, w[4 * j4 + 2], acc);
+                acc = __dp4a(xv.w, w[4 * j4 + 3], acc);
+            }
+            if (p.acc_out) p.acc_out[static_cast<long long>(m) * p.N + n] = acc;
+            if (p.Y) {
+                long long orow = m;
+                if (amode == A_BOS) {
+                    const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                    orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                           (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+                }
+                p.Y[orow * p.ldy + n] = __float2half_rn(fmaf(static_cast<float>(acc), comb, bias));
+            }
+        }
+        if (amode == A_BOS && p.Y && blockIdx.x == 0)
+            for (int b = 0; b < p.batch; ++b)
+                p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n] = p.bos_out[n];
+    }
+}
+
 template <int BN, int STAGES, bool W4, int AMODE>
 int launch_tc(const Params& p, const void* packed, int64_t pitch, int splits, cudaStream_t stream)
 {
@@ -567,6 +663,12 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1)
         return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
 
+    if (!tc_ok && !w4 && p.K <= 64) {
+        const unsigned grid = static_cast<unsigned>(ceil_div(p.M, kSmallKRows));
+        const long long pitch_ll = pitch;
+        return launch_pdl(small_k_kernel, dim3(grid), dim3(128), 0, stream, 1, static_cast<const uint8_t*>(packed),
+                          pitch_ll, p, amode);
+    }
     if (!tc_ok) {
         const long long total = static_cast<long long>(p.M) * p.N;
         const unsigned grid = static_cast<unsigned>(ceil_div(total, 128));
