@@ -113,13 +113,13 @@ int mixdq_act_scale_from_absmax(const float* amax, float* scale_out, void* strea
 /*
  * Bytes of scratch memory the layer calls below need for a given problem (HOST `out`).
  * rows = output rows (tokens or output pixels), N, K as in the layer call.  The scratch
- * must be 256-byte aligned and zero-filled once before its first use; the kernels leave
- * the part that has to be zero (the first bytes: counters and partial sums of a split
- * reduction) zero-filled again.  Calls that share a workspace must not overlap on the GPU.
+ * must be 256-byte aligned.  Nothing in it has to be initialised or to survive between calls
+ * (a call clears what it needs cleared), so one buffer of the largest size can serve every
+ * layer of a model -- as long as the calls that share it do not overlap on the GPU.
  * A result of 0 means the call runs without scratch.  The workspace is optional for every
  * call (NULL / 0 bytes): without it the int8 layers run as one fused kernel that quantizes
- * the activations while it feeds the tensor cores; with it, larger layers first quantize
- * the activations once into the workspace and then run a GEMM fed entirely by TMA.
+ * the activations while it feeds the tensor cores; with it, the activations are first
+ * quantized once into the workspace and the GEMM is then fed entirely by TMA.
  */
 int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_bits, int act_bits,
                           size_t* out);

@@ -682,18 +682,23 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     // split the reduction across CTAs when the output tiles alone cannot fill the GPU
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, 128);
     int splits = 1;
-    if (workspace && ws_bytes >= split_bytes && tiles < 96 && p.k_blocks >= 8) {
+    const bool split_room = workspace && ws_bytes >= split_bytes;
+    if (split_room && tiles < 96 && p.k_blocks >= 8) {
         splits = static_cast<int>(148 / tiles);
         if (splits > p.k_blocks / 4) splits = p.k_blocks / 4;
         if (splits < 1) splits = 1;
     }
     if (p.force_splits > 0) {
-        if (p.force_splits > 1 && !(workspace && ws_bytes >= split_bytes)) return MIXDQ_ERR_WORKSPACE;
+        if (p.force_splits > 1 && !split_room) return MIXDQ_ERR_WORKSPACE;
         splits = p.force_splits > p.k_blocks ? p.k_blocks : p.force_splits;
     }
     if (splits > 1) {
-        p.ws_tickets = static_cast<int32_t*>(workspace);
-        p.ws_acc = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + round_up(tiles * 4, 256));
+        // a workspace shared between layers may hold another layer's int8 activations here, so the
+        // counters and partial sums of the split reduction are cleared, not assumed zero
+        uint8_t* region = static_cast<uint8_t*>(workspace);
+        MIXDQ_CUDA_TRY(cudaMemsetAsync(region, 0, split_bytes, stream));
+        p.ws_tickets = reinterpret_cast<int32_t*>(region);
+        p.ws_acc = reinterpret_cast<int32_t*>(region + round_up(tiles * 4, 256));
     }
 #define MIXDQ_DISPATCH(W4V)                                                                    \
     switch (amode) {                                                                           \
