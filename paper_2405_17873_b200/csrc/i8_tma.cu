@@ -188,23 +188,43 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 ho0 = rem / p.Wo;
                 wo0 = rem - ho0 * p.Wo;
             }
+            // single-thread loop: all indices are carried along instead of being recomputed
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            uint32_t s = 0, ph = 1;
+            int tap = 0, cb = 0, kh = 0, kw = 0;
+            if (p.conv) {
+                tap = kb_begin / p.cblocks;
+                cb = kb_begin - tap * p.cblocks;
+                kh = tap / 3;
+                kw = tap - 3 * kh;
+            }
+            int kx_tap = tap * p.Cin;           // conv: first reduction index of the tap
+            int xa = kb_begin * BK, xb = kb_begin * ROW_BYTES;
             for (int i = 0; i < nkb; ++i) {
-                const int s = i % STAGES;
-                const uint32_t round = static_cast<uint32_t>(i / STAGES);
-                if (!mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort)) break;
-                mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
-                const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
-                const uint32_t dst_b = smem_u32(sB + s * L::B_BYTES + (W4 ? L::STG_OFFSET : 0));
-                const int kb = kb_begin + i;
+                if (!mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;
+                const uint32_t full = bar_full + 8 * s;
+                mbar_arrive_expect_tx(full, L::A_BYTES + BN * ROW_BYTES);
                 if (p.conv) {
-                    const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
-                    const int kh = tap / 3, kw = tap - 3 * kh;
-                    tma_load_4d(dst_a, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, bar_full + 8 * s);
-                    const int kx = tap * p.Cin + cb * BK;
-                    tma_load_2d(dst_b, &tmap_w, W4 ? kx / 2 : kx, n0, bar_full + 8 * s);
+                    tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
+                    const int kx = kx_tap + cb * BK;
+                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
+                    if (++cb == p.cblocks) {
+                        cb = 0;
+                        kx_tap += p.Cin;
+                        if (++kw == 3) {
+                            kw = 0;
+                            ++kh;
+                        }
+                    }
                 } else {
-                    tma_load_2d(dst_a, &tmap_a, kb * BK, m0, bar_full + 8 * s);
-                    tma_load_2d(dst_b, &tmap_w, kb * ROW_BYTES, n0, bar_full + 8 * s);
+                    tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
+                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
+                    xa += BK;
+                    xb += ROW_BYTES;
+                }
+                if (++s == STAGES) {
+                    s = 0;
+                    ph ^= 1;
                 }
             }
         }
@@ -214,19 +234,23 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
             bool ok = true;
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            uint32_t s = 0, ph = 0;
             for (int i = 0; i < nkb; ++i) {
-                const int s = i % STAGES;
-                const uint32_t round = static_cast<uint32_t>(i / STAGES);
-                ok = mbar_wait(bar_full + 8 * s, round & 1, s_abort);
-                if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, round & 1, s_abort);
+                ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
+                if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, ph, s_abort);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint64_t a_desc = smem_desc_sw128(smem_u32(sA + s * L::A_BYTES));
-                const uint64_t b_desc = smem_desc_sw128(smem_u32(sB + s * L::B_BYTES));
+                const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
+                const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
 #pragma unroll
                 for (int k = 0; k < BK / 32; ++k)
                     mma_i8_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0);
                 tc_commit(bar_empty + 8 * s);
+                if (++s == STAGES) {
+                    s = 0;
+                    ph ^= 1;
+                }
             }
             if (ok) tc_commit(bar_accum);
         }
@@ -326,58 +350,67 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     __syncthreads();
     if (splits > 1) cluster_sync_all();
     if (!*s_abort) {
+        // a thread keeps one group of four columns (its factors stay in registers) and walks
+        // down the rows; consecutive threads take consecutive column groups
         const int rows_per = BM / splits;
         constexpr int CHUNKS = BN / 4;
-        const bool vec = ((p.ldy & 3) == 0);
-        for (int item = tid; item < rows_per * CHUNKS; item += L::THREADS) {
-            const int rl = item / CHUNKS, chunk = item - rl * CHUNKS;
-            const int row = rank * rows_per + rl;
-            const int m = m0 + row, n = n0 + chunk * 4;
-            if (m >= p.M || n >= p.N) continue;
-            const uint32_t off = smem_u32(smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4));
-            int4 acc = make_int4(0, 0, 0, 0);
-            if (splits == 1) {
-                acc = *reinterpret_cast<const int4*>(smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4));
-            } else {
-                int4 v[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = (q < splits) ? ld_cluster_v4(off, q) : make_int4(0, 0, 0, 0);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    acc.x += v[q].x;
-                    acc.y += v[q].y;
-                    acc.z += v[q].z;
-                    acc.w += v[q].w;
-                }
-            }
-            if (p.acc_out) {
-                int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
-                const int a[4] = {acc.x, acc.y, acc.z, acc.w};
-                for (int j = 0; j < 4; ++j)
-                    if (n + j < p.N) dst[j] = W4 ? (a[j] >> 4) : a[j];
-            }
-            if (p.Y) {
-                long long out_row = m;
-                if (p.bos) {
-                    const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
-                    out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
-                              (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
-                }
-                const int c = chunk * 4;
-                const float4 cb = *reinterpret_cast<const float4*>(s_comb + c);
-                const float4 bb = *reinterpret_cast<const float4*>(s_bias + c);
-                __half2 h[2];
-                h[0] = __floats2half2_rn(fmaf(static_cast<float>(acc.x), cb.x, bb.x),
-                                         fmaf(static_cast<float>(acc.y), cb.y, bb.y));
-                h[1] = __floats2half2_rn(fmaf(static_cast<float>(acc.z), cb.z, bb.z),
-                                         fmaf(static_cast<float>(acc.w), cb.w, bb.w));
-                __half* dst = p.Y + out_row * p.ldy + n;
-                if (vec && n + 4 <= p.N) {
-                    *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
+        constexpr int RSTEP = L::THREADS / CHUNKS;
+        static_assert(L::THREADS % CHUNKS == 0, "threads must tile the column groups");
+        const int chunk = tid % CHUNKS;
+        const int n = n0 + chunk * 4;
+        const bool vec = ((p.ldy & 3) == 0) && n + 4 <= p.N;
+        const float4 cb = *reinterpret_cast<const float4*>(s_comb + chunk * 4);
+        const float4 bb = *reinterpret_cast<const float4*>(s_bias + chunk * 4);
+        if (n < p.N) {
+#pragma unroll 2
+            for (int rl = tid / CHUNKS; rl < rows_per; rl += RSTEP) {
+                const int row = rank * rows_per + rl;
+                const int m = m0 + row;
+                if (m >= p.M) break;
+                const uint8_t* src = smem + row * (BN * 4) + ((chunk ^ (row & 7)) << 4);
+                int4 acc;
+                if (splits == 1) {
+                    acc = *reinterpret_cast<const int4*>(src);
                 } else {
-                    const __half* hs = reinterpret_cast<const __half*>(h);
+                    acc = make_int4(0, 0, 0, 0);
+                    const uint32_t off = smem_u32(src);
+                    int4 v[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) v[q] = (q < splits) ? ld_cluster_v4(off, q) : make_int4(0, 0, 0, 0);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        acc.x += v[q].x;
+                        acc.y += v[q].y;
+                        acc.z += v[q].z;
+                        acc.w += v[q].w;
+                    }
+                }
+                if (p.acc_out) {
+                    int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
+                    const int a[4] = {acc.x, acc.y, acc.z, acc.w};
                     for (int j = 0; j < 4; ++j)
-                        if (n + j < p.N) dst[j] = hs[j];
+                        if (n + j < p.N) dst[j] = W4 ? (a[j] >> 4) : a[j];
+                }
+                if (p.Y) {
+                    long long out_row = m;
+                    if (p.bos) {
+                        const int prompt = m / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                        out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                                  (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+                    }
+                    __half2 h[2];
+                    h[0] = __floats2half2_rn(fmaf(static_cast<float>(acc.x), cb.x, bb.x),
+                                             fmaf(static_cast<float>(acc.y), cb.y, bb.y));
+                    h[1] = __floats2half2_rn(fmaf(static_cast<float>(acc.z), cb.z, bb.z),
+                                             fmaf(static_cast<float>(acc.w), cb.w, bb.w));
+                    __half* dst = p.Y + out_row * p.ldy + n;
+                    if (vec) {
+                        *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
+                    } else {
+                        const __half* hs = reinterpret_cast<const __half*>(h);
+                        for (int j = 0; j < 4; ++j)
+                            if (n + j < p.N) dst[j] = hs[j];
+                    }
                 }
             }
         }
@@ -477,7 +510,9 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
-            int it = 0;  // k-blocks issued so far, over all tiles
+            // single-thread loop: all indices are carried along instead of being recomputed
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            uint32_t s = 0, ph = 1;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = blockIdx.x + t * gridDim.x;
@@ -489,23 +524,33 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     ho0 = rem / p.Wo;
                     wo0 = rem - ho0 * p.Wo;
                 }
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t round = static_cast<uint32_t>(it / STAGES);
-                    ok = mbar_wait(bar_empty + 8 * s, (round & 1) ^ 1, s_abort);
+                int cb = 0, kh = 0, kw = 0, kx_tap = 0, xa = 0, xb = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(bar_full + 8 * s, L::A_BYTES + BN * ROW_BYTES);
-                    const uint32_t dst_a = smem_u32(sA + s * L::A_BYTES);
-                    const uint32_t dst_b = smem_u32(sB + s * L::B_BYTES + (W4 ? L::STG_OFFSET : 0));
+                    const uint32_t full = bar_full + 8 * s;
+                    mbar_arrive_expect_tx(full, L::A_BYTES + BN * ROW_BYTES);
                     if (p.conv) {
-                        const int tap = kb / p.cblocks, cb = kb - tap * p.cblocks;
-                        const int kh = tap / 3, kw = tap - 3 * kh;
-                        tma_load_4d(dst_a, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, bar_full + 8 * s);
-                        const int kx = tap * p.Cin + cb * BK;
-                        tma_load_2d(dst_b, &tmap_w, W4 ? kx / 2 : kx, n0, bar_full + 8 * s);
+                        tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
+                        const int kx = kx_tap + cb * BK;
+                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
+                        if (++cb == p.cblocks) {
+                            cb = 0;
+                            kx_tap += p.Cin;
+                            if (++kw == 3) {
+                                kw = 0;
+                                ++kh;
+                            }
+                        }
                     } else {
-                        tma_load_2d(dst_a, &tmap_a, kb * BK, m0, bar_full + 8 * s);
-                        tma_load_2d(dst_b, &tmap_w, kb * ROW_BYTES, n0, bar_full + 8 * s);
+                        tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
+                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
+                        xa += BK;
+                        xb += ROW_BYTES;
+                    }
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1;
                     }
                 }
             }
@@ -515,7 +560,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
-            int it = 0;
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t & 1;
@@ -524,19 +570,21 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t acc = tmem_base + buf * BN;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t round = static_cast<uint32_t>(it / STAGES);
-                    ok = mbar_wait(bar_full + 8 * s, round & 1, s_abort);
-                    if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, round & 1, s_abort);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
+                    if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, ph, s_abort);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint64_t a_desc = smem_desc_sw128(smem_u32(sA + s * L::A_BYTES));
-                    const uint64_t b_desc = smem_desc_sw128(smem_u32(sB + s * L::B_BYTES));
+                    const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
+                    const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
                         mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
                     tc_commit(bar_empty + 8 * s);
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1;
+                    }
                 }
                 if (ok) tc_commit(bar_acc_full + 8 * buf);
             }
