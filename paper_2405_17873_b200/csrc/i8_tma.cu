@@ -103,7 +103,135 @@ struct TmaParams {
     long long ldy;
     int32_t* acc_out;
     int32_t* status;
+    int small_acc;  // every |accumulator| (W4: after the >> 4) stays below 2^22
+    int tma_store;  // Y is written through its tensor map (row-contiguous output, 16-byte aligned rows)
 };
+
+// Staging tile of one epilogue warp, 32 rows x 64 fp16: dense 128-byte rows with the 128-byte swizzle
+// when a TMA store takes it from there, else rows 144 bytes apart (conflict-free both ways) for the
+// warp's own coalesced stores.  Tiles are 1024-byte aligned (the swizzle pattern follows the address).
+constexpr int EPI_ROW = 144;
+constexpr int EPI_WARP_BYTES = 5120;
+static_assert(32 * EPI_ROW <= EPI_WARP_BYTES && EPI_WARP_BYTES % 1024 == 0, "staging tile");
+
+// int32 accumulator -> float.  W4 accumulators carry the factor 16 of the nibble placement, removed
+// here by an exact shift.  SMALL: |v| < 2^22, so adding v to the bit pattern of 1.5 * 2^23 and
+// subtracting that constant is exact -- two full-rate instructions instead of a quarter-rate convert.
+template <bool W4, bool SMALL>
+__device__ __forceinline__ float acc_to_float(uint32_t r)
+{
+    const int32_t v = W4 ? (static_cast<int32_t>(r) >> 4) : static_cast<int32_t>(r);
+    if (SMALL) return __int_as_float(0x4B400000 + v) - 12582912.f;
+    return static_cast<float>(v);
+}
+
+// One warp's share of an output tile: 32 accumulator rows (one per lane, tensor-memory lanes of
+// `acc`) x `ncols` columns.  64 columns at a time: dequantize in registers, pass through the warp's
+// staging tile, and store with eight lanes along each row so that every store instruction writes
+// whole 128-byte lines.  comb / bias: per-column factors of the tile in shared memory.  acc2_off != 0:
+// a second accumulator that many columns further on holds the other half of the sum.
+template <bool W4, bool SMALL, bool TMA>
+__device__ __forceinline__ void store_rows_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                     const float* bias, uint8_t* stage, const TmaParams& p,
+                                                     const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+{
+    const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
+    if (TMA && m_first >= p.M) return;  // uniform across the warp
+    for (int c0 = 0; c0 < ncols; c0 += 64) {
+        if (n0 + c0 >= p.N) break;  // uniform across the warp
+        if (TMA) {
+            // the previous bulk store must have read the staging tile before it is overwritten
+            if (lane == 0) tma_store_wait_read();
+            __syncwarp();
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t r[32];
+            tmem_ld_32x32(acc + c0 + 32 * h, r);
+            if (acc2_off) {
+                uint32_t r2[32];
+                tmem_ld_32x32(acc + acc2_off + c0 + 32 * h, r2);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] += r2[j];
+            } else {
+                tmem_ld_wait();
+            }
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                const int c = c0 + 32 * h + j;
+                const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+                const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+                const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+                const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+                __half2 hv[4];
+                hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j]), ca.x, ba.x),
+                                          fmaf(acc_to_float<W4, SMALL>(r[j + 1]), ca.y, ba.y));
+                hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 2]), ca.z, ba.z),
+                                          fmaf(acc_to_float<W4, SMALL>(r[j + 3]), ca.w, ba.w));
+                hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 4]), cb.x, bb.x),
+                                          fmaf(acc_to_float<W4, SMALL>(r[j + 5]), cb.y, bb.y));
+                hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 6]), cb.z, bb.z),
+                                          fmaf(acc_to_float<W4, SMALL>(r[j + 7]), cb.w, bb.w));
+                const int chunk = (32 * h + j) >> 3;  // 16-byte chunk of the row
+                uint8_t* dst = TMA ? stage + lane * 128 + ((chunk ^ (lane & 7)) << 4) : stage + lane * EPI_ROW + chunk * 16;
+                *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(hv);
+            }
+        }
+        if (TMA) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(tmap_y, smem_u32(stage), n0 + c0, m_first);
+                tma_store_commit();
+            }
+            continue;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int it8 = 0; it8 < 8; ++it8) {
+            const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
+            const int mm = m_first + rl;
+            const int n = n0 + c0 + seg * 8;
+            if (mm >= p.M || n >= p.N) continue;
+            long long orow = mm;
+            if (p.bos) {
+                const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                       (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+            }
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI_ROW + seg * 16);
+            __half* dst = p.Y + orow * p.ldy + n;
+            if (vec && n + 8 <= p.N) {
+                *reinterpret_cast<uint4*>(dst) = v;
+            } else {
+                const __half* hs = reinterpret_cast<const __half*>(&v);
+                for (int q = 0; q < 8; ++q)
+                    if (n + q < p.N) dst[q] = hs[q];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// Picks the instantiation for the launch's accumulator range and store route (both uniform).
+template <bool W4>
+__device__ __forceinline__ void store_rows_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                    const float* bias, uint8_t* stage, const TmaParams& p,
+                                                    const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+{
+    if (p.tma_store) {
+        if (p.small_acc)
+            store_rows_from_tmem<W4, true, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+        else
+            store_rows_from_tmem<W4, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+    } else {
+        if (p.small_acc)
+            store_rows_from_tmem<W4, true, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+        else
+            store_rows_from_tmem<W4, false, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+    }
+}
 
 template <int BN, int STAGES, bool W4>
 struct TmaSmem {
@@ -121,13 +249,50 @@ struct TmaSmem {
     static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
     static constexpr int TOTAL = OFF_MISC + 64 + 1024;
-    static constexpr int THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
+    // warps: 0 activation producer, 1 MMA issuer, 2-5 epilogue, 6-9 epilogue helpers (the other half
+    // of the tile's columns), W4: 6-13 nibble expansion during the main loop
+    static constexpr int WORK_THREADS = W4 ? 448 : 320;
+    static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
+    // One thread issues a 128-wide MMA about every 68 cycles, the tensor core retires it in 64: a
+    // lone issuer, which also waits and commits once per k-block, cannot keep the pipe busy.  Narrow
+    // tiles therefore get a second issuer: even k-blocks accumulate into one accumulator, odd ones
+    // into another, and the epilogue adds the two (integer adds: exact).
+    static constexpr bool DUAL = BN == 128;
+    static constexpr int MMA2_WARP = B_WARP + 1;
+    static constexpr int THREADS = WORK_THREADS + 32 + (DUAL ? 32 : 0);
+    static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
 };
+
+// The k-blocks first, first + step, ... of one output tile: wait for the stage, issue its four
+// MMAs into `acc`, hand the stage back.  Runs in a single thread.
+template <int BN, int STAGES, class L>
+__device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t bar_ready,
+                                               uint32_t bar_empty, uint32_t a0, uint32_t b0, volatile int* s_abort)
+{
+    constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
+    uint32_t s = first, ph = 0;  // first < STAGES
+    for (int i = first; i < nkb; i += step) {
+        if (!mbar_wait(bar_ready + 8 * s, ph, s_abort)) return false;
+        tc_fence_after_sync();
+        const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
+        const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / 32; ++k)
+            mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (i != first) || k != 0);
+        tc_commit(bar_empty + 8 * s);
+        s += step;
+        if (s >= STAGES) {
+            s -= STAGES;
+            ph ^= 1;
+        }
+    }
+    return true;
+}
 
 template <int BN, int STAGES, bool W4>
 __global__ void __launch_bounds__(TmaSmem<BN, STAGES, W4>::THREADS, 1)
 tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                const TmaParams p)
+                const __grid_constant__ CUtensorMap tmap_y, const TmaParams p)
 {
     using L = TmaSmem<BN, STAGES, W4>;
     extern __shared__ uint8_t smem_raw[];
@@ -148,6 +313,9 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * rank) / splits);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (rank + 1)) / splits);
     const int nkb = kb_end - kb_begin;
+    // an unsplit tile needs no pass through shared memory: its epilogue warps store it themselves
+    const bool direct = splits == 1 && p.Y != nullptr && p.acc_out == nullptr;
+    const bool dual = L::DUAL && nkb >= 2;  // two MMA issuers, two accumulators
 
     const uint32_t bar_full = smem_u32(bars);                 // TMA bytes of the stage have landed
     const uint32_t bar_unpacked = smem_u32(bars + STAGES);    // W4: nibbles expanded into the B tile
@@ -157,30 +325,32 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
             mbar_init(bar_unpacked + 8 * s, 8);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        mbar_init(bar_accum, 1);
+        mbar_init(bar_accum, dual ? 2 : 1);
         *s_abort = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmap_a);
         tma_prefetch_desc(&tmap_w);
+        if (p.tma_store) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(s_tmem), BN);
+        tmem_alloc(smem_u32(s_tmem), L::TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    pdl_wait();  // everything above is independent of earlier kernels; global memory is not
+    // everything above is independent of earlier kernels; global memory is not, except the packed
+    // weights: no kernel that launches dependents early writes them, so their producer runs ahead
+    if (warp != L::B_WARP) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ activation-tile producer
         if (lane == 0) {
-            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
             int img_b = 0, ho0 = 0, wo0 = 0;
             if (p.conv) {
                 img_b = m0 / p.HoWo;
@@ -189,7 +359,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 wo0 = rem - ho0 * p.Wo;
             }
             // single-thread loop: all indices are carried along instead of being recomputed
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            const uint32_t a0 = smem_u32(sA);
             uint32_t s = 0, ph = 1;
             int tap = 0, cb = 0, kh = 0, kw = 0;
             if (p.conv) {
@@ -198,19 +368,15 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 kh = tap / 3;
                 kw = tap - 3 * kh;
             }
-            int kx_tap = tap * p.Cin;           // conv: first reduction index of the tap
-            int xa = kb_begin * BK, xb = kb_begin * ROW_BYTES;
+            int xa = kb_begin * BK;
             for (int i = 0; i < nkb; ++i) {
-                if (!mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;
+                if (i >= STAGES && !mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;  // slots start out free
                 const uint32_t full = bar_full + 8 * s;
-                mbar_arrive_expect_tx(full, L::A_BYTES + BN * ROW_BYTES);
+                mbar_arrive_expect_tx(full, L::A_BYTES);
                 if (p.conv) {
                     tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
-                    const int kx = kx_tap + cb * BK;
-                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
                     if (++cb == p.cblocks) {
                         cb = 0;
-                        kx_tap += p.Cin;
                         if (++kw == 3) {
                             kw = 0;
                             ++kh;
@@ -218,8 +384,43 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                     }
                 } else {
                     tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
-                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
                     xa += BK;
+                }
+                if (++s == STAGES) {
+                    s = 0;
+                    ph ^= 1;
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == L::B_WARP) {
+        // ------------------------------------------------------------ weight-tile producer
+        // a thread of its own: one TMA issue costs a few hundred cycles of a single thread, and
+        // with both operands on one thread the issue rate, not the MMA, sets the k-block cadence
+        if (lane == 0) {
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            const uint32_t b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            uint32_t s = 0, ph = 1;
+            int tap = 0, cb = 0;
+            if (p.conv) {
+                tap = kb_begin / p.cblocks;
+                cb = kb_begin - tap * p.cblocks;
+            }
+            int kx_tap = tap * p.Cin;  // conv: first reduction index of the tap
+            int xb = kb_begin * ROW_BYTES;
+            for (int i = 0; i < nkb; ++i) {
+                if (i >= STAGES && !mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;  // slots start out free
+                const uint32_t full = bar_full + 8 * s;
+                mbar_arrive_expect_tx(full, BN * ROW_BYTES);
+                if (p.conv) {
+                    const int kx = kx_tap + cb * BK;
+                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
+                    if (++cb == p.cblocks) {
+                        cb = 0;
+                        kx_tap += p.Cin;
+                    }
+                } else {
+                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
                     xb += ROW_BYTES;
                 }
                 if (++s == STAGES) {
@@ -232,41 +433,24 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
-            bool ok = true;
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
-            uint32_t s = 0, ph = 0;
-            for (int i = 0; i < nkb; ++i) {
-                ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
-                if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, ph, s_abort);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
-                const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
-#pragma unroll
-                for (int k = 0; k < BK / 32; ++k)
-                    mma_i8_ss(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i | k) != 0);
-                tc_commit(bar_empty + 8 * s);
-                if (++s == STAGES) {
-                    s = 0;
-                    ph ^= 1;
-                }
-            }
+            // W4: the expansion warps arrive only after they have seen the TMA bytes land, so their
+            // barrier alone orders both operands
+            const bool ok = issue_k_blocks<BN, STAGES, L>(0, dual ? 2 : 1, nkb, tmem_base, W4 ? bar_unpacked : bar_full,
+                                                          bar_empty, smem_u32(sA), smem_u32(sB), s_abort);
             if (ok) tc_commit(bar_accum);
         }
         __syncwarp();
-    } else if (warp < 6) {
-        // ------------------------------------------------------------ epilogue warps
-        // while the main loop runs: per-column dequantization factors of this tile, and the
-        // stored BOS rows
-        {
+    } else if (warp < L::B_WARP) {
+        if (warp < 6) {
+            // -------------------------------------------------------- epilogue warps
+            // while the main loop runs: per-column dequantization factors of this tile, and the
+            // stored BOS rows
             const float sx = __ldg(p.act_scale);
             for (int j = tid - 64; j < BN; j += 128) {
                 const int n = n0 + j;
                 float comb = 0.f, b = 0.f;
                 if (n < p.N && p.w_scale) {
                     comb = sx * __ldg(p.w_scale + n);
-                    if (W4) comb *= 0.0625f;
                     if (p.bias) b = __half2float(p.bias[n]);
                 }
                 s_comb[j] = comb;
@@ -280,66 +464,95 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                         p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
                 }
             }
-        }
-        // ------------------------------------------------------------ epilogue, part 1
-        // accumulators: tensor memory -> registers -> shared memory (the pipeline buffers are
-        // free once the last MMA has completed), 16-byte chunks XOR-swizzled by row
-        bool ok = mbar_wait(bar_accum, 0, s_abort);
-        tc_fence_after_sync();
-        const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
-        const int lg = warp & 3;
-        const int row = lg * 32 + lane;
-        if (go) {
-            uint8_t* prow = smem + row * (BN * 4);
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0, r);
-                tmem_ld_wait();
+        } else if (W4) {
+            // -------------------------------------------------------- int4 -> int8 (x16) expansion
+            const int ut = tid - 192;
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % STAGES;
+                const uint32_t round = static_cast<uint32_t>(i / STAGES);
+                if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
+                const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
+                uint8_t* b_stage = sB + s * L::B_BYTES;
+                // in place: every thread first reads its packed runs, then (after all have) writes
+                uint4 wv[(BN * 4) / 256];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int chunk = (c0 >> 2) + j;
-                    *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
-                        make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                for (int t = 0; t < (BN * 4) / 256; ++t) {
+                    const int task = ut + t * 256;
+                    wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
+                }
+                asm volatile("bar.sync 2, 256;" ::: "memory");
+#pragma unroll
+                for (int t = 0; t < (BN * 4) / 256; ++t) {
+                    const int task = ut + t * 256;
+                    const int r = task >> 2, j = task & 3;
+                    const uint4 w = wv[t];
+                    uint4 c0, c1;
+                    c0.x = (w.x << 4) & 0xF0F0F0F0u;
+                    c0.y = w.x & 0xF0F0F0F0u;
+                    c0.z = (w.y << 4) & 0xF0F0F0F0u;
+                    c0.w = w.y & 0xF0F0F0F0u;
+                    c1.x = (w.z << 4) & 0xF0F0F0F0u;
+                    c1.y = w.z & 0xF0F0F0F0u;
+                    c1.z = (w.w << 4) & 0xF0F0F0F0u;
+                    c1.w = w.w & 0xF0F0F0F0u;
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
+            }
+        }
+        if (warp < 10) {
+            // -------------------------------------------------------- epilogue, part 1
+            // warps 2-5 take the first half of the tile's columns, warps 6-9 the second half; both
+            // read the 32 tensor-memory lanes their rank within a warpgroup gives access to
+            asm volatile("bar.sync 1, 256;" ::: "memory");  // the factor tables above are complete
+            bool ok = mbar_wait(bar_accum, 0, s_abort);
+            tc_fence_after_sync();
+            const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
+            const int lg = warp & 3;
+            const int row = lg * 32 + lane;
+            const int cbeg = warp < 6 ? 0 : BN / 2;
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + cbeg;
+            if (go && direct) {
+                // unsplit tile: dequantize and store straight from tensor memory; the staging tiles
+                // sit in the pipeline buffers, which are free once the last MMA has completed
+                uint8_t* stage = smem + (warp - 2) * EPI_WARP_BYTES;
+                store_rows_dispatch<W4>(acc, dual ? BN : 0, BN / 2, s_comb + cbeg, s_bias + cbeg, stage, p, &tmap_y,
+                                        m0 + lg * 32, n0 + cbeg, lane);
+                if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
+            } else if (go) {
+                // split tile (or accumulator dump): tensor memory -> registers -> shared memory,
+                // 16-byte chunks XOR-swizzled by row
+                uint8_t* prow = smem + row * (BN * 4);
+                for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc + c0, r);
+                    if (dual) {
+                        uint32_t r2[32];
+                        tmem_ld_32x32(acc + BN + c0, r2);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] += r2[j];
+                    } else {
+                        tmem_ld_wait();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int chunk = ((cbeg + c0) >> 2) + j;
+                        *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
+                            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    }
                 }
             }
         }
-    } else if (W4) {
-        // ------------------------------------------------------------ int4 -> int8 (x16) expansion
-        const int ut = tid - 192;
-        for (int i = 0; i < nkb; ++i) {
-            const int s = i % STAGES;
-            const uint32_t round = static_cast<uint32_t>(i / STAGES);
-            if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
-            const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
-            uint8_t* b_stage = sB + s * L::B_BYTES;
-            // in place: every thread first reads its packed runs, then (after all have) writes
-            uint4 wv[(BN * 4) / 256];
-#pragma unroll
-            for (int t = 0; t < (BN * 4) / 256; ++t) {
-                const int task = ut + t * 256;
-                wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
-            }
-            asm volatile("bar.sync 2, 256;" ::: "memory");
-#pragma unroll
-            for (int t = 0; t < (BN * 4) / 256; ++t) {
-                const int task = ut + t * 256;
-                const int r = task >> 2, j = task & 3;
-                const uint4 w = wv[t];
-                uint4 c0, c1;
-                c0.x = (w.x << 4) & 0xF0F0F0F0u;
-                c0.y = w.x & 0xF0F0F0F0u;
-                c0.z = (w.y << 4) & 0xF0F0F0F0u;
-                c0.w = w.y & 0xF0F0F0F0u;
-                c1.x = (w.z << 4) & 0xF0F0F0F0u;
-                c1.y = w.z & 0xF0F0F0F0u;
-                c1.z = (w.w << 4) & 0xF0F0F0F0u;
-                c1.w = w.w & 0xF0F0F0F0u;
-                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
-                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
+    } else if (L::DUAL && warp == L::MMA2_WARP) {
+        // ------------------------------------------------------------ second MMA issuer: odd k-blocks
+        if (lane == 0 && dual) {
+            const bool ok = issue_k_blocks<BN, STAGES, L>(1, 2, nkb, tmem_base + BN, W4 ? bar_unpacked : bar_full,
+                                                          bar_empty, smem_u32(sA), smem_u32(sB), s_abort);
+            if (ok) tc_commit(bar_accum);
         }
     }
 
@@ -349,19 +562,19 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // order-free), dequantizes and stores; threads run along a row so stores coalesce.
     __syncthreads();
     if (splits > 1) cluster_sync_all();
-    if (!*s_abort) {
+    if (!*s_abort && !direct) {
         // a thread keeps one group of four columns (its factors stay in registers) and walks
         // down the rows; consecutive threads take consecutive column groups
         const int rows_per = BM / splits;
         constexpr int CHUNKS = BN / 4;
-        constexpr int RSTEP = L::THREADS / CHUNKS;
-        static_assert(L::THREADS % CHUNKS == 0, "threads must tile the column groups");
+        constexpr int RSTEP = L::WORK_THREADS / CHUNKS;
+        static_assert(L::WORK_THREADS % CHUNKS == 0, "threads must tile the column groups");
         const int chunk = tid % CHUNKS;
         const int n = n0 + chunk * 4;
         const bool vec = ((p.ldy & 3) == 0) && n + 4 <= p.N;
         const float4 cb = *reinterpret_cast<const float4*>(s_comb + chunk * 4);
         const float4 bb = *reinterpret_cast<const float4*>(s_bias + chunk * 4);
-        if (n < p.N) {
+        if (n < p.N && tid < L::WORK_THREADS) {
 #pragma unroll 2
             for (int rl = tid / CHUNKS; rl < rows_per; rl += RSTEP) {
                 const int row = rank * rows_per + rl;
@@ -399,10 +612,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                                   (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
                     }
                     __half2 h[2];
-                    h[0] = __floats2half2_rn(fmaf(static_cast<float>(acc.x), cb.x, bb.x),
-                                             fmaf(static_cast<float>(acc.y), cb.y, bb.y));
-                    h[1] = __floats2half2_rn(fmaf(static_cast<float>(acc.z), cb.z, bb.z),
-                                             fmaf(static_cast<float>(acc.w), cb.w, bb.w));
+                    h[0] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.x), cb.x, bb.x),
+                                             fmaf(acc_to_float<W4, false>(acc.y), cb.y, bb.y));
+                    h[1] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.z), cb.z, bb.z),
+                                             fmaf(acc_to_float<W4, false>(acc.w), cb.w, bb.w));
                     __half* dst = p.Y + out_row * p.ldy + n;
                     if (vec) {
                         *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
@@ -422,7 +635,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     tc_fence_before_sync();
     __syncthreads();
     if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's shared memory
-    if (warp == 1) tmem_dealloc(tmem_base, BN);
+    if (warp == 1) tmem_dealloc(tmem_base, L::TMEM_COLS);
 }
 
 // Persistent form for problems with at least as many output tiles as SMs: one CTA per SM
@@ -445,17 +658,18 @@ struct PersistSmem {
     static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] floats
     static constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
-    static constexpr int OFF_EPI = OFF_MISC + 64;  // per epilogue warp: 32 rows x 64 fp16, rows 144 bytes apart
-    static constexpr int EPI_ROW = 144;
-    static constexpr int EPI_WARP_BYTES = 32 * EPI_ROW;
+    static constexpr int OFF_EPI = (OFF_MISC + 64 + 1023) & ~1023;  // staging tiles of the four epilogue warps
     static constexpr int TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
-    static constexpr int THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
+    static constexpr int WORK_THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
+    static constexpr int B_WARP = WORK_THREADS / 32;      // last warp: TMA producer of the weight tiles
+    static constexpr int THREADS = WORK_THREADS + 32;
 };
 
 template <int BN, int STAGES, bool W4>
 __global__ void __launch_bounds__(PersistSmem<BN, STAGES, W4>::THREADS, 1)
 tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                           const TmaParams p, int n_tiles, int total_tiles)
+                           const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, int n_tiles,
+                           int total_tiles)
 {
     using L = PersistSmem<BN, STAGES, W4>;
     extern __shared__ uint8_t smem_raw[];
@@ -483,7 +697,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
             mbar_init(bar_unpacked + 8 * s, 8);
             mbar_init(bar_empty + 8 * s, 1);
         }
@@ -495,6 +709,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         fence_barrier_init();
         tma_prefetch_desc(&tmap_a);
         tma_prefetch_desc(&tmap_w);
+        if (p.tma_store) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(s_tmem), 2 * BN);
@@ -503,20 +718,19 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    pdl_wait();
+    if (warp != L::B_WARP) pdl_wait();  // the weight producer runs ahead of earlier kernels
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ activation-tile producer
         if (lane == 0) {
-            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
             // single-thread loop: all indices are carried along instead of being recomputed
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            const uint32_t a0 = smem_u32(sA);
             uint32_t s = 0, ph = 1;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = blockIdx.x + t * gridDim.x;
-                const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+                const int m0 = (tile / n_tiles) * BM;
                 int img_b = 0, ho0 = 0, wo0 = 0;
                 if (p.conv) {
                     img_b = m0 / p.HoWo;
@@ -524,19 +738,16 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     ho0 = rem / p.Wo;
                     wo0 = rem - ho0 * p.Wo;
                 }
-                int cb = 0, kh = 0, kw = 0, kx_tap = 0, xa = 0, xb = 0;
+                int cb = 0, kh = 0, kw = 0, xa = 0;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);
+                    if (t > 0 || kb >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);  // slots start out free
                     if (!ok) break;
                     const uint32_t full = bar_full + 8 * s;
-                    mbar_arrive_expect_tx(full, L::A_BYTES + BN * ROW_BYTES);
+                    mbar_arrive_expect_tx(full, L::A_BYTES);
                     if (p.conv) {
                         tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
-                        const int kx = kx_tap + cb * BK;
-                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
                         if (++cb == p.cblocks) {
                             cb = 0;
-                            kx_tap += p.Cin;
                             if (++kw == 3) {
                                 kw = 0;
                                 ++kh;
@@ -544,8 +755,41 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                         }
                     } else {
                         tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
-                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
                         xa += BK;
+                    }
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == L::B_WARP) {
+        // ------------------------------------------------------------ weight-tile producer
+        if (lane == 0) {
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            const uint32_t b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
+            uint32_t s = 0, ph = 1;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = blockIdx.x + t * gridDim.x;
+                const int n0 = (tile % n_tiles) * BN;
+                int cb = 0, kx_tap = 0, xb = 0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (t > 0 || kb >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);  // slots start out free
+                    if (!ok) break;
+                    const uint32_t full = bar_full + 8 * s;
+                    mbar_arrive_expect_tx(full, BN * ROW_BYTES);
+                    if (p.conv) {
+                        const int kx = kx_tap + cb * BK;
+                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
+                        if (++cb == p.cblocks) {
+                            cb = 0;
+                            kx_tap += p.Cin;
+                        }
+                    } else {
+                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
                         xb += ROW_BYTES;
                     }
                     if (++s == STAGES) {
@@ -561,6 +805,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
             const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            const uint32_t bar_ready = W4 ? bar_unpacked : bar_full;  // W4: implies the TMA bytes landed
             uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
@@ -571,8 +816,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 tc_fence_after_sync();
                 const uint32_t acc = tmem_base + buf * BN;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
-                    if (ok && W4) ok = mbar_wait(bar_unpacked + 8 * s, ph, s_abort);
+                    ok = mbar_wait(bar_ready + 8 * s, ph, s_abort);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
@@ -595,7 +839,6 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         const int lg = warp & 3;
         const int et = tid - 64;
         const float sx = __ldg(p.act_scale);
-        const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
         bool ok = true;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
@@ -610,7 +853,6 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 float c = 0.f, b = 0.f;
                 if (n < p.N && p.w_scale) {
                     c = sx * __ldg(p.w_scale + n);
-                    if (W4) c *= 0.0625f;
                     if (p.bias) b = __half2float(p.bias[n]);
                 }
                 comb[j] = c;
@@ -631,8 +873,6 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 ok = false;
                 continue;
             }
-            const int m = m0 + lg * 32 + lane;
-            const bool m_ok = m < p.M;
             const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
             if (p.acc_out) {
                 // parity hook: raw accumulators, one row per thread
@@ -641,7 +881,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     uint32_t r[32];
                     tmem_ld_32x32(acc + c0, r);
                     tmem_ld_wait();
-                    if (!m_ok) continue;
+                    const int m = m0 + lg * 32 + lane;
+                    if (m >= p.M) continue;
                     const int n = n0 + c0;
                     int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
 #pragma unroll
@@ -650,69 +891,16 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 }
             }
             if (p.Y) {
-                // 64 columns at a time: dequantize in registers (one row per thread), pass through a
-                // small shared-memory tile, and store with eight lanes along each row so that
-                // every store instruction writes whole 128-byte lines
-                uint8_t* stage = smem + L::OFF_EPI + (warp - 2) * L::EPI_WARP_BYTES;
-                for (int c0 = 0; c0 < BN; c0 += 64) {
-                    if (n0 + c0 >= p.N) break;  // uniform across the warp
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t r[32];
-                        tmem_ld_32x32(acc + c0 + 32 * h, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            const int c = c0 + 32 * h + j;
-                            const float4 ca = *reinterpret_cast<const float4*>(comb + c);
-                            const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
-                            const float4 ba = *reinterpret_cast<const float4*>(bias + c);
-                            const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
-                            __half2 hv[4];
-                            hv[0] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j])), ca.x, ba.x),
-                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 1])), ca.y, ba.y));
-                            hv[1] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 2])), ca.z, ba.z),
-                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 3])), ca.w, ba.w));
-                            hv[2] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 4])), cb.x, bb.x),
-                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 5])), cb.y, bb.y));
-                            hv[3] = __floats2half2_rn(fmaf(static_cast<float>(static_cast<int32_t>(r[j + 6])), cb.z, bb.z),
-                                                      fmaf(static_cast<float>(static_cast<int32_t>(r[j + 7])), cb.w, bb.w));
-                            *reinterpret_cast<uint4*>(stage + lane * L::EPI_ROW + (32 * h + j) * 2) =
-                                *reinterpret_cast<const uint4*>(hv);
-                        }
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int it8 = 0; it8 < 8; ++it8) {
-                        const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
-                        const int mm = m0 + lg * 32 + rl;
-                        const int n = n0 + c0 + seg * 8;
-                        if (mm >= p.M || n >= p.N) continue;
-                        long long orow = mm;
-                        if (p.bos) {
-                            const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
-                            orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
-                                   (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
-                        }
-                        const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * L::EPI_ROW + seg * 16);
-                        __half* dst = p.Y + orow * p.ldy + n;
-                        if (vec && n + 8 <= p.N) {
-                            *reinterpret_cast<uint4*>(dst) = v;
-                        } else {
-                            const __half* hs = reinterpret_cast<const __half*>(&v);
-                            for (int q = 0; q < 8; ++q)
-                                if (n + q < p.N) dst[q] = hs[q];
-                        }
-                    }
-                    __syncwarp();
-                }
+                uint8_t* stage = smem + L::OFF_EPI + (warp - 2) * EPI_WARP_BYTES;
+                store_rows_dispatch<W4>(acc, 0, BN, comb, bias, stage, p, &tmap_y, m0 + lg * 32, n0, lane);
             }
             // the accumulator may be overwritten once every epilogue warp has read it
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
         }
-    } else if (W4) {
+        if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
+    } else if (W4 && warp < L::B_WARP) {
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion
         const int ut = tid - 192;
         const int total_kb = my_tiles * nkb;
@@ -763,7 +951,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
 }
 
 template <int BN, int STAGES, bool W4>
-int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp, int num_sms,
+int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int num_sms,
                       cudaStream_t stream)
 {
     using L = PersistSmem<BN, STAGES, W4>;
@@ -776,11 +964,12 @@ int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const TmaPar
     const int n_tiles = static_cast<int>(ceil_div(tp.N, BN));
     const int total = n_tiles * static_cast<int>(ceil_div(tp.M, BM));
     const dim3 grid(static_cast<unsigned>(total < num_sms ? total : num_sms));
-    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, tp, n_tiles, total);
+    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, ty, tp, n_tiles, total);
 }
 
 template <int BN, int STAGES, bool W4>
-int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp, int splits, cudaStream_t stream)
+int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int splits,
+               cudaStream_t stream)
 {
     using L = TmaSmem<BN, STAGES, W4>;
     auto kernel = tma_gemm_kernel<BN, STAGES, W4>;
@@ -791,7 +980,7 @@ int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const TmaParams& tp
     }
     const dim3 grid(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
                     static_cast<unsigned>(splits));
-    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, static_cast<unsigned>(splits), ta, tw, tp);
+    return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, static_cast<unsigned>(splits), ta, tw, ty, tp);
 }
 
 // Reduction splits (cluster size): enough CTAs to cover the SMs, at least 4 k-blocks each.
@@ -855,7 +1044,7 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     if (rc != MIXDQ_OK) return rc;
 
     // 2. tensor maps
-    CUtensorMap ta, tw;
+    CUtensorMap ta, tw, ty{};
     TmaParams tp{};
     tp.M = p.M;
     tp.N = p.N;
@@ -869,6 +1058,16 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     tp.ldy = p.ldy;
     tp.acc_out = p.acc_out;
     tp.status = p.status;
+    // bound of any accumulator: K products of at most 127 * 127 (W4, after the shift: 127 * 7)
+    tp.small_acc = static_cast<long long>(p.K) * 127 * (w4 ? 7 : 127) < (1ll << 22);
+    // output tiles leave through TMA stores when Y's rows are 16-byte aligned and consecutive output
+    // rows are consecutive rows of Y (not so for the cross-attention K/V layout, which skips row 0)
+    tp.tma_store = p.Y && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
+    if (tp.tma_store) {
+        const int rcy = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
+                                           static_cast<uint64_t>(p.ldy), 64, 32);
+        if (rcy != MIXDQ_OK) return rcy;
+    }
     if (conv) {
         int Wb, Hb, Bb;
         if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
@@ -908,10 +1107,10 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     }
     if (tiles >= num_sms && p.force_splits <= 0) {
         if (wide)
-            return w4 ? launch_persistent<256, 4, true>(ta, tw, tp, num_sms, stream)
-                      : launch_persistent<256, 4, false>(ta, tw, tp, num_sms, stream);
-        return w4 ? launch_persistent<128, 6, true>(ta, tw, tp, num_sms, stream)
-                  : launch_persistent<128, 6, false>(ta, tw, tp, num_sms, stream);
+            return w4 ? launch_persistent<256, 4, true>(ta, tw, ty, tp, num_sms, stream)
+                      : launch_persistent<256, 4, false>(ta, tw, ty, tp, num_sms, stream);
+        return w4 ? launch_persistent<128, 6, true>(ta, tw, ty, tp, num_sms, stream)
+                  : launch_persistent<128, 6, false>(ta, tw, ty, tp, num_sms, stream);
     }
     int splits = pick_splits(tiles, tp.k_blocks);
     if (p.force_splits > 0) {
@@ -919,10 +1118,10 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;
     }
     if (wide)
-        return w4 ? launch_tma<256, 4, true>(ta, tw, tp, splits, stream)
-                  : launch_tma<256, 4, false>(ta, tw, tp, splits, stream);
-    return w4 ? launch_tma<128, 6, true>(ta, tw, tp, splits, stream)
-              : launch_tma<128, 6, false>(ta, tw, tp, splits, stream);
+        return w4 ? launch_tma<256, 4, true>(ta, tw, ty, tp, splits, stream)
+                  : launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
+    return w4 ? launch_tma<128, 6, true>(ta, tw, ty, tp, splits, stream)
+              : launch_tma<128, 6, false>(ta, tw, ty, tp, splits, stream);
 }
 
 }  // namespace i8
