@@ -263,6 +263,69 @@ struct TmaSmem {
     static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
 };
 
+// int4 -> int8 (x16) expansion of the weight tiles, run by two groups of four warps: group g takes
+// the k-blocks g, g + 2, ... of the CTA's sequence, so two stages are in flight at a time (one stage's
+// chain -- wait, read, group barrier, write, fence, arrive -- is longer than the MMAs of a k-block).
+// The packed rows of a stage sit in the last half of its B slot and are expanded in place: every
+// thread first reads its packed runs, then (after the whole group has) writes.
+template <int BN, int STAGES, class L>
+__device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int total_kb, uint8_t* sB, uint32_t bar_full,
+                                               uint32_t bar_unpacked, volatile int* s_abort)
+{
+    constexpr int RUNS = (BN * 4) / 128;  // 16-byte packed runs per thread
+    uint32_t s = group, ph = 0;           // group < STAGES
+    for (int it = group; it < total_kb; it += 2) {
+        const uint32_t landed = mbar_wait(bar_full + 8 * s, ph, s_abort) ? 1u : 0u;
+        const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
+        uint8_t* b_stage = sB + s * L::B_BYTES;
+        uint4 wv[RUNS];
+#pragma unroll
+        for (int t = 0; t < RUNS; ++t) {
+            const int task = gt + t * 128;
+            wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
+        }
+        // group barrier between the reads and the in-place writes; it also carries the vote on whether
+        // every thread's wait succeeded, so that the group leaves the loop together after a timeout
+        uint32_t all_landed;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %1, 0;\n\t"
+            "barrier.cta.red.and.pred p, %2, 128, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}\n"
+            : "=r"(all_landed)
+            : "r"(landed), "r"(2 + group)
+            : "memory");
+        if (!all_landed) break;
+#pragma unroll
+        for (int t = 0; t < RUNS; ++t) {
+            const int task = gt + t * 128;
+            const int r = task >> 2, j = task & 3;
+            const uint4 w = wv[t];
+            uint4 c0, c1;
+            c0.x = (w.x << 4) & 0xF0F0F0F0u;
+            c0.y = w.x & 0xF0F0F0F0u;
+            c0.z = (w.y << 4) & 0xF0F0F0F0u;
+            c0.w = w.y & 0xF0F0F0F0u;
+            c1.x = (w.z << 4) & 0xF0F0F0F0u;
+            c1.y = w.z & 0xF0F0F0F0u;
+            c1.z = (w.w << 4) & 0xF0F0F0F0u;
+            c1.w = w.w & 0xF0F0F0F0u;
+            *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
+            *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
+        s += 2;
+        if (s >= STAGES) {
+            s -= STAGES;
+            ph ^= 1;
+        }
+    }
+}
+
 // The k-blocks first, first + step, ... of one output tile: wait for the stage, issue its four
 // MMAs into `acc`, hand the stage back.  Runs in a single thread.
 template <int BN, int STAGES, class L>
@@ -326,7 +389,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
-            mbar_init(bar_unpacked + 8 * s, 8);
+            mbar_init(bar_unpacked + 8 * s, 4);  // the four warps of an expansion group
             mbar_init(bar_empty + 8 * s, 1);
         }
         mbar_init(bar_accum, dual ? 2 : 1);
@@ -466,42 +529,8 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             }
         } else if (W4) {
             // -------------------------------------------------------- int4 -> int8 (x16) expansion
-            const int ut = tid - 192;
-            for (int i = 0; i < nkb; ++i) {
-                const int s = i % STAGES;
-                const uint32_t round = static_cast<uint32_t>(i / STAGES);
-                if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
-                const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
-                uint8_t* b_stage = sB + s * L::B_BYTES;
-                // in place: every thread first reads its packed runs, then (after all have) writes
-                uint4 wv[(BN * 4) / 256];
-#pragma unroll
-                for (int t = 0; t < (BN * 4) / 256; ++t) {
-                    const int task = ut + t * 256;
-                    wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
-                }
-                asm volatile("bar.sync 2, 256;" ::: "memory");
-#pragma unroll
-                for (int t = 0; t < (BN * 4) / 256; ++t) {
-                    const int task = ut + t * 256;
-                    const int r = task >> 2, j = task & 3;
-                    const uint4 w = wv[t];
-                    uint4 c0, c1;
-                    c0.x = (w.x << 4) & 0xF0F0F0F0u;
-                    c0.y = w.x & 0xF0F0F0F0u;
-                    c0.z = (w.y << 4) & 0xF0F0F0F0u;
-                    c0.w = w.y & 0xF0F0F0F0u;
-                    c1.x = (w.z << 4) & 0xF0F0F0F0u;
-                    c1.y = w.z & 0xF0F0F0F0u;
-                    c1.z = (w.w << 4) & 0xF0F0F0F0u;
-                    c1.w = w.w & 0xF0F0F0F0u;
-                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
-                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
-            }
+            const int group = (warp - 6) >> 2;  // warps 6-9 and 10-13
+            expand_nibbles<BN, STAGES, L>(group, tid - 192 - group * 128, lane, nkb, sB, bar_full, bar_unpacked, s_abort);
         }
         if (warp < 10) {
             // -------------------------------------------------------- epilogue, part 1
@@ -698,7 +727,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
-            mbar_init(bar_unpacked + 8 * s, 8);
+            mbar_init(bar_unpacked + 8 * s, 4);  // the four warps of an expansion group
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -902,43 +931,9 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
     } else if (W4 && warp < L::B_WARP) {
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion
-        const int ut = tid - 192;
-        const int total_kb = my_tiles * nkb;
-        for (int it = 0; it < total_kb; ++it) {
-            const int s = it % STAGES;
-            const uint32_t round = static_cast<uint32_t>(it / STAGES);
-            if (!mbar_wait(bar_full + 8 * s, round & 1, s_abort)) break;
-            const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
-            uint8_t* b_stage = sB + s * L::B_BYTES;
-            // in place: every thread first reads its packed runs, then (after all have) writes
-            uint4 wv[(BN * 4) / 256];
-#pragma unroll
-            for (int t = 0; t < (BN * 4) / 256; ++t) {
-                const int task = ut + t * 256;
-                wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
-            }
-            asm volatile("bar.sync 2, 256;" ::: "memory");
-#pragma unroll
-            for (int t = 0; t < (BN * 4) / 256; ++t) {
-                const int task = ut + t * 256;
-                const int r = task >> 2, j = task & 3;
-                const uint4 w = wv[t];
-                uint4 c0, c1;
-                c0.x = (w.x << 4) & 0xF0F0F0F0u;
-                c0.y = w.x & 0xF0F0F0F0u;
-                c0.z = (w.y << 4) & 0xF0F0F0F0u;
-                c0.w = w.y & 0xF0F0F0F0u;
-                c1.x = (w.z << 4) & 0xF0F0F0F0u;
-                c1.y = w.z & 0xF0F0F0F0u;
-                c1.z = (w.w << 4) & 0xF0F0F0F0u;
-                c1.w = w.w & 0xF0F0F0F0u;
-                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
-                *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
-        }
+        const int group = (warp - 6) >> 2;  // warps 6-9 and 10-13
+        expand_nibbles<BN, STAGES, L>(group, tid - 192 - group * 128, lane, my_tiles * nkb, sB, bar_full, bar_unpacked,
+                                      s_abort);
     }
 
     if (*s_abort) {
