@@ -327,13 +327,16 @@ __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int 
 }
 
 // The k-blocks first, first + step, ... of one output tile: wait for the stage, issue its four
-// MMAs into `acc`, hand the stage back.  Runs in a single thread.
+// MMAs into `acc`, hand the stage back.  Runs in a single thread (step <= STAGES).
 template <int BN, int STAGES, class L>
 __device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t bar_ready,
-                                               uint32_t bar_empty, uint32_t a0, uint32_t b0, volatile int* s_abort)
+                                               uint32_t bar_empty, uint32_t a0, uint32_t b0, volatile int* s_abort,
+                                               int seq0 = 0)
 {
     constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
-    uint32_t s = first, ph = 0;  // first < STAGES
+    // seq0: position of the tile's first k-block in the CTA's running sequence of pipeline stages
+    const uint32_t seq = static_cast<uint32_t>(seq0 + first);
+    uint32_t s = seq % STAGES, ph = (seq / STAGES) & 1;
     for (int i = first; i < nkb; i += step) {
         if (!mbar_wait(bar_ready + 8 * s, ph, s_abort)) return false;
         tc_fence_after_sync();
@@ -690,8 +693,11 @@ struct PersistSmem {
     static constexpr int OFF_EPI = (OFF_MISC + 64 + 1023) & ~1023;  // staging tiles of the four epilogue warps
     static constexpr int TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
     static constexpr int WORK_THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
-    static constexpr int B_WARP = WORK_THREADS / 32;      // last warp: TMA producer of the weight tiles
-    static constexpr int THREADS = WORK_THREADS + 32;
+    static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
+    static constexpr bool DUAL = BN == 128;               // second MMA issuer, as in the one-tile kernel
+    static constexpr int MMA2_WARP = B_WARP + 1;
+    static constexpr int THREADS = WORK_THREADS + 32 + (DUAL ? 32 : 0);
+    static constexpr int ACC_COLS = DUAL ? 2 * BN : BN;   // tensor-memory columns of one tile's accumulator(s)
 };
 
 template <int BN, int STAGES, bool W4>
@@ -714,6 +720,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nkb = p.k_blocks;
+    const bool dual = L::DUAL && nkb >= 2;  // two MMA issuers, two accumulators per tile
     const int my_tiles = (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                          static_cast<int>(gridDim.x);
 
@@ -731,7 +738,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_full + 8 * b, dual ? 2 : 1);
             mbar_init(bar_acc_empty + 8 * b, 4);
         }
         *s_abort = 0;
@@ -741,7 +748,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         if (p.tma_store) tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(s_tmem), 2 * BN);
+        tmem_alloc(smem_u32(s_tmem), 2 * L::ACC_COLS);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -829,13 +836,12 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+    } else if (warp == 1 || (L::DUAL && warp == L::MMA2_WARP)) {
+        // ------------------------------------------------------------ MMA issuers
+        // warp 1 (and, for narrow tiles, warp MMA2_WARP with the odd k-blocks and an accumulator of its own)
+        if (lane == 0 && (warp == 1 || dual)) {
+            const int which = warp == 1 ? 0 : 1;
             const uint32_t bar_ready = W4 ? bar_unpacked : bar_full;  // W4: implies the TMA bytes landed
-            uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t & 1;
@@ -843,22 +849,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 ok = mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, s_abort);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t acc = tmem_base + buf * BN;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    ok = mbar_wait(bar_ready + 8 * s, ph, s_abort);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
-                    const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / 32; ++k)
-                        mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                    tc_commit(bar_empty + 8 * s);
-                    if (++s == STAGES) {
-                        s = 0;
-                        ph ^= 1;
-                    }
-                }
+                ok = issue_k_blocks<BN, STAGES, L>(which, dual ? 2 : 1, nkb, tmem_base + buf * L::ACC_COLS + which * BN,
+                                                   bar_ready, bar_empty, smem_u32(sA), smem_u32(sB), s_abort, t * nkb);
                 if (ok) tc_commit(bar_acc_full + 8 * buf);
             }
         }
@@ -902,14 +894,22 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 ok = false;
                 continue;
             }
-            const uint32_t acc = tmem_base + buf * BN + (static_cast<uint32_t>(lg * 32) << 16);
+            const uint32_t acc = tmem_base + buf * L::ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
             if (p.acc_out) {
                 // parity hook: raw accumulators, one row per thread
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     if (n0 + c0 >= p.N) break;  // uniform across the warp
                     uint32_t r[32];
                     tmem_ld_32x32(acc + c0, r);
-                    tmem_ld_wait();
+                    if (dual) {
+                        uint32_t r2[32];
+                        tmem_ld_32x32(acc + BN + c0, r2);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] += r2[j];
+                    } else {
+                        tmem_ld_wait();
+                    }
                     const int m = m0 + lg * 32 + lane;
                     if (m >= p.M) continue;
                     const int n = n0 + c0;
@@ -921,7 +921,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             }
             if (p.Y) {
                 uint8_t* stage = smem + L::OFF_EPI + (warp - 2) * EPI_WARP_BYTES;
-                store_rows_dispatch<W4>(acc, 0, BN, comb, bias, stage, p, &tmap_y, m0 + lg * 32, n0, lane);
+                store_rows_dispatch<W4>(acc, dual ? BN : 0, BN, comb, bias, stage, p, &tmap_y, m0 + lg * 32, n0, lane);
             }
             // the accumulator may be overwritten once every epilogue warp has read it
             tc_fence_before_sync();
@@ -942,7 +942,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * L::ACC_COLS);
 }
 
 template <int BN, int STAGES, bool W4>
