@@ -61,6 +61,12 @@ int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4]
 int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
                        const uint32_t box[4]);
 
+// Once per kernel: ask for the largest shared-memory carve-out.  An SM changes its L1 / shared
+// split only when idle, so kernels with different preferences cannot share an SM and the change
+// itself costs time at every kernel boundary; with one preference everywhere, a small kernel's
+// tail and the next GEMM's set-up overlap.  Returns MIXDQ_OK or MIXDQ_ERR_CUDA.
+int prefer_max_shared_carveout(const void* kernel);
+
 #ifdef __CUDACC__
 
 // Launch with programmatic dependent launch enabled (and an optional cluster along z): the
@@ -85,6 +91,7 @@ inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     attr[1].val.clusterDim.z = cluster_z;
     cfg.attrs = attr;
     cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    if (prefer_max_shared_carveout(reinterpret_cast<const void*>(kernel)) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     g_layer_kernel_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
     if (err != cudaSuccess) {

@@ -356,7 +356,7 @@ __device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uin
 }
 
 template <int BN, int STAGES, bool W4>
-__global__ void __launch_bounds__(TmaSmem<BN, STAGES, W4>::THREADS, 1)
+__global__ void __maxnreg__(96)
 tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                 const __grid_constant__ CUtensorMap tmap_y, const TmaParams p)
 {

@@ -2,6 +2,7 @@
 // runtime so that the library has no link-time dependency on libcuda and still loads on
 // a machine without a GPU driver.
 #include <mutex>
+#include <unordered_set>
 
 #include "common.cuh"
 
@@ -101,6 +102,21 @@ static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const voi
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;
+}
+
+int prefer_max_shared_carveout(const void* kernel)
+{
+    static std::mutex mu;
+    static std::unordered_set<const void*> done;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done.count(kernel)) return MIXDQ_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return MIXDQ_ERR_CUDA;
+    }
+    done.insert(kernel);
+    return MIXDQ_OK;
 }
 
 }  // namespace mixdq
