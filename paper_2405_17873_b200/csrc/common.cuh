@@ -50,9 +50,10 @@ inline int check_launch() { return cudaGetLastError() == cudaSuccess ? MIXDQ_OK 
 // 2-D byte tensor map (rows x row_bytes, pitch in bytes) for TMA tile loads.
 int encode_tmap_2d_u8(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows,
                       uint64_t pitch_bytes, uint32_t box_bytes, uint32_t box_rows, bool swizzle128);
-// 2-D fp16 tensor map (rows x cols elements, pitch in elements), 128-byte swizzle.
+// 2-D fp16 tensor map (rows x cols elements, pitch in elements), 128-byte swizzle (64-byte for
+// boxes of 32 columns when swizzle64 is set).
 int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows,
-                       uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows);
+                       uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows, bool swizzle64 = false);
 
 // 4-D byte tensor map with the 128-byte swizzle (NHWC int8 image: dims {C, W, H, B}).
 int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],

@@ -233,6 +233,115 @@ __device__ __forceinline__ void store_rows_dispatch(uint32_t acc, uint32_t acc2_
     }
 }
 
+// The same in passes of 32 columns, for the persistent kernel, whose eight epilogue warps have to fit
+// their staging tiles beside a full pipeline: 32 rows x 32 fp16, as dense 64-byte rows with the
+// 64-byte swizzle when a TMA store (box 32 x 32) takes the tile, else rows 80 bytes apart.
+constexpr int EPI32_ROW = 80;
+constexpr int EPI32_TILE = 32 * EPI32_ROW;  // 2560: a multiple of 512, the period of the 64-byte swizzle
+
+template <bool W4, bool SMALL, bool TMA>
+__device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                       const float* bias, uint8_t* stage, const TmaParams& p,
+                                                       const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+{
+    const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
+    if (TMA && m_first >= p.M) return;  // uniform across the warp
+    for (int c0 = 0; c0 < ncols; c0 += 32) {
+        if (n0 + c0 >= p.N) break;  // uniform across the warp
+        uint32_t r[32];
+        tmem_ld_32x32(acc + c0, r);
+        if (acc2_off) {
+            uint32_t r2[32];
+            tmem_ld_32x32(acc + acc2_off + c0, r2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] += r2[j];
+        } else {
+            tmem_ld_wait();
+        }
+        uint4 out[4];  // this lane's row of the pass as fp16
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+            const int c = c0 + j;
+            const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+            const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+            const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+            const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+            __half2 hv[4];
+            hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j]), ca.x, ba.x),
+                                      fmaf(acc_to_float<W4, SMALL>(r[j + 1]), ca.y, ba.y));
+            hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 2]), ca.z, ba.z),
+                                      fmaf(acc_to_float<W4, SMALL>(r[j + 3]), ca.w, ba.w));
+            hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 4]), cb.x, bb.x),
+                                      fmaf(acc_to_float<W4, SMALL>(r[j + 5]), cb.y, bb.y));
+            hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 6]), cb.z, bb.z),
+                                      fmaf(acc_to_float<W4, SMALL>(r[j + 7]), cb.w, bb.w));
+            out[j >> 3] = *reinterpret_cast<const uint4*>(hv);
+        }
+        if (TMA) {
+            // the previous bulk store must have read the staging tile; the conversion above hid that wait
+            if (lane == 0) tma_store_wait_read();
+            __syncwarp();
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint8_t* dst = TMA ? stage + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4) : stage + lane * EPI32_ROW + q * 16;
+            *reinterpret_cast<uint4*>(dst) = out[q];
+        }
+        if (TMA) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(tmap_y, smem_u32(stage), n0 + c0, m_first);
+                tma_store_commit();
+            }
+            continue;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int rl = it * 8 + (lane >> 2), seg = lane & 3;
+            const int mm = m_first + rl;
+            const int n = n0 + c0 + seg * 8;
+            if (mm >= p.M || n >= p.N) continue;
+            long long orow = mm;
+            if (p.bos) {
+                const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
+                orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
+                       (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
+            }
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI32_ROW + seg * 16);
+            __half* dst = p.Y + orow * p.ldy + n;
+            if (vec && n + 8 <= p.N) {
+                *reinterpret_cast<uint4*>(dst) = v;
+            } else {
+                const __half* hs = reinterpret_cast<const __half*>(&v);
+                for (int q = 0; q < 8; ++q)
+                    if (n + q < p.N) dst[q] = hs[q];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+template <bool W4>
+__device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                      const float* bias, uint8_t* stage, const TmaParams& p,
+                                                      const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+{
+    if (p.tma_store) {
+        if (p.small_acc)
+            store_rows32_from_tmem<W4, true, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+        else
+            store_rows32_from_tmem<W4, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+    } else {
+        if (p.small_acc)
+            store_rows32_from_tmem<W4, true, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+        else
+            store_rows32_from_tmem<W4, false, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+    }
+}
+
 template <int BN, int STAGES, bool W4>
 struct TmaSmem {
     static constexpr int A_BYTES = BM * BK;
@@ -690,9 +799,13 @@ struct PersistSmem {
     static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] floats
     static constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
-    static constexpr int OFF_EPI = (OFF_MISC + 64 + 1023) & ~1023;  // staging tiles of the four epilogue warps
-    static constexpr int TOTAL = OFF_EPI + 4 * EPI_WARP_BYTES + 1024;
-    static constexpr int WORK_THREADS = W4 ? 448 : 192;  // W4: eight nibble-expansion warps
+    static constexpr int OFF_EPI = (OFF_MISC + 64 + 1023) & ~1023;  // staging tiles of the eight epilogue warps
+    static constexpr int TOTAL = OFF_EPI + 8 * EPI32_TILE + 1024;
+    static_assert(TOTAL <= 232448, "shared memory of one CTA");
+    // warps: 0 activation producer, 1 MMA issuer, 2-5 epilogue (first half of the tile's columns),
+    // W4: 6-13 nibble expansion, then four epilogue helpers (second half of the columns)
+    static constexpr int HELPER0 = W4 ? 14 : 6;
+    static constexpr int WORK_THREADS = (HELPER0 + 4) * 32;
     static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
     static constexpr bool DUAL = BN == 128;               // second MMA issuer, as in the one-tile kernel
     static constexpr int MMA2_WARP = B_WARP + 1;
@@ -739,7 +852,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, dual ? 2 : 1);
-            mbar_init(bar_acc_empty + 8 * b, 4);
+            mbar_init(bar_acc_empty + 8 * b, 8);  // epilogue warps and their helpers
         }
         *s_abort = 0;
         fence_barrier_init();
@@ -855,10 +968,11 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             }
         }
         __syncwarp();
-    } else if (warp < 6) {
-        // ------------------------------------------------------------ epilogue warps
+    } else if (warp < 6 || (warp >= L::HELPER0 && warp < L::HELPER0 + 4)) {
+        // ------------------------------------------------------------ epilogue warps and helpers
         const int lg = warp & 3;
-        const int et = tid - 64;
+        const int half = warp < 6 ? 0 : 1;
+        const int et = tid - 64;  // epilogue warps only: 0..127
         const float sx = __ldg(p.act_scale);
         bool ok = true;
         for (int t = 0; t < my_tiles; ++t) {
@@ -869,7 +983,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             float* comb = s_comb + buf * BN;
             float* bias = s_bias + buf * BN;
             // this tile's per-column factors (the buffer was last read two tiles ago)
-            for (int j = et; j < BN; j += 128) {
+            for (int j = et; half == 0 && j < BN; j += 128) {
                 const int n = n0 + j;
                 float c = 0.f, b = 0.f;
                 if (n < p.N && p.w_scale) {
@@ -879,23 +993,34 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 comb[j] = c;
                 bias[j] = b;
             }
-            if (p.bos && p.Y && m0 == 0) {
+            if (half == 0 && p.bos && p.Y && m0 == 0) {
                 for (int idx = et; idx < p.batch * BN; idx += 128) {
                     const int b = idx / BN, j = idx - b * BN;
                     if (n0 + j < p.N)
                         p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
                 }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
             if (ok) ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, s_abort);
             tc_fence_after_sync();
-            const bool go = __all_sync(0xffffffffu, ok && !*s_abort);
+            // the factor tables are complete; the same barrier carries the vote on whether every warp's
+            // wait succeeded, so that all eight take the same path from here
+            uint32_t go;
+            asm volatile(
+                "{\n\t"
+                ".reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "barrier.cta.red.and.pred p, 1, 256, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t"
+                "}\n"
+                : "=r"(go)
+                : "r"((ok && !*s_abort) ? 1u : 0u)
+                : "memory");
             if (!go) {
                 ok = false;
                 continue;
             }
             const uint32_t acc = tmem_base + buf * L::ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
-            if (p.acc_out) {
+            if (p.acc_out && half == 0) {
                 // parity hook: raw accumulators, one row per thread
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     if (n0 + c0 >= p.N) break;  // uniform across the warp
@@ -920,8 +1045,10 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 }
             }
             if (p.Y) {
-                uint8_t* stage = smem + L::OFF_EPI + (warp - 2) * EPI_WARP_BYTES;
-                store_rows_dispatch<W4>(acc, dual ? BN : 0, BN, comb, bias, stage, p, &tmap_y, m0 + lg * 32, n0, lane);
+                const int cbeg = half * (BN / 2);
+                uint8_t* stage = smem + L::OFF_EPI + (half * 4 + lg) * EPI32_TILE;
+                store_rows32_dispatch<W4>(acc + cbeg, dual ? BN : 0, BN / 2, comb + cbeg, bias + cbeg, stage, p, &tmap_y,
+                                          m0 + lg * 32, n0 + cbeg, lane);
             }
             // the accumulator may be overwritten once every epilogue warp has read it
             tc_fence_before_sync();
@@ -929,7 +1056,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
         }
         if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
-    } else if (W4 && warp < L::B_WARP) {
+    } else if (W4 && warp < L::HELPER0) {
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion
         const int group = (warp - 6) >> 2;  // warps 6-9 and 10-13
         expand_nibbles<BN, STAGES, L>(group, tid - 192 - group * 128, lane, my_tiles * nkb, sB, bar_full, bar_unpacked,
@@ -1058,11 +1185,6 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     // output tiles leave through TMA stores when Y's rows are 16-byte aligned and consecutive output
     // rows are consecutive rows of Y (not so for the cross-attention K/V layout, which skips row 0)
     tp.tma_store = p.Y && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
-    if (tp.tma_store) {
-        const int rcy = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
-                                           static_cast<uint64_t>(p.ldy), 64, 32);
-        if (rcy != MIXDQ_OK) return rcy;
-    }
     if (conv) {
         int Wb, Hb, Bb;
         if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
@@ -1100,7 +1222,15 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         MIXDQ_CUDA_TRY(cudaGetDevice(&dev));
         MIXDQ_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     }
-    if (tiles >= num_sms && p.force_splits <= 0) {
+    const bool persistent = tiles >= num_sms && p.force_splits <= 0;
+    if (tp.tma_store) {
+        // store box: 64 x 32 (128-byte swizzle) in the one-tile kernel, 32 x 32 (64-byte swizzle) in the
+        // persistent one, whose staging tiles are smaller
+        rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
+                                static_cast<uint64_t>(p.ldy), persistent ? 32 : 64, 32, persistent);
+        if (rc != MIXDQ_OK) return rc;
+    }
+    if (persistent) {
         if (wide)
             return w4 ? launch_persistent<256, 4, true>(ta, tw, ty, tp, num_sms, stream)
                       : launch_persistent<256, 4, false>(ta, tw, ty, tp, num_sms, stream);

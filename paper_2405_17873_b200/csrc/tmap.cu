@@ -51,7 +51,7 @@ int encode_tmap_2d_u8(CUtensorMap* map, const void* base, uint64_t row_bytes, ui
 }
 
 int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows,
-                       uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
+                       uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows, bool swizzle64)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return MIXDQ_ERR_CUDA;
@@ -61,7 +61,7 @@ int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;
 }
