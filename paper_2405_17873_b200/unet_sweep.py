@@ -148,3 +148,59 @@ class UNetSweep:
             return False
         unit = l.Cin if l.kind == "conv3x3" else l.K
         return unit % 16 == 0 and l.N >= 16
+
+
+def _main(argv=None) -> int:
+    """Run one layer of the sweep a few times (e.g. under a profiler):
+
+        python -m paper_2405_17873_b200.unet_sweep --layer attn_1280#0 --w-bits 4 --table w4a8 --batch 4
+
+    Prints the layer's shape, the average time of a CUDA-graph replay of `--reps` runs and the
+    device status word.
+    """
+    import argparse
+
+    ap = argparse.ArgumentParser(description=_main.__doc__)
+    ap.add_argument("--layer", required=True, help="layer name from synth.unet_layers(), e.g. ffn1_1280#0")
+    ap.add_argument("--w-bits", type=int, default=None, help="override the table's weight bit-width")
+    ap.add_argument("--table", default="w4a8", choices=["w4a8", "a16"])
+    ap.add_argument("--batch", type=int, default=4)
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--eager", action="store_true", help="plain launches only, no graph and no timing")
+    a = ap.parse_args(argv)
+
+    specs = synth.unet_layers()
+    (synth.assign_bits_w4a8 if a.table == "w4a8" else synth.assign_bits_weight_only)(specs)
+    pick = [l for l in specs if l.name == a.layer]
+    if not pick:
+        raise SystemExit(f"no layer named {a.layer!r}")
+    if a.w_bits is not None:
+        pick[0].w_bits = a.w_bits
+    sw = UNetSweep(a.batch, a.table, layers=pick)
+    pl = sw.layers[0]
+    for _ in range(a.reps):
+        sw.run_layer(pl)
+    torch.cuda.synchronize()
+    l = pl.spec
+    line = f"{l.name} {l.kind} M={l.M * a.batch} N={l.N} K={l.K} W{l.w_bits}A{l.a_bits}"
+    if not a.eager:
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                for _ in range(a.reps):
+                    sw.run_layer(pl)
+            g.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+        line += f" {e0.elapsed_time(e1) * 1e3 / a.reps:.1f} us/run"
+    print(line, "status", int(sw.status.item()))
+    return 0
+
+
+if __name__ == "__main__":
+    raise SystemExit(_main())
