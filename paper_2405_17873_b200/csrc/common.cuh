@@ -55,9 +55,10 @@ int encode_tmap_2d_u8(CUtensorMap* map, const void* base, uint64_t row_bytes, ui
 int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows,
                        uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows, bool swizzle64 = false);
 
-// 4-D byte tensor map with the 128-byte swizzle (NHWC int8 image: dims {C, W, H, B}).
+// 4-D byte tensor map with the 128-byte swizzle (NHWC int8 image: dims {C, W, H, B}).  box: elements
+// loaded per dimension; hw_step > 1 takes every hw_step-th pixel along W and H (strided convolution).
 int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                      const uint32_t box[4]);
+                      const uint32_t box[4], uint32_t hw_step = 1);
 // The same for an fp16 NHWC image (box extents in elements, strides in bytes).
 int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
                        const uint32_t box[4]);

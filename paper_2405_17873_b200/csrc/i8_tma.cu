@@ -93,6 +93,7 @@ struct TmaParams {
     int conv;     // 0: A is a [M, K] int8 matrix; 1: A is an int8 NHWC image gathered per filter tap
     int cblocks;  // conv: k-blocks per filter tap = ceil(Cin / 128)
     int Cin, HoWo, Wo;
+    int stride;   // conv: input pixels per output pixel along H and W (1 or 2)
     int bos;      // output row m maps to row (m / 76) * 77 + m % 76 + 1 of Y
     int batch;
     const float* act_scale;
@@ -549,7 +550,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 const uint32_t full = bar_full + 8 * s;
                 mbar_arrive_expect_tx(full, L::A_BYTES);
                 if (p.conv) {
-                    tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
+                    tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
                     if (++cb == p.cblocks) {
                         cb = 0;
                         if (++kw == 3) {
@@ -894,7 +895,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     const uint32_t full = bar_full + 8 * s;
                     mbar_arrive_expect_tx(full, L::A_BYTES);
                     if (p.conv) {
-                        tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, wo0 + kw - 1, ho0 + kh - 1, img_b, full);
+                        tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
                         if (++cb == p.cblocks) {
                             cb = 0;
                             if (++kw == 3) {
@@ -1142,7 +1143,9 @@ bool tma_path_ok(const Params& p, int amode, int w_bits)
 {
     if (amode == A_CONV3) {
         int a, b, c;
-        if (p.stride != 1 || p.Cin % 32 != 0) return false;
+        if (p.Cin % 32 != 0) return false;
+        // stride 2: through the tensor map's element strides, for even images (Ho = H / 2, Wo = W / 2)
+        if (p.stride != 1 && !(p.stride == 2 && p.H % 2 == 0 && p.W % 2 == 0)) return false;
         return conv_box(p.Ho, p.Wo, &a, &b, &c);
     }
     (void)w_bits;
@@ -1193,8 +1196,9 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         const uint64_t strides[3] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.Cin) * p.W,
                                      static_cast<uint64_t>(p.Cin) * p.W * p.H};
         const uint32_t box[4] = {BK, static_cast<uint32_t>(Wb), static_cast<uint32_t>(Hb), static_cast<uint32_t>(Bb)};
-        rc = encode_tmap_4d_u8(&ta, aq, dims, strides, box);
+        rc = encode_tmap_4d_u8(&ta, aq, dims, strides, box, static_cast<uint32_t>(p.stride));
         tp.conv = 1;
+        tp.stride = p.stride;
         tp.cblocks = static_cast<int>(ceil_div(p.Cin, BK));
         tp.Cin = p.Cin;
         tp.HoWo = p.Ho * p.Wo;

@@ -68,31 +68,34 @@ int encode_tmap_2d_f16(CUtensorMap* map, const void* base, uint64_t cols, uint64
 
 
 static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, const uint64_t dims[4],
-                          const uint64_t strides_bytes[3], const uint32_t box[4]);
+                          const uint64_t strides_bytes[3], const uint32_t box[4], uint32_t hw_step);
 
 int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                      const uint32_t box[4])
+                      const uint32_t box[4], uint32_t hw_step)
 {
-    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, dims, strides_bytes, box);
+    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, dims, strides_bytes, box, hw_step);
 }
 
 int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
                        const uint32_t box[4])
 {
-    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, base, dims, strides_bytes, box);
+    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, base, dims, strides_bytes, box, 1);
 }
 
 static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, const uint64_t dims[4],
-                          const uint64_t strides_bytes[3], const uint32_t box[4])
+                          const uint64_t strides_bytes[3], const uint32_t box[4], uint32_t hw_step)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return MIXDQ_ERR_CUDA;
     if (reinterpret_cast<uintptr_t>(base) & 15) return MIXDQ_ERR_ALIGNMENT;
     cuuint64_t d[4], st[3];
-    cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
+    // hw_step > 1 (strided convolution): the box takes every hw_step-th pixel along W and H; the
+    // encoder wants the traversed extent, of which it loads ceil(extent / step) elements
+    cuuint32_t b[4], estr[4] = {1, hw_step, hw_step, 1};
     for (int i = 0; i < 4; ++i) {
         d[i] = dims[i];
-        b[i] = box[i];
+        b[i] = (i == 1 || i == 2) ? box[i] * hw_step : box[i];
+        if (b[i] > 256) return MIXDQ_ERR_UNSUPPORTED;
     }
     for (int i = 0; i < 3; ++i) {
         if (strides_bytes[i] & 15) return MIXDQ_ERR_ALIGNMENT;
