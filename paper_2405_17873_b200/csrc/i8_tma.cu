@@ -343,74 +343,171 @@ __device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc
     }
 }
 
-template <int BN, int STAGES, bool W4>
-struct TmaSmem {
+// Rings of the pipeline and their barriers.  W8: activation and weight tiles move in lockstep, STAGES
+// deep.  W4 (128-wide tiles only): the packed int4 rows have a ring of their own, deep enough to hide
+// the TMA round trip, and are expanded into a short ring of int8 weight tiles; the chain TMA ->
+// expansion -> MMA is longer than the activations' TMA -> MMA, and it is depth, not bandwidth, that
+// bounds it (measured: 4 instead of 6 common stages cost 20 % on long reductions).
+template <int BN, int STAGES, bool W4, bool PERSIST>
+struct Rings {
+    static_assert(!W4 || BN == 128, "W4 runs on 128-wide tiles");
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
-    // packed int4 rows land in the last half of the B slot and are expanded in place
-    static constexpr int STG_BYTES = 0;
-    static constexpr int STG_OFFSET = BN * (BK / 2);
+    static constexpr int P_BYTES = BN * (BK / 2);
+    static constexpr int AS = W4 ? (PERSIST ? 4 : 5) : STAGES;  // activation tiles
+    static constexpr int ES = W4 ? 6 : STAGES;                  // int8 weight tiles (W4: expanded; four in the making)
+    static constexpr int PS = W4 ? (PERSIST ? 4 : 5) : 0;       // packed int4 weight tiles
     static constexpr int OFF_A = 0;
-    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
-    static constexpr int OFF_BARS = OFF_STG + STAGES * STG_BYTES;
-    static constexpr int NUM_BARS = 3 * STAGES + 1;
-    static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // read as float4
-    static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
-    static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
-    static constexpr int TOTAL = OFF_MISC + 64 + 1024;
-    // warps: 0 activation producer, 1 MMA issuer, 2-5 epilogue, 6-9 epilogue helpers (the other half
-    // of the tile's columns), W4: 6-13 nibble expansion during the main loop
-    static constexpr int WORK_THREADS = W4 ? 448 : 320;
-    static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
-    // One thread issues a 128-wide MMA about every 68 cycles, the tensor core retires it in 64: a
-    // lone issuer, which also waits and commits once per k-block, cannot keep the pipe busy.  Narrow
-    // tiles therefore get a second issuer: even k-blocks accumulate into one accumulator, odd ones
-    // into another, and the epilogue adds the two (integer adds: exact).
-    static constexpr bool DUAL = BN == 128;
-    static constexpr int MMA2_WARP = B_WARP + 1;
-    static constexpr int THREADS = WORK_THREADS + 32 + (DUAL ? 32 : 0);
-    static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
+    static constexpr int OFF_B = OFF_A + AS * A_BYTES;
+    static constexpr int OFF_P = OFF_B + ES * B_BYTES;
+    static constexpr int RINGS_END = OFF_P + PS * P_BYTES;
+    // barrier indices (8 bytes each)
+    static constexpr int FULL_A = 0;                  // TMA bytes of the activation tile have landed
+    static constexpr int EMPTY_A = FULL_A + AS;       // MMAs reading the tile have finished (W8: frees both tiles)
+    static constexpr int READY_B = EMPTY_A + AS;      // W8: TMA bytes landed; W4: expansion finished
+    static constexpr int EMPTY_B = READY_B + ES;      // W4: MMAs reading the int8 weight tile have finished
+    static constexpr int FULL_P = EMPTY_B + ES;       // W4: TMA bytes of the packed tile have landed
+    static constexpr int EMPTY_P = FULL_P + PS;       // W4: the packed tile has been read
+    static constexpr int RING_BARS = EMPTY_P + PS;
 };
 
-// int4 -> int8 (x16) expansion of the weight tiles, run by two groups of four warps: group g takes
-// the k-blocks g, g + 2, ... of the CTA's sequence, so two stages are in flight at a time (one stage's
-// chain -- wait, read, group barrier, write, fence, arrive -- is longer than the MMAs of a k-block).
-// The packed rows of a stage sit in the last half of its B slot and are expanded in place: every
-// thread first reads its packed runs, then (after the whole group has) writes.
-template <int BN, int STAGES, class L>
-__device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int total_kb, uint8_t* sB, uint32_t bar_full,
-                                               uint32_t bar_unpacked, volatile int* s_abort)
+template <class L>
+__device__ __forceinline__ void init_ring_barriers(uint32_t bar0, bool w4)
 {
-    constexpr int RUNS = (BN * 4) / 128;  // 16-byte packed runs per thread
-    uint32_t s = group, ph = 0;           // group < STAGES
-    for (int it = group; it < total_kb; it += 2) {
-        const uint32_t landed = mbar_wait(bar_full + 8 * s, ph, s_abort) ? 1u : 0u;
-        const uint8_t* stg = sB + s * L::B_BYTES + L::STG_OFFSET;
-        uint8_t* b_stage = sB + s * L::B_BYTES;
+    for (int s = 0; s < L::AS; ++s) {
+        mbar_init(bar0 + 8 * (L::FULL_A + s), 1);
+        mbar_init(bar0 + 8 * (L::EMPTY_A + s), 1);
+    }
+    for (int s = 0; s < L::ES; ++s) {
+        mbar_init(bar0 + 8 * (L::READY_B + s), w4 ? 2 : 1);  // W4: the two warps of an expansion group
+        mbar_init(bar0 + 8 * (L::EMPTY_B + s), 1);
+    }
+    for (int s = 0; s < L::PS; ++s) {
+        mbar_init(bar0 + 8 * (L::FULL_P + s), 1);
+        mbar_init(bar0 + 8 * (L::EMPTY_P + s), 2);
+    }
+}
+
+// Activation tiles of one output tile, k-blocks kb_begin .. kb_begin + nkb - 1; seq0 = position of the
+// first one in the CTA's running sequence of k-blocks (ring slot and phase follow from it).  Runs in a
+// single thread; all indices are carried along instead of being recomputed.
+template <class L>
+__device__ __forceinline__ bool produce_a_tile(const CUtensorMap* tmap_a, const TmaParams& p, uint32_t seq0, int kb_begin,
+                                               int nkb, int m0, uint32_t a0, uint32_t bar0, volatile int* s_abort)
+{
+    int img_b = 0, ho0 = 0, wo0 = 0, cb = 0, kh = 0, kw = 0;
+    if (p.conv) {
+        img_b = m0 / p.HoWo;
+        const int rem = m0 - img_b * p.HoWo;
+        ho0 = rem / p.Wo;
+        wo0 = rem - ho0 * p.Wo;
+        const int tap = kb_begin / p.cblocks;
+        cb = kb_begin - tap * p.cblocks;
+        kh = tap / 3;
+        kw = tap - 3 * kh;
+    }
+    int xa = kb_begin * BK;
+    uint32_t s = seq0 % L::AS, round = seq0 / L::AS;
+    for (int i = 0; i < nkb; ++i) {
+        // slots start out free
+        if (round > 0 && !mbar_wait(bar0 + 8 * (L::EMPTY_A + s), (round & 1) ^ 1, s_abort)) return false;
+        const uint32_t full = bar0 + 8 * (L::FULL_A + s);
+        mbar_arrive_expect_tx(full, L::A_BYTES);
+        if (p.conv) {
+            tma_load_4d(a0 + s * L::A_BYTES, tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
+            if (++cb == p.cblocks) {
+                cb = 0;
+                if (++kw == 3) {
+                    kw = 0;
+                    ++kh;
+                }
+            }
+        } else {
+            tma_load_2d(a0 + s * L::A_BYTES, tmap_a, xa, m0, full);
+            xa += BK;
+        }
+        if (++s == L::AS) {
+            s = 0;
+            ++round;
+        }
+    }
+    return true;
+}
+
+// Weight tiles of one output tile: int8 tiles into the weight ring (W8) or packed int4 tiles into the
+// packed ring (W4).  A thread of its own: one TMA issue costs a few hundred cycles of a single
+// thread, and with both operands on one thread the issue rate sets the k-block cadence.
+template <int BN, bool W4, class L>
+__device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const TmaParams& p, uint32_t seq0, int kb_begin,
+                                               int nkb, int n0, uint32_t ring0, uint32_t bar0, volatile int* s_abort)
+{
+    constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+    constexpr int R = W4 ? L::PS : L::ES;
+    constexpr int SLOT = W4 ? L::P_BYTES : L::B_BYTES;
+    constexpr int FULL = W4 ? L::FULL_P : L::READY_B;
+    constexpr int EMPTY = W4 ? L::EMPTY_P : L::EMPTY_A;  // W8: the MMA's one commit frees both tiles
+    int cb = 0, kx_tap = 0;
+    if (p.conv) {
+        const int tap = kb_begin / p.cblocks;
+        cb = kb_begin - tap * p.cblocks;
+        kx_tap = tap * p.Cin;  // first reduction index of the filter tap
+    }
+    int xb = kb_begin * ROW_BYTES;
+    uint32_t s = seq0 % R, round = seq0 / R;
+    for (int i = 0; i < nkb; ++i) {
+        if (round > 0 && !mbar_wait(bar0 + 8 * (EMPTY + s), (round & 1) ^ 1, s_abort)) return false;
+        const uint32_t full = bar0 + 8 * (FULL + s);
+        mbar_arrive_expect_tx(full, BN * ROW_BYTES);
+        if (p.conv) {
+            const int kx = kx_tap + cb * BK;
+            tma_load_2d(ring0 + s * SLOT, tmap_w, W4 ? kx / 2 : kx, n0, full);
+            if (++cb == p.cblocks) {
+                cb = 0;
+                kx_tap += p.Cin;
+            }
+        } else {
+            tma_load_2d(ring0 + s * SLOT, tmap_w, xb, n0, full);
+            xb += ROW_BYTES;
+        }
+        if (++s == R) {
+            s = 0;
+            ++round;
+        }
+    }
+    return true;
+}
+
+// int4 -> int8 (x16) expansion of the weight tiles, run by four groups of two warps: group g takes
+// the k-blocks g, g + 4, ... of the CTA's sequence, so four tiles are in the making at a time.  (A
+// group's turn costs some 350 cycles of waits, fence and arrivals on top of its arithmetic, and a
+// lone warp issues an instruction every four to five cycles: with two groups of four warps a tile
+// took about 900 cycles per group against 620 for the two k-blocks' MMAs.)  A thread reads
+// 16-byte runs of packed codes from the packed ring and writes them as two 16-byte chunks of the
+// swizzled int8 tile: nibble -> high half of the byte (= 16 q), two ANDs and a shift per 8 codes.
+template <int BN, class L>
+__device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int total_kb, uint8_t* sB, const uint8_t* sP,
+                                               uint32_t bar0, volatile int* s_abort)
+{
+    constexpr int RUNS = (BN * 4) / 64;           // 16-byte packed runs per thread
+    constexpr uint32_t PS = L::PS > 0 ? L::PS : 1;  // (instantiated, never run, for W8)
+    for (int it = group; it < total_kb; it += 4) {
+        const uint32_t sp = static_cast<uint32_t>(it) % PS, rp = static_cast<uint32_t>(it) / PS;
+        const uint32_t se = static_cast<uint32_t>(it) % L::ES, re = static_cast<uint32_t>(it) / L::ES;
+        bool ok = mbar_wait(bar0 + 8 * (L::FULL_P + sp), rp & 1, s_abort);
+        if (ok && re > 0) ok = mbar_wait(bar0 + 8 * (L::EMPTY_B + se), (re & 1) ^ 1, s_abort);
+        if (!__all_sync(0xffffffffu, ok)) break;  // the warp leaves together
+        const uint8_t* stg = sP + sp * L::P_BYTES;
+        uint8_t* b_stage = sB + se * L::B_BYTES;
+        // all loads first: the compiler cannot move a load above a store to the other ring by itself
         uint4 wv[RUNS];
 #pragma unroll
         for (int t = 0; t < RUNS; ++t) {
-            const int task = gt + t * 128;
+            const int task = gt + t * 64;
             wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
         }
-        // group barrier between the reads and the in-place writes; it also carries the vote on whether
-        // every thread's wait succeeded, so that the group leaves the loop together after a timeout
-        uint32_t all_landed;
-        asm volatile(
-            "{\n\t"
-            ".reg .pred p, q;\n\t"
-            "setp.ne.u32 q, %1, 0;\n\t"
-            "barrier.cta.red.and.pred p, %2, 128, q;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t"
-            "}\n"
-            : "=r"(all_landed)
-            : "r"(landed), "r"(2 + group)
-            : "memory");
-        if (!all_landed) break;
 #pragma unroll
         for (int t = 0; t < RUNS; ++t) {
-            const int task = gt + t * 128;
+            const int task = gt + t * 64;
             const int r = task >> 2, j = task & 3;
             const uint4 w = wv[t];
             uint4 c0, c1;
@@ -427,43 +524,60 @@ __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int 
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_unpacked + 8 * s);
-        s += 2;
-        if (s >= STAGES) {
-            s -= STAGES;
-            ph ^= 1;
+        if (lane == 0) {
+            mbar_arrive(bar0 + 8 * (L::READY_B + se));
+            mbar_arrive(bar0 + 8 * (L::EMPTY_P + sp));
         }
     }
 }
 
-// The k-blocks first, first + step, ... of one output tile: wait for the stage, issue its four
-// MMAs into `acc`, hand the stage back.  Runs in a single thread (step <= STAGES).
-template <int BN, int STAGES, class L>
-__device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t bar_ready,
-                                               uint32_t bar_empty, uint32_t a0, uint32_t b0, volatile int* s_abort,
-                                               int seq0 = 0)
+// The k-blocks first, first + step, ... of one output tile: wait for the tiles, issue the four MMAs
+// into `acc`, hand the slots back.  Runs in a single thread.  seq0 as above.
+template <int BN, bool W4, class L>
+__device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t seq0, uint32_t a0,
+                                               uint32_t b0, uint32_t bar0, volatile int* s_abort)
 {
     constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
-    // seq0: position of the tile's first k-block in the CTA's running sequence of pipeline stages
-    const uint32_t seq = static_cast<uint32_t>(seq0 + first);
-    uint32_t s = seq % STAGES, ph = (seq / STAGES) & 1;
     for (int i = first; i < nkb; i += step) {
-        if (!mbar_wait(bar_ready + 8 * s, ph, s_abort)) return false;
+        const uint32_t q = seq0 + i;
+        const uint32_t sa = q % L::AS, ra = q / L::AS, se = q % L::ES, re = q / L::ES;
+        if (!mbar_wait(bar0 + 8 * (L::FULL_A + sa), ra & 1, s_abort)) return false;
+        if (!mbar_wait(bar0 + 8 * (L::READY_B + se), re & 1, s_abort)) return false;
         tc_fence_after_sync();
-        const uint64_t a_desc = smem_desc_sw128(a0 + s * L::A_BYTES);
-        const uint64_t b_desc = smem_desc_sw128(b0 + s * L::B_BYTES);
+        const uint64_t a_desc = smem_desc_sw128(a0 + sa * L::A_BYTES);
+        const uint64_t b_desc = smem_desc_sw128(b0 + se * L::B_BYTES);
 #pragma unroll
         for (int k = 0; k < BK / 32; ++k)
             mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (i != first) || k != 0);
-        tc_commit(bar_empty + 8 * s);
-        s += step;
-        if (s >= STAGES) {
-            s -= STAGES;
-            ph ^= 1;
-        }
+        tc_commit(bar0 + 8 * (L::EMPTY_A + sa));
+        if (W4) tc_commit(bar0 + 8 * (L::EMPTY_B + se));
     }
     return true;
 }
+
+template <int BN, int STAGES, bool W4>
+struct TmaSmem : Rings<BN, STAGES, W4, false> {
+    using R = Rings<BN, STAGES, W4, false>;
+    static constexpr int OFF_BARS = R::RINGS_END;
+    static constexpr int NUM_BARS = R::RING_BARS + 1;
+    static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // read as float4
+    static constexpr int OFF_BIAS = OFF_COMB + BN * 4;
+    static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
+    static constexpr int TOTAL = OFF_MISC + 64 + 1024;
+    static_assert(TOTAL <= 232448, "shared memory of one CTA");
+    // warps: 0 activation producer, 1 MMA issuer, 2-5 epilogue, 6-9 epilogue helpers (the other half
+    // of the tile's columns), W4: 6-13 nibble expansion during the main loop
+    static constexpr int WORK_THREADS = W4 ? 448 : 320;
+    static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
+    // One thread issues a 128-wide MMA about every 68 cycles, the tensor core retires it in 64: a
+    // lone issuer, which also waits and commits once per k-block, cannot keep the pipe busy.  Narrow
+    // tiles therefore get a second issuer: even k-blocks accumulate into one accumulator, odd ones
+    // into another, and the epilogue adds the two (integer adds: exact).
+    static constexpr bool DUAL = BN == 128;
+    static constexpr int MMA2_WARP = B_WARP + 1;
+    static constexpr int THREADS = WORK_THREADS + 32 + (DUAL ? 32 : 0);
+    static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
+};
 
 template <int BN, int STAGES, bool W4>
 __global__ void __maxnreg__(96)
@@ -476,6 +590,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                                                ~static_cast<uintptr_t>(1023));
     uint8_t* sA = smem + L::OFF_A;
     uint8_t* sB = smem + L::OFF_B;
+    uint8_t* sP = smem + L::OFF_P;  // W4: packed weight tiles
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
     float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
     float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
@@ -493,18 +608,12 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const bool direct = splits == 1 && p.Y != nullptr && p.acc_out == nullptr;
     const bool dual = L::DUAL && nkb >= 2;  // two MMA issuers, two accumulators
 
-    const uint32_t bar_full = smem_u32(bars);                 // TMA bytes of the stage have landed
-    const uint32_t bar_unpacked = smem_u32(bars + STAGES);    // W4: nibbles expanded into the B tile
-    const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);   // MMAs reading the stage have finished
-    const uint32_t bar_accum = smem_u32(bars + 3 * STAGES);
+    const uint32_t bar0 = smem_u32(bars);  // ring barriers, see Rings
+    const uint32_t bar_accum = smem_u32(bars + L::RING_BARS);
 
     pdl_launch_dependents();
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
-            mbar_init(bar_unpacked + 8 * s, 4);  // the four warps of an expansion group
-            mbar_init(bar_empty + 8 * s, 1);
-        }
+        init_ring_barriers<L>(bar0, W4);
         mbar_init(bar_accum, dual ? 2 : 1);
         *s_abort = 0;
         fence_barrier_init();
@@ -526,93 +635,18 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------------------ activation-tile producer
-        if (lane == 0) {
-            int img_b = 0, ho0 = 0, wo0 = 0;
-            if (p.conv) {
-                img_b = m0 / p.HoWo;
-                const int rem = m0 - img_b * p.HoWo;
-                ho0 = rem / p.Wo;
-                wo0 = rem - ho0 * p.Wo;
-            }
-            // single-thread loop: all indices are carried along instead of being recomputed
-            const uint32_t a0 = smem_u32(sA);
-            uint32_t s = 0, ph = 1;
-            int tap = 0, cb = 0, kh = 0, kw = 0;
-            if (p.conv) {
-                tap = kb_begin / p.cblocks;
-                cb = kb_begin - tap * p.cblocks;
-                kh = tap / 3;
-                kw = tap - 3 * kh;
-            }
-            int xa = kb_begin * BK;
-            for (int i = 0; i < nkb; ++i) {
-                if (i >= STAGES && !mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;  // slots start out free
-                const uint32_t full = bar_full + 8 * s;
-                mbar_arrive_expect_tx(full, L::A_BYTES);
-                if (p.conv) {
-                    tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
-                    if (++cb == p.cblocks) {
-                        cb = 0;
-                        if (++kw == 3) {
-                            kw = 0;
-                            ++kh;
-                        }
-                    }
-                } else {
-                    tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
-                    xa += BK;
-                }
-                if (++s == STAGES) {
-                    s = 0;
-                    ph ^= 1;
-                }
-            }
-        }
+        if (lane == 0) produce_a_tile<L>(&tmap_a, p, 0, kb_begin, nkb, m0, smem_u32(sA), bar0, s_abort);
         __syncwarp();
     } else if (warp == L::B_WARP) {
         // ------------------------------------------------------------ weight-tile producer
-        // a thread of its own: one TMA issue costs a few hundred cycles of a single thread, and
-        // with both operands on one thread the issue rate, not the MMA, sets the k-block cadence
-        if (lane == 0) {
-            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
-            const uint32_t b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
-            uint32_t s = 0, ph = 1;
-            int tap = 0, cb = 0;
-            if (p.conv) {
-                tap = kb_begin / p.cblocks;
-                cb = kb_begin - tap * p.cblocks;
-            }
-            int kx_tap = tap * p.Cin;  // conv: first reduction index of the tap
-            int xb = kb_begin * ROW_BYTES;
-            for (int i = 0; i < nkb; ++i) {
-                if (i >= STAGES && !mbar_wait(bar_empty + 8 * s, ph, s_abort)) break;  // slots start out free
-                const uint32_t full = bar_full + 8 * s;
-                mbar_arrive_expect_tx(full, BN * ROW_BYTES);
-                if (p.conv) {
-                    const int kx = kx_tap + cb * BK;
-                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
-                    if (++cb == p.cblocks) {
-                        cb = 0;
-                        kx_tap += p.Cin;
-                    }
-                } else {
-                    tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
-                    xb += ROW_BYTES;
-                }
-                if (++s == STAGES) {
-                    s = 0;
-                    ph ^= 1;
-                }
-            }
-        }
+        if (lane == 0)
+            produce_b_tile<BN, W4, L>(&tmap_w, p, 0, kb_begin, nkb, n0, smem_u32(W4 ? sP : sB), bar0, s_abort);
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            // W4: the expansion warps arrive only after they have seen the TMA bytes land, so their
-            // barrier alone orders both operands
-            const bool ok = issue_k_blocks<BN, STAGES, L>(0, dual ? 2 : 1, nkb, tmem_base, W4 ? bar_unpacked : bar_full,
-                                                          bar_empty, smem_u32(sA), smem_u32(sB), s_abort);
+            const bool ok = issue_k_blocks<BN, W4, L>(0, dual ? 2 : 1, nkb, tmem_base, 0, smem_u32(sA), smem_u32(sB), bar0,
+                                                      s_abort);
             if (ok) tc_commit(bar_accum);
         }
         __syncwarp();
@@ -642,8 +676,8 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             }
         } else if (W4) {
             // -------------------------------------------------------- int4 -> int8 (x16) expansion
-            const int group = (warp - 6) >> 2;  // warps 6-9 and 10-13
-            expand_nibbles<BN, STAGES, L>(group, tid - 192 - group * 128, lane, nkb, sB, bar_full, bar_unpacked, s_abort);
+            const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
+            expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, nkb, sB, sP, bar0, s_abort);
         }
         if (warp < 10) {
             // -------------------------------------------------------- epilogue, part 1
@@ -692,8 +726,8 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     } else if (L::DUAL && warp == L::MMA2_WARP) {
         // ------------------------------------------------------------ second MMA issuer: odd k-blocks
         if (lane == 0 && dual) {
-            const bool ok = issue_k_blocks<BN, STAGES, L>(1, 2, nkb, tmem_base + BN, W4 ? bar_unpacked : bar_full,
-                                                          bar_empty, smem_u32(sA), smem_u32(sB), s_abort);
+            const bool ok = issue_k_blocks<BN, W4, L>(1, 2, nkb, tmem_base + BN, 0, smem_u32(sA), smem_u32(sB), bar0,
+                                                      s_abort);
             if (ok) tc_commit(bar_accum);
         }
     }
@@ -786,17 +820,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 // tile (tensor memory -> registers -> fp16 stores) runs while the MMAs of the next tile are
 // already being issued, and the TMA pipeline never drains between tiles.
 template <int BN, int STAGES, bool W4>
-struct PersistSmem {
-    static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
-    // packed int4 rows land in the last half of the B slot and are expanded in place
-    static constexpr int STG_BYTES = 0;
-    static constexpr int STG_OFFSET = BN * (BK / 2);
-    static constexpr int OFF_A = 0;
-    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_STG = OFF_B + STAGES * B_BYTES;
-    static constexpr int OFF_BARS = OFF_STG + STAGES * STG_BYTES;
-    static constexpr int NUM_BARS = 3 * STAGES + 4;
+struct PersistSmem : Rings<BN, STAGES, W4, true> {
+    using R = Rings<BN, STAGES, W4, true>;
+    static constexpr int OFF_BARS = R::RINGS_END;
+    static constexpr int NUM_BARS = R::RING_BARS + 4;
     static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][BN] floats
     static constexpr int OFF_BIAS = OFF_COMB + 2 * BN * 4;
     static constexpr int OFF_MISC = OFF_BIAS + 2 * BN * 4;
@@ -826,6 +853,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                                                ~static_cast<uintptr_t>(1023));
     uint8_t* sA = smem + L::OFF_A;
     uint8_t* sB = smem + L::OFF_B;
+    uint8_t* sP = smem + L::OFF_P;  // W4: packed weight tiles
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
     float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
     float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
@@ -838,19 +866,13 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     const int my_tiles = (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                          static_cast<int>(gridDim.x);
 
-    const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_unpacked = smem_u32(bars + STAGES);
-    const uint32_t bar_empty = smem_u32(bars + 2 * STAGES);
-    const uint32_t bar_acc_full = smem_u32(bars + 3 * STAGES);       // [2]: accumulator complete
-    const uint32_t bar_acc_empty = smem_u32(bars + 3 * STAGES + 2);  // [2]: accumulator drained
+    const uint32_t bar0 = smem_u32(bars);  // ring barriers, see Rings
+    const uint32_t bar_acc_full = smem_u32(bars + L::RING_BARS);       // [2]: accumulator complete
+    const uint32_t bar_acc_empty = smem_u32(bars + L::RING_BARS + 2);  // [2]: accumulator drained
 
     pdl_launch_dependents();
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 2);  // activation producer + weight producer
-            mbar_init(bar_unpacked + 8 * s, 4);  // the four warps of an expansion group
-            mbar_init(bar_empty + 8 * s, 1);
-        }
+        init_ring_barriers<L>(bar0, W4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, dual ? 2 : 1);
             mbar_init(bar_acc_empty + 8 * b, 8);  // epilogue warps and their helpers
@@ -874,79 +896,22 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     if (warp == 0) {
         // ------------------------------------------------------------ activation-tile producer
         if (lane == 0) {
-            // single-thread loop: all indices are carried along instead of being recomputed
-            const uint32_t a0 = smem_u32(sA);
-            uint32_t s = 0, ph = 1;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = blockIdx.x + t * gridDim.x;
-                const int m0 = (tile / n_tiles) * BM;
-                int img_b = 0, ho0 = 0, wo0 = 0;
-                if (p.conv) {
-                    img_b = m0 / p.HoWo;
-                    const int rem = m0 - img_b * p.HoWo;
-                    ho0 = rem / p.Wo;
-                    wo0 = rem - ho0 * p.Wo;
-                }
-                int cb = 0, kh = 0, kw = 0, xa = 0;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (t > 0 || kb >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);  // slots start out free
-                    if (!ok) break;
-                    const uint32_t full = bar_full + 8 * s;
-                    mbar_arrive_expect_tx(full, L::A_BYTES);
-                    if (p.conv) {
-                        tma_load_4d(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
-                        if (++cb == p.cblocks) {
-                            cb = 0;
-                            if (++kw == 3) {
-                                kw = 0;
-                                ++kh;
-                            }
-                        }
-                    } else {
-                        tma_load_2d(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
-                        xa += BK;
-                    }
-                    if (++s == STAGES) {
-                        s = 0;
-                        ph ^= 1;
-                    }
-                }
+                ok = produce_a_tile<L>(&tmap_a, p, static_cast<uint32_t>(t * nkb), 0, nkb, (tile / n_tiles) * BM, smem_u32(sA),
+                                       bar0, s_abort);
             }
         }
         __syncwarp();
     } else if (warp == L::B_WARP) {
         // ------------------------------------------------------------ weight-tile producer
         if (lane == 0) {
-            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
-            const uint32_t b0 = smem_u32(sB) + (W4 ? L::STG_OFFSET : 0);
-            uint32_t s = 0, ph = 1;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = blockIdx.x + t * gridDim.x;
-                const int n0 = (tile % n_tiles) * BN;
-                int cb = 0, kx_tap = 0, xb = 0;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (t > 0 || kb >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ph, s_abort);  // slots start out free
-                    if (!ok) break;
-                    const uint32_t full = bar_full + 8 * s;
-                    mbar_arrive_expect_tx(full, BN * ROW_BYTES);
-                    if (p.conv) {
-                        const int kx = kx_tap + cb * BK;
-                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, W4 ? kx / 2 : kx, n0, full);
-                        if (++cb == p.cblocks) {
-                            cb = 0;
-                            kx_tap += p.Cin;
-                        }
-                    } else {
-                        tma_load_2d(b0 + s * L::B_BYTES, &tmap_w, xb, n0, full);
-                        xb += ROW_BYTES;
-                    }
-                    if (++s == STAGES) {
-                        s = 0;
-                        ph ^= 1;
-                    }
-                }
+                ok = produce_b_tile<BN, W4, L>(&tmap_w, p, static_cast<uint32_t>(t * nkb), 0, nkb, (tile % n_tiles) * BN,
+                                               smem_u32(W4 ? sP : sB), bar0, s_abort);
             }
         }
         __syncwarp();
@@ -955,7 +920,6 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         // warp 1 (and, for narrow tiles, warp MMA2_WARP with the odd k-blocks and an accumulator of its own)
         if (lane == 0 && (warp == 1 || dual)) {
             const int which = warp == 1 ? 0 : 1;
-            const uint32_t bar_ready = W4 ? bar_unpacked : bar_full;  // W4: implies the TMA bytes landed
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t & 1;
@@ -963,8 +927,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 ok = mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, s_abort);
                 if (!ok) break;
                 tc_fence_after_sync();
-                ok = issue_k_blocks<BN, STAGES, L>(which, dual ? 2 : 1, nkb, tmem_base + buf * L::ACC_COLS + which * BN,
-                                                   bar_ready, bar_empty, smem_u32(sA), smem_u32(sB), s_abort, t * nkb);
+                ok = issue_k_blocks<BN, W4, L>(which, dual ? 2 : 1, nkb, tmem_base + buf * L::ACC_COLS + which * BN,
+                                               static_cast<uint32_t>(t * nkb), smem_u32(sA), smem_u32(sB), bar0, s_abort);
                 if (ok) tc_commit(bar_acc_full + 8 * buf);
             }
         }
@@ -1059,9 +1023,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
     } else if (W4 && warp < L::HELPER0) {
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion
-        const int group = (warp - 6) >> 2;  // warps 6-9 and 10-13
-        expand_nibbles<BN, STAGES, L>(group, tid - 192 - group * 128, lane, my_tiles * nkb, sB, bar_full, bar_unpacked,
-                                      s_abort);
+        const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
+        expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, my_tiles * nkb, sB, sP, bar0, s_abort);
     }
 
     if (*s_abort) {
@@ -1211,7 +1174,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     }
     if (rc != MIXDQ_OK) return rc;
     // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
-    const bool wide = (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
+    // (W4 runs on 128-wide tiles only: its packed ring needs the room, and it measured no slower)
+    const bool wide = !w4 && (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
     const uint32_t bn = wide ? 256 : 128;
     if (w4)
         rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, bn, false);
@@ -1235,9 +1199,7 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         if (rc != MIXDQ_OK) return rc;
     }
     if (persistent) {
-        if (wide)
-            return w4 ? launch_persistent<256, 4, true>(ta, tw, ty, tp, num_sms, stream)
-                      : launch_persistent<256, 4, false>(ta, tw, ty, tp, num_sms, stream);
+        if (wide) return launch_persistent<256, 4, false>(ta, tw, ty, tp, num_sms, stream);
         return w4 ? launch_persistent<128, 6, true>(ta, tw, ty, tp, num_sms, stream)
                   : launch_persistent<128, 6, false>(ta, tw, ty, tp, num_sms, stream);
     }
@@ -1246,9 +1208,7 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         splits = 1;
         while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;
     }
-    if (wide)
-        return w4 ? launch_tma<256, 4, true>(ta, tw, ty, tp, splits, stream)
-                  : launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
+    if (wide) return launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
     return w4 ? launch_tma<128, 6, true>(ta, tw, ty, tp, splits, stream)
               : launch_tma<128, 6, false>(ta, tw, ty, tp, splits, stream);
 }
