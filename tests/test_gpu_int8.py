@@ -171,7 +171,9 @@ def test_bos_aware_kv(bits, B, N, use_ws):
                                                     (3, 9, 7, 48, 24, 2), (3, 8, 8, 32, 40, 1),
                                                     (2, 32, 32, 160, 136, 1), (1, 64, 64, 32, 24, 1),
                                                     (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2),
-                                                    (1, 12, 12, 256, 32, 1), (1, 64, 64, 32, 648, 1)])
+                                                    (1, 12, 12, 256, 32, 1), (1, 64, 64, 32, 648, 1),
+                                                    # stride 2 on the TMA path: boxes of 4 and of 8 output rows
+                                                    (1, 64, 64, 64, 40, 2), (2, 32, 32, 160, 136, 2)])
 def test_conv3x3(bits, B, H, W, Cin, Cout, stride, use_ws):
     X = synth.normal_f16((B, H, W, Cin), 1.0, seed=H * W + Cin)
     Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin)
