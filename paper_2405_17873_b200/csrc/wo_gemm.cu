@@ -319,8 +319,11 @@ wo_kernel(const uint8_t* __restrict__ packed, long long pitch, const Params p, i
 // packed weights, so the kernel is built around that stream.  The first weight loads go out
 // before the wait on the previous kernel -- weights and their parameters are constants of the
 // layer, only the activations can come from the kernel before -- so consecutive layers keep
-// the memory system busy across the kernel boundary.  The few activation rows are read
-// straight from global memory (they stay in L1) instead of being staged in shared memory.
+// the memory system busy across the kernel boundary.  The token rows come into shared memory
+// by bulk copies (one per row, issued by one thread right after the wait): the load/store
+// units are full of weight loads by then, and a staging pass through registers queued behind
+// them took 2 to 6 us.  The rows stay in their natural order; the decode's pair order is
+// applied to the fragments as they are read.
 // CTA = 8 warps = TILES channel tiles x (8 / TILES) slices of the reduction.
 template <int BITS, bool SIGNED, int NT, int TILES>
 __global__ void __launch_bounds__(kThreads, 3)
@@ -330,12 +333,19 @@ wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Param
     constexpr int MB = 8 * NT;
     constexpr int GROUP = BITS == 8 ? 2 : 4;
     extern __shared__ __align__(16) uint8_t smem[];
-    const int x_stride = k_pad * 2 + 64;  // 64 mod 128 bytes: quad reads of two token rows do not collide
+    const int x_stride = k_pad * 2 + 16;  // token rows 16 bytes off a multiple of 128
     uint8_t* sX = smem;
     float* sRed = reinterpret_cast<float*>(smem + MB * x_stride);  // [SLICES][TILES * 16][MB]
+    __shared__ __align__(8) uint64_t x_bar;
+    __shared__ int x_abort;
 
     pdl_launch_dependents();
     const int tid = threadIdx.x;
+    if (tid == 0) {
+        mbar_init(smem_u32(&x_bar), 1);
+        x_abort = 0;
+        fence_barrier_init();
+    }
     const int warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
     const int tile = warp % TILES, slice = warp / TILES;
@@ -376,34 +386,29 @@ wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Param
     if (grp < groups) begin_group(grp);  // issued before the wait: weights are constants of the layer
     pdl_wait();                          // the activations may be the previous kernel's output
 
-    // the token rows, once per CTA, in the order in which the decode produces the weights
+    // the token rows, once per CTA: bulk copies of the rows that exist, zeros elsewhere
+    __syncthreads();  // the barrier is initialised
     {
-        const int per_row = k_pad / 8, total16 = MB * per_row;
-        for (int base = tid; base < total16; base += kThreads * 6) {
-            uint4 v[6];
-#pragma unroll
-            for (int i = 0; i < 6; ++i) {
-                const int idx = base + i * kThreads;
-                const int r = idx / per_row, k = (idx - r * per_row) * 8;
-                v[i] = (idx < total16 && r < p.M && k < p.K)
-                           ? __ldg(reinterpret_cast<const uint4*>(p.X + static_cast<long long>(r) * p.ldx + k))
-                           : make_uint4(0, 0, 0, 0);
-            }
-#pragma unroll
-            for (int i = 0; i < 6; ++i) {
-                const int idx = base + i * kThreads;
-                if (idx >= total16) break;
-                const int r = idx / per_row, j = idx - r * per_row;
-                uint4 x = v[i];
-                if (BITS != 8)  // the decode yields pairs (0, 2), (1, 3) of each run of four
-                    x = make_uint4(__byte_perm(x.x, x.y, 0x5410), __byte_perm(x.x, x.y, 0x7632),
-                                   __byte_perm(x.z, x.w, 0x5410), __byte_perm(x.z, x.w, 0x7632));
-                const int U = j >> 4, tt = (j >> 2) & 3, sub = j & 3;
-                *reinterpret_cast<uint4*>(sX + r * x_stride + (16 * U + 4 * sub + tt) * 16) = x;
-            }
+        const int rows = p.M < MB ? p.M : MB;
+        if (tid == 0) {
+            mbar_arrive_expect_tx(smem_u32(&x_bar), static_cast<uint32_t>(rows) * p.K * 2);
+            for (int r = 0; r < rows; ++r)
+                bulk_load(smem_u32(sX + r * x_stride), p.X + static_cast<long long>(r) * p.ldx, p.K * 2, smem_u32(&x_bar));
+        }
+        const int pad16 = (k_pad - p.K) / 8;  // 16-byte chunks past the end of a row
+        for (int idx = tid; idx < rows * pad16; idx += kThreads) {
+            const int r = idx / pad16, c = idx - r * pad16;
+            *reinterpret_cast<uint4*>(sX + r * x_stride + (p.K + c * 8) * 2) = make_uint4(0, 0, 0, 0);
+        }
+        const int per_row = k_pad / 8;
+        for (int idx = tid; idx < (MB - rows) * per_row; idx += kThreads) {
+            const int r = rows + idx / per_row, c = idx % per_row;
+            *reinterpret_cast<uint4*>(sX + r * x_stride + c * 16) = make_uint4(0, 0, 0, 0);
         }
     }
     __syncthreads();
+    const bool x_ok = mbar_wait(smem_u32(&x_bar), 0, &x_abort);
+    if (!x_ok && tid == 0 && p.status) atomicExch(p.status, MIXDQ_ERR_TIMEOUT);
 
     for (; grp < groups; grp += gridDim.x) {
         const __half2 zlo_a = __float2half2_rn(1024.f + z_a), zhi_a = __float2half2_rn(-(64.f + z_a));
@@ -426,10 +431,14 @@ wo_small_kernel(const uint8_t* __restrict__ packed, long long pitch, const Param
                     decode_substep<BITS, SIGNED>(rb[i], sub, zlo_b, zhi_b, fb);
                     const uint32_t a1[4] = {fa[0], fb[0], fa[1], fb[1]};
                     const uint32_t a2[4] = {fa[2], fb[2], fa[3], fb[3]};
-                    const int slot = (16 * (u0 + i) + 4 * sub + t) * 16;
+                    // the thread's eight reduction indices of this substep are one 16-byte chunk of the row
+                    const int slot = (16 * (u0 + i) + 4 * t + sub) * 16;
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(sX + (g + 8 * nt) * x_stride + slot);
+                        uint4 x = *reinterpret_cast<const uint4*>(sX + (g + 8 * nt) * x_stride + slot);
+                        if (BITS != 8)  // the decode yields pairs (0, 2), (1, 3) of each run of four
+                            x = make_uint4(__byte_perm(x.x, x.y, 0x5410), __byte_perm(x.x, x.y, 0x7632),
+                                           __byte_perm(x.z, x.w, 0x5410), __byte_perm(x.z, x.w, 0x7632));
                         mma_16816(acc[nt], a1, x.x, x.y);
                         mma_16816(acc[nt], a2, x.z, x.w);
                     }
@@ -470,7 +479,7 @@ int launch_small_tiles(const Params& p, const void* packed, long long pitch, cud
 {
     constexpr int MB = 8 * NT;
     const int k_pad = static_cast<int>(round_up(p.K, kUnit));
-    const size_t smem = static_cast<size_t>(MB) * (k_pad * 2 + 64) + 8 * 16 * MB * sizeof(float);
+    const size_t smem = static_cast<size_t>(MB) * (k_pad * 2 + 16) + 8 * 16 * MB * sizeof(float);
     auto kernel = wo_small_kernel<BITS, SIGNED, NT, TILES>;
     static bool attr_set = false;
     if (!attr_set) {
