@@ -38,12 +38,17 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--table", default="w4a8", choices=["w4a8", "a16"])
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="weight-bound regime: only the linear layers of the a16 table, each on this many rows "
+                         "(e.g. 16); reports the weight stream in GB/s against the HBM roofline")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
 
 def workload_name(args):
+    if args.tokens > 0:
+        return f"unet_linear_sweep_{args.table}_{args.tokens}tokens"
     return f"unet_sweep_sdxl512_{args.table}_b{args.batch}"
 
 
@@ -247,7 +252,9 @@ def run_ours(args):
     build.build()
     mixdq.lib()  # fail here, loudly, if the CUDA library is missing
 
-    sweep = UNetSweep(args.batch, args.table, seed=5 + rank)
+    if args.tokens > 0 and args.table != "a16":
+        raise SystemExit("--tokens needs --table a16 (the weight-only engine)")
+    sweep = UNetSweep(args.batch, args.table, seed=5 + rank, tokens=args.tokens)
     tc_layers = [pl for pl in sweep.layers if sweep.uses_tensor_int8(pl)]
     other_layers = [pl for pl in sweep.layers if not sweep.uses_tensor_int8(pl)]
     if args.table == "a16":
@@ -358,6 +365,17 @@ def run_ours(args):
                               "their quant_kernel pre-pass, all tensor-core int8 layers of the step",
                     "peak_source": f"{peaks['source']} bf16 sustained x {INT8_TO_BF16_NOMINAL:g} (nominal int8:bf16)",
                     "launches_per_step": group_launches[0], "layers": len(tc_layers), "ms_per_step": tc_ms}
+    elif args.tokens > 0:
+        # a few tokens per layer: one stream over the packed weights, bound by HBM
+        alg = sum(sweep.algorithmic_bytes(pl) for pl in sweep.layers)
+        achieved = alg / (other_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "kernel": "wo::wo_small_kernel (packed weights streamed once, decoded in registers, mma.sync fp16), "
+                              "all layers of the step",
+                    "peak_source": f"{peaks['source']} copy bandwidth",
+                    "launches_per_step": group_launches[1], "ms_per_step": other_ms,
+                    "algorithmic_bytes_per_step": alg}
     else:
         # image batch >= 1 means hundreds of tokens per layer: the weight-only layers run on the
         # fp16 tensor cores (tcgen05 kind::f16) and are bound by that pipe, not by the weight stream
@@ -390,7 +408,7 @@ def run_ours(args):
             "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
             "device_status": status,
         }
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and args.tokens == 0:
             out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
         print(json.dumps(out))
     if world > 1:

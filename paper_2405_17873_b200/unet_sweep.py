@@ -30,12 +30,17 @@ class PackedLayer:
 
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
-                 layers: Optional[List[synth.LayerSpec]] = None):
+                 layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0):
+        """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
+        (whatever the image size), so that a layer is one stream over its packed weights."""
         assert table in ("w4a8", "a16")
         self.batch = batch
+        self.tokens = tokens
         self.table = table
         self.device = device
         self.specs = layers if layers is not None else synth.unet_layers()
+        if tokens > 0:
+            self.specs = [l for l in self.specs if l.kind == "linear"]
         if layers is None:
             if table == "w4a8":
                 synth.assign_bits_w4a8(self.specs, seed)
@@ -55,7 +60,7 @@ class UNetSweep:
             return ("nhwc", B, l.H, l.H, l.Cin)
         if l.kind == "bos_kv":
             return ("text", B, synth.TOKENS_PER_PROMPT, l.K)
-        return ("rows", l.M * B, l.K)
+        return ("rows", self.tokens if self.tokens > 0 else l.M * B, l.K)
 
     def _y_shape(self, l: synth.LayerSpec):
         B = self.batch
@@ -66,7 +71,7 @@ class UNetSweep:
             return (B, l.H, l.H, l.N)
         if l.kind == "bos_kv":
             return (B, synth.TOKENS_PER_PROMPT, l.N)
-        return (l.M * B, l.N)
+        return (self.tokens if self.tokens > 0 else l.M * B, l.N)
 
     def _build(self, seed: int):
         g = torch.Generator(device=self.device).manual_seed(seed)
@@ -129,7 +134,10 @@ class UNetSweep:
 
     # ------------------------------------------------------------------ accounting
     def total_ops(self, subset=None) -> int:
-        return sum(pl.spec.ops(self.batch) for pl in (self.layers if subset is None else subset))
+        group = self.layers if subset is None else subset
+        if self.tokens > 0:
+            return sum(2 * self.tokens * pl.spec.N * pl.spec.K for pl in group)
+        return sum(pl.spec.ops(self.batch) for pl in group)
 
     def packed_weight_bytes(self) -> int:
         return sum(pl.packed.numel() for pl in self.layers)
