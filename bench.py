@@ -359,8 +359,12 @@ def run_ours(args):
         tc_ops = sweep.total_ops(tc_layers)
         achieved = tc_ops / (tc_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL
+        # DRAM bytes per step of these kernels from one ncu capture of this command at batch 4 (caches flushed
+        # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.00 GB read by the quantization
+        # passes (every layer's input once) + 2.96 GB by the GEMMs (weights and int8 activations once)
+        traffic = 5.97e9 if (args.batch == 4 and world == 1) else None
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
-                    "traffic": None,
+                    "traffic": traffic,
                     "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
                               "their quant_kernel pre-pass, all tensor-core int8 layers of the step",
                     "peak_source": f"{peaks['source']} bf16 sustained x {INT8_TO_BF16_NOMINAL:g} (nominal int8:bf16)",
