@@ -354,9 +354,17 @@ struct Rings {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
     static constexpr int P_BYTES = BN * (BK / 2);
-    static constexpr int AS = W4 ? (PERSIST ? 4 : 5) : STAGES;  // activation tiles
+    // W4 needs an even number of int8 weight tiles: k-blocks alternate between the two MMA issuers by
+    // the parity of their position in the CTA's sequence, so a weight slot always belongs to the same
+    // issuer and its MMAs retire in order.  An expansion group reaches k-block i only after it has seen
+    // the MMAs of k-block i - 4 - ES retire, which are the same issuer's as those of i - 2 ES: the
+    // barrier of the slot can then never be a whole pair of phases behind what the group's parity wait
+    // assumes.  (All rings of the W8 kernels are even for the same reason: an issuer must meet every
+    // phase of the barriers it waits on.)
+    static constexpr int AS = W4 ? 4 : STAGES;                  // activation tiles
     static constexpr int ES = W4 ? 6 : STAGES;                  // int8 weight tiles (W4: expanded; four in the making)
-    static constexpr int PS = W4 ? (PERSIST ? 4 : 5) : 0;       // packed int4 weight tiles
+    static_assert(AS % 2 == 0 && ES % 2 == 0, "slots must keep their MMA issuer");
+    static constexpr int PS = W4 ? (PERSIST ? 4 : 6) : 0;       // packed int4 weight tiles
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + AS * A_BYTES;
     static constexpr int OFF_P = OFF_B + ES * B_BYTES;
@@ -445,7 +453,7 @@ __device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const 
     constexpr int R = W4 ? L::PS : L::ES;
     constexpr int SLOT = W4 ? L::P_BYTES : L::B_BYTES;
     constexpr int FULL = W4 ? L::FULL_P : L::READY_B;
-    constexpr int EMPTY = W4 ? L::EMPTY_P : L::EMPTY_A;  // W8: the MMA's one commit frees both tiles
+    constexpr int EMPTY = W4 ? L::EMPTY_P : L::EMPTY_A;  // W8: the MMA's commit frees both tiles of the slot
     int cb = 0, kx_tap = 0;
     if (p.conv) {
         const int tap = kb_begin / p.cblocks;
@@ -927,7 +935,10 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 ok = mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, s_abort);
                 if (!ok) break;
                 tc_fence_after_sync();
-                ok = issue_k_blocks<BN, W4, L>(which, dual ? 2 : 1, nkb, tmem_base + buf * L::ACC_COLS + which * BN,
+                // k-blocks alternate between the issuers by the parity of their position in the CTA's
+                // sequence (not in the tile: see Rings), so an issuer's first k-block of a tile is 0 or 1
+                const int first = dual ? ((which + t * nkb) & 1) : 0;
+                ok = issue_k_blocks<BN, W4, L>(first, dual ? 2 : 1, nkb, tmem_base + buf * L::ACC_COLS + which * BN,
                                                static_cast<uint32_t>(t * nkb), smem_u32(sA), smem_u32(sB), bar0, s_abort);
                 if (ok) tc_commit(bar_acc_full + 8 * buf);
             }
