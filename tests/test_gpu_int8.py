@@ -63,7 +63,10 @@ def test_linear_split_reduction(bits, M, K, N):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
-@pytest.mark.parametrize("M,K,N", [(2048, 272, 1288), (4100, 144, 1290), (2500, 1040, 1032)])
+@pytest.mark.parametrize("M,K,N", [(2048, 272, 1288), (4100, 144, 1290), (2500, 1040, 1032),
+                                   # three tiles per CTA with an odd number of k-blocks: ring slots and MMA
+                                   # issuers must stay in step across tile boundaries
+                                   (4096, 384, 1280), (6144, 640, 1536)])
 def test_linear_persistent_tiles(bits, M, K, N):
     # at least as many output tiles as SMs: the persistent kernel walks several tiles per CTA
     g = synth.normal_f16((M, K), 1.0, seed=M + K + 3)
