@@ -168,6 +168,30 @@ def test_bos_aware_kv(bits, B, N, use_ws):
 
 
 @pytest.mark.parametrize("bits", [8, 4])
+def test_fused_k_and_v_projection_equals_two_calls(bits):
+    # K and V of a cross-attention block read the same text embedding with the same scale: one call on
+    # the stacked weights [W_k; W_v] (per-channel scales and BOS rows stacked alike) must give, bit for
+    # bit, what the two separate calls give
+    B, N = 4, 640
+    E = synth.text_embedding(B, seed=4200)
+    Wk, Wv = synth.kv_weight(N, seed=4300), synth.kv_weight(N, seed=4301)
+    Ed = dev(E)
+    sx = mixdq.act_scale(Ed.reshape(-1, E.shape[-1]), skip_rows_mod=77)
+    st = status_word()
+    outs = []
+    for W in (Wk, Wv, np.concatenate([Wk, Wv], axis=0)):
+        s, _, packed = device_weights(W, bits, True)
+        bos = orc.bos_row(E[0, 0], W)
+        ws = workspace_for(B * 76, W.shape[0], 2048, bits)
+        outs.append(host(mixdq.crossattn_kv(Ed, packed, W.shape[0], bits, s, sx, dev(bos), workspace=ws, status=st)))
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    yk, yv, ykv = outs
+    assert np.array_equal(ykv[..., :N].view(np.uint16), yk.view(np.uint16))
+    assert np.array_equal(ykv[..., N:].view(np.uint16), yv.view(np.uint16))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("use_ws", [False, True])
 @pytest.mark.parametrize("B,H,W,Cin,Cout,stride", [(1, 8, 8, 16, 16, 1), (2, 12, 10, 32, 48, 1),
                                                     (2, 12, 10, 32, 48, 2), (1, 16, 16, 320, 136, 1),
