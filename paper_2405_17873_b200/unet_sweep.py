@@ -174,6 +174,7 @@ def _main(argv=None) -> int:
     ap.add_argument("--table", default="w4a8", choices=["w4a8", "a16"])
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--tokens", type=int, default=0, help="linear layers only: run on this many rows (weight-bound regime)")
     ap.add_argument("--eager", action="store_true", help="plain launches only, no graph and no timing")
     a = ap.parse_args(argv)
 
@@ -184,13 +185,13 @@ def _main(argv=None) -> int:
         raise SystemExit(f"no layer named {a.layer!r}")
     if a.w_bits is not None:
         pick[0].w_bits = a.w_bits
-    sw = UNetSweep(a.batch, a.table, layers=pick)
+    sw = UNetSweep(a.batch, a.table, layers=pick, tokens=a.tokens)
     pl = sw.layers[0]
     for _ in range(a.reps):
         sw.run_layer(pl)
     torch.cuda.synchronize()
     l = pl.spec
-    line = f"{l.name} {l.kind} M={l.M * a.batch} N={l.N} K={l.K} W{l.w_bits}A{l.a_bits}"
+    line = f"{l.name} {l.kind} M={a.tokens if a.tokens > 0 else l.M * a.batch} N={l.N} K={l.K} W{l.w_bits}A{l.a_bits}"
     if not a.eager:
         st = torch.cuda.Stream()
         with torch.cuda.stream(st):
