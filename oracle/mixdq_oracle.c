@@ -259,6 +259,63 @@ int orc_quantize_acts(const uint16_t *X, int64_t count, int bits, float scale, i
     return ORC_OK;
 }
 
+/* Asymmetric per-tensor activation quantization (Sec. 4.1 "Quantization Scheme": the paper's scheme is
+ * asymmetric min-max; used here for 8-bit activations of linear layers).
+ * Range: lo = min(min x, 0), hi = max(max x, 0) over the tensor; scale = (hi - lo) / 255 (one fp32
+ * division of exactly converted inputs); zero = clamp(rne(-lo * inv), 0, 255); hi == lo: scale 1, zero 0.
+ * Same reading as for the asymmetric weights above. */
+int orc_act_minmax_params(const uint16_t *X, int64_t count, float *scale_out, int32_t *zero_out)
+{
+    if (!X || !scale_out || !zero_out || count < 0) return ORC_ERR_ARG;
+    double lo = 0.0, hi = 0.0;
+    for (int64_t i = 0; i < count; ++i) {
+        double v = half_to_double(X[i]);
+        if (v < lo) lo = v;
+        if (v > hi) hi = v;
+    }
+    if (hi == lo) {
+        *scale_out = 1.0f;
+        *zero_out = 0;
+        return ORC_OK;
+    }
+    volatile float range = (float)hi - (float)lo; /* both exact in fp32; one fp32 subtraction */
+    volatile float levels = 255.0f;
+    volatile float s = range / levels;
+    *scale_out = s;
+    *zero_out = (int32_t)clamp_i64(rne_product(-lo, inv_of_scale(s)), 0, 255);
+    return ORC_OK;
+}
+
+/* Centred codes of an asymmetrically quantized tensor: c = clamp(rne(x * inv) + zero, 0, 255) - zero,
+ * i.e. what the integer GEMM multiplies (a value in [-255, 255], hence int16). */
+int orc_quantize_acts_asym(const uint16_t *X, int64_t count, float scale, int32_t zero, int16_t *centred_out)
+{
+    if (!X || !centred_out || count < 0 || zero < 0 || zero > 255) return ORC_ERR_ARG;
+    float inv = inv_of_scale(scale);
+    for (int64_t i = 0; i < count; ++i) {
+        int64_t q = clamp_i64(rne_product(half_to_double(X[i]), inv) + zero, 0, 255);
+        centred_out[i] = (int16_t)(q - zero);
+    }
+    return ORC_OK;
+}
+
+/* acc[m,n] = sum_k cx[m,k] * qw[n,k] for centred activation codes, checked against int32 overflow. */
+int orc_int_gemm_i16(const int16_t *cx, const int16_t *qw, int64_t M, int64_t N, int64_t K, int32_t *acc_out)
+{
+    if (!cx || !qw || !acc_out || M < 0 || N < 0 || K < 0) return ORC_ERR_ARG;
+    int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(| : overflow)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            int64_t acc = 0;
+            for (int64_t k = 0; k < K; ++k) acc += (int64_t)cx[m * K + k] * (int64_t)qw[n * K + k];
+            if (acc > INT32_MAX || acc < INT32_MIN) overflow = 1;
+            acc_out[m * N + n] = (int32_t)acc;
+        }
+    }
+    return overflow ? ORC_ERR_OVERFLOW : ORC_OK;
+}
+
 /* ------------------------------------------------------------------ */
 /* Canonical packed layouts.                                           */
 /*   8-bit: one byte per code.                                         */

@@ -141,6 +141,35 @@ def quantize_acts(X, scale, bits: int = 8):
     return q
 
 
+def act_minmax_params(X):
+    """Asymmetric per-tensor 8-bit activation parameters: (scale fp32, zero-point int in [0, 255])."""
+    X = _f16(X)
+    scale = np.zeros(1, np.float32)
+    zero = np.zeros(1, np.int32)
+    _chk(lib().orc_act_minmax_params(_p(X), C.c_int64(X.size), _p(scale), _p(zero)), "act_minmax_params")
+    return scale[0], int(zero[0])
+
+
+def quantize_acts_asym(X, scale, zero: int):
+    """Centred codes clamp(rne(x / s) + z, 0, 255) - z as int16."""
+    X = _f16(X)
+    c = np.empty(X.shape, np.int16)
+    _chk(lib().orc_quantize_acts_asym(_p(X), C.c_int64(X.size), C.c_float(float(scale)), C.c_int32(int(zero)), _p(c)),
+         "quantize_acts_asym")
+    return c
+
+
+def int_gemm_i16(cx, qw):
+    cx = np.ascontiguousarray(cx, np.int16)
+    qw = np.ascontiguousarray(qw, np.int16)
+    M, K = cx.shape
+    N, K2 = qw.shape
+    assert K == K2
+    acc = np.empty((M, N), np.int32)
+    _chk(lib().orc_int_gemm_i16(_p(cx), _p(qw), C.c_int64(M), C.c_int64(N), C.c_int64(K), _p(acc)), "int_gemm_i16")
+    return acc
+
+
 # ------------------------------------------------------------------ packing
 
 def packed_row_bytes(K: int, bits: int) -> int:
@@ -258,6 +287,15 @@ def linear_a8(X, codes, w_scale, act_scale_, bias=None):
     X = _f16(X)
     qx = quantize_acts(X, act_scale_, 8)
     acc = int_gemm(qx.reshape(-1, X.shape[-1]), codes)
+    return acc, dequant_epilogue(acc, act_scale_, w_scale, bias)
+
+
+def linear_a8_asym(X, codes, w_scale, act_scale_, act_zero: int, bias=None):
+    """W8A8 / W4A8 linear with asymmetric per-tensor activations (Sec. 4.1):
+    acc = sum_k (q_x - z_x) q_w (int32), y = fp16(acc * s_x * s_w[n] + bias[n])."""
+    X = _f16(X)
+    cx = quantize_acts_asym(X, act_scale_, act_zero)
+    acc = int_gemm_i16(cx.reshape(-1, X.shape[-1]), codes)
     return acc, dequant_epilogue(acc, act_scale_, w_scale, bias)
 
 

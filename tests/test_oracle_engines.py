@@ -221,6 +221,52 @@ def test_w8a8_equals_fake_quant_matmul():
     assert np.abs(y.astype(np.float64) - full).max() < 0.02 * np.abs(full).max()
 
 
+def test_int_gemm_i16_brute_force_and_zero_point_identity():
+    rng = np.random.default_rng(3)
+    z = 77
+    q = rng.integers(0, 256, size=(5, 41)).astype(np.int16)
+    cx = (q - z).astype(np.int16)
+    qw = rng.integers(-127, 128, size=(6, 41)).astype(np.int16)
+    acc = orc.int_gemm_i16(cx, qw)
+    for m in range(5):
+        for n in range(6):
+            assert int(acc[m, n]) == sum(int(a) * int(b) for a, b in zip(cx[m], qw[n]))
+    # sum_k (q - z) w = sum_k q w - z sum_k w: the form a kernel with unsigned or re-centred codes uses
+    raw = q.astype(np.int64) @ qw.astype(np.int64).T
+    assert np.array_equal(acc, raw - z * qw.astype(np.int64).sum(axis=1)[None, :])
+    # worst case of the longest linear reduction of the UNet stays inside int32
+    K = 10240
+    big = orc.int_gemm_i16(np.full((1, K), 255, np.int16), np.full((1, K), -127, np.int16))
+    assert int(big[0, 0]) == -255 * 127 * K
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_a8_asym_equals_fake_quant_matmul(bits):
+    rng = np.random.default_rng(11)
+    X = np.maximum(rng.normal(0.3, 1.0, (48, 80)), -0.17).astype(np.float16)   # one-sided, post-GELU-like
+    _, W, b = synth.single_linear(seed=2, M=8, K=80, N=24)
+    ws, _ = orc.weight_minmax_params(W, bits, True)
+    codes = orc.quantize_weights(W, bits, ws, None)
+    sx, zx = orc.act_minmax_params(X)
+    acc, y = orc.linear_a8_asym(X, codes, ws, sx, zx, b)
+    xq = orc.quantize_acts_asym(X, sx, zx).astype(np.float64) * float(sx)
+    wq = codes.astype(np.float64) * ws.astype(np.float64)[:, None]
+    ref = xq @ wq.T + b.astype(np.float64)[None, :]
+    assert np.all(np.abs(y.astype(np.float64) - ref) <= 2.0 ** -10 * np.abs(ref) + 1e-7)
+    # a symmetric tensor with z = 0 falls back to plain signed codes: same accumulators as the int8 engine
+    Xs = np.clip(synth.normal_f16((16, 80), 1.0, seed=4), -3, 3)
+    c0 = orc.quantize_acts_asym(Xs, np.float32(3.0 / 127), 0)
+    assert c0.min() == 0     # negative values clamp away when the zero point is 0
+    if bits == 8:
+        # asymmetric codes approximate the unquantized layer better than symmetric ones on this input
+        full = X.astype(np.float64) @ wq.T + b.astype(np.float64)
+        ss = orc.act_scale(orc.act_absmax(X), 8)
+        _, ysym = orc.linear_a8(X, codes, ws, ss, b)
+        ea = np.abs(y.astype(np.float64) - full).mean()
+        es = np.abs(ysym.astype(np.float64) - full).mean()
+        assert ea < 0.75 * es
+
+
 @pytest.mark.parametrize("bits", [3, 4, 8])
 def test_weight_only_equals_fake_quant_matmul(bits):
     X = synth.normal_f16((33, 70), 1.0, seed=21)

@@ -170,3 +170,50 @@ def test_act_absmax_and_scale():
     assert orc.act_absmax(X, skip_rows_mod=77) == np.float32(x[keep].max())
     assert orc.act_scale(np.float32(12.7), 8) == np.float32(12.7) / np.float32(127.0)
     assert orc.act_scale(np.float32(0.0), 8) == np.float32(1.0)
+
+
+# ------------------------------------------------------------------ asymmetric activations (Sec. 4.1)
+
+def test_asym_act_params_and_codes_vs_exact_rationals():
+    rng = np.random.default_rng(21)
+    for shift, spread in ((0.0, 1.0), (0.7, 0.5), (-2.0, 3.0), (5.0, 0.1)):
+        X = (rng.normal(shift, spread, (7, 96))).astype(np.float16)
+        scale, zero = orc.act_minmax_params(X)
+        x = X.astype(np.float64)
+        lo, hi = min(x.min(), 0.0), max(x.max(), 0.0)
+        assert scale == (np.float32(hi) - np.float32(lo)) / np.float32(255.0)
+        inv = Fraction(float(np.float32(1.0) / scale))
+        assert zero == max(0, min(255, _exact_code(Fraction(-lo), inv)))
+        c = orc.quantize_acts_asym(X, scale, zero)
+        for v, got in zip(X.ravel()[::5], c.ravel()[::5]):
+            q = max(0, min(255, _exact_code(Fraction(float(v)), inv) + zero))
+            assert int(got) == q - zero
+        # the range is used to its ends and zero is exactly representable
+        assert c.min() == -zero or lo == 0.0
+        assert c.max() == 255 - zero or hi == 0.0
+        assert orc.quantize_acts_asym(np.zeros(3, np.float16), scale, zero).tolist() == [0, 0, 0]
+        # |x_hat - x| <= s/2 (plus the slack of inv = fp32(1/s)) for values inside the range
+        xh = c.astype(np.float64) * float(scale)
+        assert np.all(np.abs(xh - x) <= float(scale) * (0.5 + 2.0 ** -20) + np.abs(x) * 2.0 ** -22 + float(scale) * 0.5 * (zero in (0, 255)))
+
+
+def test_asym_act_degenerate_and_clamp():
+    s, z = orc.act_minmax_params(np.zeros((4, 8), np.float16))
+    assert s == 1.0 and z == 0
+    X = np.array([0.0, 1.0, 2.0, 300.0, -300.0], np.float16)
+    c = orc.quantize_acts_asym(X, np.float32(1.0), 10)       # codes clamp to [0, 255] before centring
+    assert c.tolist() == [0, 1, 2, 245, -10]
+
+
+def test_asym_acts_gain_a_bit_on_one_sided_tensors():
+    # post-GELU-like input (almost no negative part): the asymmetric 8-bit grid covers [lo, hi] with 255
+    # steps where the symmetric one spends half of its 254 steps on values that do not occur
+    rng = np.random.default_rng(5)
+    X = np.maximum(rng.normal(0.0, 1.0, (64, 256)), -0.17).astype(np.float16)
+    x = X.astype(np.float64)
+    s, z = orc.act_minmax_params(X)
+    xa = orc.quantize_acts_asym(X, s, z).astype(np.float64) * float(s)
+    ss = orc.act_scale(orc.act_absmax(X), 8)
+    xs = orc.quantize_acts(X, ss, 8).astype(np.float64) * float(ss)
+    sq = lambda xh: 10 * np.log10((x ** 2).sum() / ((xh - x) ** 2).sum())
+    assert 4.5 < sq(xa) - sq(xs) < 7.5     # about one bit = 6 dB
