@@ -111,6 +111,24 @@ int mixdq_act_absmax(const void* X, int64_t rows, int64_t cols, int64_t row_stri
 int mixdq_act_scale_from_absmax(const float* amax, float* scale_out, void* stream);
 
 /*
+ * Range of an fp16 matrix [rows, cols] (row stride `row_stride` elements) with 0 included:
+ * minmax_out[0] = min(min x, 0), minmax_out[1] = max(max x, 0) (device fp32 [2]).  The first step of the
+ * asymmetric min-max activation quantizer (Sec. 4.1 "Quantization Scheme").
+ */
+int mixdq_act_minmax(const void* X, int64_t rows, int64_t cols, int64_t row_stride, float* minmax_out,
+                     void* stream);
+
+/* Asymmetric 8-bit parameters from that range, on the device: scale_out[0] = (hi - lo) / 255 (fp32),
+ * zero_out[0] = clamp(rne(-lo / scale), 0, 255) (int32); scale 1 and zero 0 when hi == lo. */
+int mixdq_act_asym_params_from_minmax(const float* minmax, float* scale_out, int32_t* zero_out,
+                                      void* stream);
+
+/* sums_out[n] = sum_k q[n, k] (device int32 [N]) of the signed codes of a MIXDQ_LAYOUT_DEVICE weight with
+ * bits in {4, 8}: computed once per layer, it carries the activation zero-point through the int8 GEMM. */
+int mixdq_weight_code_sums(const void* packed_W, int64_t N, int64_t K, int bits, int32_t* sums_out,
+                           void* stream);
+
+/*
  * Bytes of scratch memory the layer calls below need for a given problem (HOST `out`).
  * rows = output rows (tokens or output pixels), N, K as in the layer call.  The scratch
  * must be 256-byte aligned.  Nothing in it has to be initialised or to survive between calls
@@ -150,6 +168,28 @@ int mixdq_linear(const void* X, int64_t M, int64_t K, int64_t ldx, const void* p
 int mixdq_linear_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
                          int64_t N, int w_bits, const float* act_scale, int32_t* acc_out,
                          void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * W8A8 / W4A8 linear layer with ASYMMETRIC per-tensor activations, the quantizer the paper uses
+ * (Sec. 4.1 "Quantization Scheme": asymmetric min-max): unsigned codes q = clamp(rne(x / s) + z, 0, 255),
+ *   Y[m, n] = fp16( s * w_scale[n] * sum_k (q[m, k] - z) * qw[n, k] + bias[n] ).
+ * The tensor cores multiply the re-centred int8 codes q - 128; the term (128 - z) * w_code_sums[n]
+ * (mixdq_weight_code_sums) restores the zero-point in the epilogue.  act_scale (fp32) and act_zero (int32)
+ * are device scalars, e.g. from mixdq_act_asym_params_from_minmax.  Other arguments as in mixdq_linear.
+ * Unlike mixdq_linear this call NEEDS the workspace (mixdq_workspace_bytes(M, N, K, w_bits, 8)) and
+ * K % 16 == 0, ldx % 8 == 0, K <= 66000; it returns MIXDQ_ERR_UNSUPPORTED otherwise.  Linear layers only:
+ * a zero-padded convolution would need the code sums per filter tap at the image border.
+ */
+int mixdq_linear_a8_asym(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
+                         int w_bits, const float* w_scale, const int32_t* w_code_sums,
+                         const float* act_scale, const int32_t* act_zero, const void* bias, void* Y,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/* Parity hook: acc[M, N] = sum_k (q[m, k] - z) * qw[n, k] as int32. */
+int mixdq_linear_a8_asym_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
+                                 int64_t N, int w_bits, const int32_t* w_code_sums, const float* act_scale,
+                                 const int32_t* act_zero, int32_t* acc_out, void* workspace,
+                                 size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
  * Quantized 3x3 convolution as an implicit GEMM (all linear and conv layers are quantized,

@@ -28,7 +28,8 @@ bool fits_int(int64_t v) { return v > 0 && v <= 0x7fffffff; }
 int linear_impl(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
                 int w_bits, const float* w_scale, const int32_t* w_zero, int act_bits,
                 const float* act_scale, const void* bias, void* Y, int32_t* acc_out, void* workspace,
-                size_t ws_bytes, int32_t* status, void* stream)
+                size_t ws_bytes, int32_t* status, void* stream, const int32_t* act_zero = nullptr,
+                const int32_t* w_code_sums = nullptr)
 {
     if (!X || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
     if (!fits_int(M) || !fits_int(K) || !fits_int(N) || ldx < K) return MIXDQ_ERR_INVALID_ARG;
@@ -46,6 +47,8 @@ int linear_impl(const void* X, int64_t M, int64_t K, int64_t ldx, const void* pa
         p.N = static_cast<int>(N);
         p.K = static_cast<int>(K);
         p.act_scale = act_scale;
+        p.act_zero = act_zero;
+        p.w_code_sums = w_code_sums;
         p.w_scale = w_scale;
         p.bias = static_cast<const __half*>(bias);
         p.Y = static_cast<__half*>(Y);
@@ -221,6 +224,33 @@ extern "C" int mixdq_linear_acc_i32(const void* X, int64_t M, int64_t K, int64_t
     if (!acc_out) return MIXDQ_ERR_INVALID_ARG;
     return linear_impl(X, M, K, ldx, packed_W, N, w_bits, nullptr, nullptr, 8, act_scale, nullptr, nullptr,
                        acc_out, workspace, workspace_bytes, status, stream);
+}
+
+// |sum_k (q - z) qw| <= K * 255 * 127 must fit the int32 accumulator.
+static bool asym_args_ok(int64_t K, const float* act_scale, const int32_t* act_zero, const int32_t* w_code_sums)
+{
+    return act_scale && act_zero && w_code_sums && K * 255 * 127 <= 0x7fffffffll;
+}
+
+extern "C" int mixdq_linear_a8_asym(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
+                                    int64_t N, int w_bits, const float* w_scale, const int32_t* w_code_sums,
+                                    const float* act_scale, const int32_t* act_zero, const void* bias, void* Y,
+                                    void* workspace, size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!Y || !asym_args_ok(K, act_scale, act_zero, w_code_sums)) return MIXDQ_ERR_INVALID_ARG;
+    return linear_impl(X, M, K, ldx, packed_W, N, w_bits, w_scale, nullptr, 8, act_scale, bias, Y, nullptr,
+                       workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
+}
+
+extern "C" int mixdq_linear_a8_asym_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx,
+                                            const void* packed_W, int64_t N, int w_bits,
+                                            const int32_t* w_code_sums, const float* act_scale,
+                                            const int32_t* act_zero, int32_t* acc_out, void* workspace,
+                                            size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!acc_out || !asym_args_ok(K, act_scale, act_zero, w_code_sums)) return MIXDQ_ERR_INVALID_ARG;
+    return linear_impl(X, M, K, ldx, packed_W, N, w_bits, nullptr, nullptr, 8, act_scale, nullptr, nullptr,
+                       acc_out, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
 }
 
 extern "C" int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,

@@ -660,6 +660,11 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     const int64_t in_rows = amode == A_CONV3 ? static_cast<int64_t>(p.batch) * p.H * p.W : p.M;
     const int64_t row_len = amode == A_CONV3 ? p.Cin : p.K;
     const bool tma_room = workspace && ws_bytes >= split_bytes + tma_scratch_bytes(in_rows, row_len);
+    if (p.act_zero) {
+        // asymmetric activations exist in the two-kernel form only
+        if (amode != A_LINEAR || !p.w_code_sums || !tma_room || !tma_path_ok(p, amode, w_bits)) return MIXDQ_ERR_UNSUPPORTED;
+        return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
+    }
     if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1)
         return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
 

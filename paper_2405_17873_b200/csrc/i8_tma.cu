@@ -21,20 +21,24 @@ constexpr int BM = 128;
 constexpr int BK = 128;
 constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: fma(x, inv, magic) rounds x * inv to nearest even
 
-__device__ __forceinline__ uint32_t q4(float a, float b, float c, float d, float inv)
+// Four codes as bytes.  Symmetric: clamp(rne(x * inv), -127, 127).  Asymmetric (zoff = zero - 128):
+// clamp(rne(x * inv) + zero, 0, 255) - 128, the unsigned code moved into int8 range; the rounding is done
+// against the even magic constant before the offset is added, so that ties fall as they do without it.
+__device__ __forceinline__ uint32_t q4(float a, float b, float c, float d, float inv, float lo, float hi, uint32_t zoff)
 {
-    const float lo = kMagic - 127.f, hi = kMagic + 127.f;
-    const uint32_t qa = __float_as_uint(fminf(fmaxf(fmaf(a, inv, kMagic), lo), hi));
-    const uint32_t qb = __float_as_uint(fminf(fmaxf(fmaf(b, inv, kMagic), lo), hi));
-    const uint32_t qc = __float_as_uint(fminf(fmaxf(fmaf(c, inv, kMagic), lo), hi));
-    const uint32_t qd = __float_as_uint(fminf(fmaxf(fmaf(d, inv, kMagic), lo), hi));
+    const uint32_t qa = __float_as_uint(fminf(fmaxf(fmaf(a, inv, kMagic), lo), hi)) + zoff;
+    const uint32_t qb = __float_as_uint(fminf(fmaxf(fmaf(b, inv, kMagic), lo), hi)) + zoff;
+    const uint32_t qc = __float_as_uint(fminf(fmaxf(fmaf(c, inv, kMagic), lo), hi)) + zoff;
+    const uint32_t qd = __float_as_uint(fminf(fmaxf(fmaf(d, inv, kMagic), lo), hi)) + zoff;
     return __byte_perm(__byte_perm(qa, qb, 0x0040), __byte_perm(qc, qd, 0x0040), 0x5410);
 }
 
 // One thread per 16 consecutive elements of a row.  bos != 0: output row r reads input row
 // (r / 76) * 77 + r % 76 + 1, i.e. the BOS token of every prompt is left out.
+// act_zero != nullptr: asymmetric codes with that zero-point (see q4).
 __global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long long rows, int K, int bos,
-                             const float* __restrict__ act_scale, int8_t* __restrict__ out)
+                             const float* __restrict__ act_scale, const int32_t* __restrict__ act_zero,
+                             int8_t* __restrict__ out)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -49,6 +53,14 @@ __global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long l
         src_row = prompt * MIXDQ_TOKENS_PER_PROMPT + (r - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1)) + 1;
     }
     const float inv = __fdiv_rn(1.f, __ldg(act_scale));
+    float lo = kMagic - 127.f, hi = kMagic + 127.f;
+    uint32_t zoff = 0;
+    if (act_zero) {
+        const int z = __ldg(act_zero);
+        lo = kMagic - static_cast<float>(z);
+        hi = kMagic + static_cast<float>(255 - z);
+        zoff = static_cast<uint32_t>(z - 128);
+    }
     const uint4* src = reinterpret_cast<const uint4*>(X + src_row * ldx + c * 16);
     const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
     const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
@@ -60,10 +72,10 @@ __global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long l
         f[4 + j] = __half22float2(h1[j]);
     }
     uint4 o;
-    o.x = q4(f[0].x, f[0].y, f[1].x, f[1].y, inv);
-    o.y = q4(f[2].x, f[2].y, f[3].x, f[3].y, inv);
-    o.z = q4(f[4].x, f[4].y, f[5].x, f[5].y, inv);
-    o.w = q4(f[6].x, f[6].y, f[7].x, f[7].y, inv);
+    o.x = q4(f[0].x, f[0].y, f[1].x, f[1].y, inv, lo, hi, zoff);
+    o.y = q4(f[2].x, f[2].y, f[3].x, f[3].y, inv, lo, hi, zoff);
+    o.z = q4(f[4].x, f[4].y, f[5].x, f[5].y, inv, lo, hi, zoff);
+    o.w = q4(f[6].x, f[6].y, f[7].x, f[7].y, inv, lo, hi, zoff);
     *reinterpret_cast<uint4*>(out + r * K + c * 16) = o;
 }
 
@@ -97,6 +109,8 @@ struct TmaParams {
     int bos;      // output row m maps to row (m / 76) * 77 + m % 76 + 1 of Y
     int batch;
     const float* act_scale;
+    const int32_t* act_zero;     // asymmetric activations: zero-point (the int8 operand holds q - 128) ...
+    const int32_t* w_code_sums;  // ... and sum_k qw[n, k], so that sum_k (q - z) qw = acc + (128 - z) * sums[n]
     const float* w_scale;
     const __half* bias;
     const __half* bos_out;
@@ -664,12 +678,15 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             // while the main loop runs: per-column dequantization factors of this tile, and the
             // stored BOS rows
             const float sx = __ldg(p.act_scale);
+            const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
             for (int j = tid - 64; j < BN; j += 128) {
                 const int n = n0 + j;
                 float comb = 0.f, b = 0.f;
                 if (n < p.N && p.w_scale) {
                     comb = sx * __ldg(p.w_scale + n);
                     if (p.bias) b = __half2float(p.bias[n]);
+                    // the zero-point term is constant along a column: it rides in the bias
+                    if (p.act_zero) b = fmaf(static_cast<float>(zshift * __ldg(p.w_code_sums + n)), comb, b);
                 }
                 s_comb[j] = comb;
                 s_bias[j] = b;
@@ -785,8 +802,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 if (p.acc_out) {
                     int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
                     const int a[4] = {acc.x, acc.y, acc.z, acc.w};
+                    const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
                     for (int j = 0; j < 4; ++j)
-                        if (n + j < p.N) dst[j] = W4 ? (a[j] >> 4) : a[j];
+                        if (n + j < p.N)
+                            dst[j] = (W4 ? (a[j] >> 4) : a[j]) + (p.act_zero ? zshift * __ldg(p.w_code_sums + n + j) : 0);
                 }
                 if (p.Y) {
                     long long out_row = m;
@@ -950,6 +969,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         const int half = warp < 6 ? 0 : 1;
         const int et = tid - 64;  // epilogue warps only: 0..127
         const float sx = __ldg(p.act_scale);
+        const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
         bool ok = true;
         for (int t = 0; t < my_tiles; ++t) {
             const int tile = blockIdx.x + t * gridDim.x;
@@ -965,6 +985,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 if (n < p.N && p.w_scale) {
                     c = sx * __ldg(p.w_scale + n);
                     if (p.bias) b = __half2float(p.bias[n]);
+                    if (p.act_zero) b = fmaf(static_cast<float>(zshift * __ldg(p.w_code_sums + n)), c, b);
                 }
                 comb[j] = c;
                 bias[j] = b;
@@ -1017,7 +1038,9 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (n + j < p.N) dst[j] = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
+                        if (n + j < p.N)
+                            dst[j] = (W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j])) +
+                                     (p.act_zero ? zshift * __ldg(p.w_code_sums + n + j) : 0);
                 }
             }
             if (p.Y) {
@@ -1139,7 +1162,7 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     const long long ldx = conv ? p.Cin : p.ldx;
     const long long tasks = in_rows * (row_len / 16);
     int rc = launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
-                        p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, aq);
+                        p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, p.act_zero, aq);
     if (rc != MIXDQ_OK) return rc;
 
     // 2. tensor maps
@@ -1150,6 +1173,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     tp.bos = amode == A_BOS;
     tp.batch = p.batch;
     tp.act_scale = p.act_scale;
+    tp.act_zero = p.act_zero;
+    tp.w_code_sums = p.w_code_sums;
     tp.w_scale = p.w_scale;
     tp.bias = p.bias;
     tp.bos_out = p.bos_out;
@@ -1157,8 +1182,9 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     tp.ldy = p.ldy;
     tp.acc_out = p.acc_out;
     tp.status = p.status;
-    // bound of any accumulator: K products of at most 127 * 127 (W4, after the shift: 127 * 7)
-    tp.small_acc = static_cast<long long>(p.K) * 127 * (w4 ? 7 : 127) < (1ll << 22);
+    // bound of any accumulator: K products of at most 127 * 127 (W4, after the shift: 127 * 7); the
+    // re-centred codes of asymmetric activations reach -128
+    tp.small_acc = static_cast<long long>(p.K) * (p.act_zero ? 128 : 127) * (w4 ? 7 : 127) < (1ll << 22);
     // output tiles leave through TMA stores when Y's rows are 16-byte aligned and consecutive output
     // rows are consecutive rows of Y (not so for the cross-attention K/V layout, which skips row 0)
     tp.tma_store = p.Y && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;

@@ -135,15 +135,10 @@ __global__ void pack_kernel(const __half* __restrict__ W, int64_t N, int64_t K, 
     for (int b = 0; b < 4 && byte0 + b < pitch; ++b) row[byte0 + b] = (word >> (8 * b)) & 0xff;
 }
 
-// One thread per code.
-__global__ void unpack_kernel(const uint8_t* __restrict__ packed, int64_t N, int64_t K, int bits,
-                              int is_signed, int layout, int64_t pitch, int16_t* __restrict__ codes)
+// Code k of a packed row.
+__device__ __forceinline__ int decode_code(const uint8_t* __restrict__ row, int64_t k, int bits, int is_signed,
+                                           int layout)
 {
-    const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
-    if (idx >= N * K) return;
-    const int64_t n = idx / K;
-    const int64_t k = idx - n * K;
-    const uint8_t* row = packed + n * pitch;
     int c;
     if (bits == 8) {
         c = is_signed ? static_cast<int>(static_cast<int8_t>(row[k])) : static_cast<int>(row[k]);
@@ -178,7 +173,116 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ packed, int64_t N, int
             c |= ((row[byte] >> bit) & 1) << p;
         }
     }
-    codes[idx] = static_cast<int16_t>(c);
+    return c;
+}
+
+// One thread per code.
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, int64_t N, int64_t K, int bits,
+                              int is_signed, int layout, int64_t pitch, int16_t* __restrict__ codes)
+{
+    const int64_t idx = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (idx >= N * K) return;
+    const int64_t n = idx / K;
+    const int64_t k = idx - n * K;
+    codes[idx] = static_cast<int16_t>(decode_code(packed + n * pitch, k, bits, is_signed, layout));
+}
+
+// One CTA of 128 threads per output channel: sum over k of its signed codes.
+__global__ void code_sums_kernel(const uint8_t* __restrict__ packed, int64_t K, int bits, int64_t pitch,
+                                 int32_t* __restrict__ sums)
+{
+    __shared__ int part[4];
+    const uint8_t* row = packed + blockIdx.x * pitch;
+    int s = 0;
+    for (int64_t k = threadIdx.x; k < K; k += blockDim.x) s += decode_code(row, k, bits, 1, MIXDQ_LAYOUT_DEVICE);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) sums[blockIdx.x] = part[0] + part[1] + part[2] + part[3];
+}
+
+// Range of a tensor with 0 included: floats ordered through a monotone map to unsigned integers.
+__device__ __forceinline__ unsigned int ordered_bits(float f)
+{
+    const unsigned int u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// range_bits[0]: ordered bits of the running minimum, [1]: of the running maximum.
+__global__ void minmax_kernel(const __half* __restrict__ X, int64_t rows, int64_t cols, int64_t row_stride,
+                              unsigned int* __restrict__ range_bits)
+{
+    float lo = 0.f, hi = 0.f;
+    const int64_t chunks_per_row = (cols + 7) / 8;
+    const int64_t total = rows * chunks_per_row;
+    const bool vec_ok = (cols % 8 == 0) && (row_stride % 8 == 0) &&
+                        ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / chunks_per_row;
+        const int64_t c = (i - r * chunks_per_row) * 8;
+        const __half* p = X + r * row_stride + c;
+        if (vec_ok) {
+            const uint4 v = *reinterpret_cast<const uint4*>(p);
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __half22float2(h[j]);
+                lo = fminf(lo, fminf(f.x, f.y));
+                hi = fmaxf(hi, fmaxf(f.x, f.y));
+            }
+        } else {
+            for (int j = 0; j < 8 && c + j < cols; ++j) {
+                const float f = __half2float(p[j]);
+                lo = fminf(lo, f);
+                hi = fmaxf(hi, f);
+            }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (lo < 0.f) atomicMin(range_bits, ordered_bits(lo));
+        if (hi > 0.f) atomicMax(range_bits + 1, ordered_bits(hi));
+    }
+}
+
+// Both accumulators start at the ordered bits of +0.
+__global__ void minmax_init_kernel(unsigned int* __restrict__ range_bits)
+{
+    range_bits[0] = 0x80000000u;
+    range_bits[1] = 0x80000000u;
+}
+
+// Ordered bits back to the bit patterns of {lo, hi}.
+__global__ void minmax_finish_kernel(unsigned int* __restrict__ range_bits)
+{
+    for (int i = 0; i < 2; ++i) {
+        const unsigned int o = range_bits[i];
+        range_bits[i] = (o & 0x80000000u) ? (o & 0x7fffffffu) : ~o;
+    }
+}
+
+// scale = (hi - lo) / 255, zero = clamp(rne(-lo / scale), 0, 255); an all-zero tensor: scale 1, zero 0.
+__global__ void act_asym_params_kernel(const float* __restrict__ minmax, float* __restrict__ scale_out,
+                                       int32_t* __restrict__ zero_out)
+{
+    const float lo = minmax[0], hi = minmax[1];
+    if (hi == lo) {
+        scale_out[0] = 1.f;
+        zero_out[0] = 0;
+        return;
+    }
+    const float s = __fdiv_rn(__fsub_rn(hi, lo), 255.f);
+    const float inv = __fdiv_rn(1.f, s);
+    // -lo * inv <= 255 * (1 + 2^-22): the magic-number addition rounds the exact product to nearest even
+    const float t = __fmaf_rn(-lo, inv, 12582912.f);
+    int z = static_cast<int>(__float_as_uint(t)) - 0x4B400000;
+    z = z < 0 ? 0 : (z > 255 ? 255 : z);
+    scale_out[0] = s;
+    zero_out[0] = z;
 }
 
 // max |x| as an atomic max on the bit pattern (non-negative floats order like integers).
@@ -298,5 +402,42 @@ extern "C" int mixdq_act_scale_from_absmax(const float* amax, float* scale_out, 
 {
     if (!amax || !scale_out) return MIXDQ_ERR_INVALID_ARG;
     act_scale_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(amax, scale_out);
+    return check_launch();
+}
+
+extern "C" int mixdq_act_minmax(const void* X, int64_t rows, int64_t cols, int64_t row_stride,
+                                float* minmax_out, void* stream)
+{
+    if (!X || !minmax_out || rows <= 0 || cols <= 0 || row_stride < cols) return MIXDQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int* bits = reinterpret_cast<unsigned int*>(minmax_out);
+    minmax_init_kernel<<<1, 1, 0, st>>>(bits);
+    int rc = check_launch();
+    if (rc != MIXDQ_OK) return rc;
+    const int64_t chunks = rows * ((cols + 7) / 8);
+    const unsigned grid = static_cast<unsigned>(chunks < 256 * 1184 ? ceil_div(chunks, 256) : 1184);
+    minmax_kernel<<<grid, 256, 0, st>>>(static_cast<const __half*>(X), rows, cols, row_stride, bits);
+    rc = check_launch();
+    if (rc != MIXDQ_OK) return rc;
+    minmax_finish_kernel<<<1, 1, 0, st>>>(bits);
+    return check_launch();
+}
+
+extern "C" int mixdq_act_asym_params_from_minmax(const float* minmax, float* scale_out, int32_t* zero_out,
+                                                 void* stream)
+{
+    if (!minmax || !scale_out || !zero_out) return MIXDQ_ERR_INVALID_ARG;
+    act_asym_params_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(minmax, scale_out, zero_out);
+    return check_launch();
+}
+
+extern "C" int mixdq_weight_code_sums(const void* packed_W, int64_t N, int64_t K, int bits, int32_t* sums_out,
+                                      void* stream)
+{
+    if (!packed_W || !sums_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
+    if (bits != 4 && bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    const int64_t pitch = row_pitch_bytes(K, bits, MIXDQ_LAYOUT_DEVICE);
+    code_sums_kernel<<<static_cast<unsigned>(N), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(packed_W), K, bits, pitch, sums_out);
     return check_launch();
 }

@@ -31,6 +31,13 @@ _SIGNATURES = {
     "mixdq_unpack_weights": (_int, [_vp, _i64, _i64, _int, _int, _int, _vp, _vp]),
     "mixdq_act_absmax": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp]),
     "mixdq_act_scale_from_absmax": (_int, [_vp, _vp, _vp]),
+    "mixdq_act_minmax": (_int, [_vp, _i64, _i64, _i64, _vp, _vp]),
+    "mixdq_act_asym_params_from_minmax": (_int, [_vp, _vp, _vp, _vp]),
+    "mixdq_weight_code_sums": (_int, [_vp, _i64, _i64, _int, _vp, _vp]),
+    "mixdq_linear_a8_asym": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                    _sz, _vp, _vp]),
+    "mixdq_linear_a8_asym_acc_i32": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp,
+                                            _sz, _vp, _vp]),
     "mixdq_workspace_bytes": (_int, [_i64, _i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_conv3x3_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, _int, _int, _int, C.POINTER(_sz)]),
     "mixdq_linear": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp, _sz,
@@ -170,6 +177,31 @@ def act_scale(X: torch.Tensor, skip_rows_mod: int = 0) -> torch.Tensor:
     return act_scale_from_absmax(act_absmax(X, skip_rows_mod))
 
 
+def act_minmax(X: torch.Tensor) -> torch.Tensor:
+    """Device fp32 [2]: min(min x, 0), max(max x, 0)."""
+    X2 = X.reshape(-1, X.shape[-1])
+    out = torch.empty(2, dtype=torch.float32, device=X.device)
+    _chk(lib().mixdq_act_minmax(_ptr(X2), X2.shape[0], X2.shape[1], X2.stride(0), _ptr(out), _stream()),
+         "mixdq_act_minmax")
+    return out
+
+
+def act_asym_params(X: torch.Tensor):
+    """Asymmetric 8-bit activation parameters (device fp32 scale [1], device int32 zero-point [1])."""
+    mm = act_minmax(X)
+    scale = torch.empty(1, dtype=torch.float32, device=X.device)
+    zero = torch.empty(1, dtype=torch.int32, device=X.device)
+    _chk(lib().mixdq_act_asym_params_from_minmax(_ptr(mm), _ptr(scale), _ptr(zero), _stream()),
+         "mixdq_act_asym_params_from_minmax")
+    return scale, zero
+
+
+def weight_code_sums(packed_W: torch.Tensor, N: int, K: int, bits: int) -> torch.Tensor:
+    out = torch.empty(N, dtype=torch.int32, device=packed_W.device)
+    _chk(lib().mixdq_weight_code_sums(_ptr(packed_W), N, K, bits, _ptr(out), _stream()), "mixdq_weight_code_sums")
+    return out
+
+
 def _ws(workspace):
     return (_ptr(workspace), workspace.numel() if workspace is not None else 0)
 
@@ -191,6 +223,28 @@ def linear_acc_i32(X, packed_W, N: int, w_bits: int, act_scale, workspace=None, 
     wp, wb = _ws(workspace)
     _chk(lib().mixdq_linear_acc_i32(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits, _ptr(act_scale),
                                     _ptr(acc), wp, wb, _ptr(status), _stream()), "mixdq_linear_acc_i32")
+    return acc
+
+
+def linear_a8_asym(X, packed_W, N: int, w_bits: int, w_scale, w_code_sums, act_scale, act_zero, bias=None,
+                   workspace=None, status=None, out=None):
+    M, K = X.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear_a8_asym(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits, _ptr(w_scale),
+                                    _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(bias), _ptr(Y),
+                                    wp, wb, _ptr(status), _stream()), "mixdq_linear_a8_asym")
+    return Y
+
+
+def linear_a8_asym_acc_i32(X, packed_W, N: int, w_bits: int, w_code_sums, act_scale, act_zero, workspace=None,
+                           status=None):
+    M, K = X.shape
+    acc = torch.empty((M, N), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear_a8_asym_acc_i32(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits,
+                                            _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(acc), wp,
+                                            wb, _ptr(status), _stream()), "mixdq_linear_a8_asym_acc_i32")
     return acc
 
 

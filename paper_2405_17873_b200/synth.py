@@ -79,6 +79,13 @@ def geglu(h: np.ndarray) -> np.ndarray:
     return (v * torch.nn.functional.gelu(gate)).to(torch.float16).numpy()
 
 
+def one_sided_f16(shape, seed: int, shift: float = 0.0, gain: float = 1.0) -> np.ndarray:
+    """gain * GELU(N(shift, 1)): the skewed value range (a short negative tail near -0.17 * gain, a long
+    positive one) of a tensor that follows a GELU / SiLU, where an asymmetric grid pays (Sec. 4.1)."""
+    t = torch.randn(*shape, generator=_gen(seed)) + shift
+    return (gain * torch.nn.functional.gelu(t)).to(torch.float16).numpy()
+
+
 def text_embedding(B: int, seed: int = 4000, n_outlier_ch: int = 8, outlier_mag: float = 50.0):
     """Text embedding [B,77,2048] ~ N(0,1); token 0 is one seeded row shared by every prompt
     with a few fixed channels at +-outlier_mag."""
