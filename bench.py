@@ -41,6 +41,9 @@ def parse():
     ap.add_argument("--tokens", type=int, default=0,
                     help="weight-bound regime: only the linear layers of the a16 table, each on this many rows "
                          "(e.g. 16); reports the weight stream in GB/s against the HBM roofline")
+    ap.add_argument("--act-asym", action="store_true",
+                    help="w4a8 table: asymmetric 8-bit activations on the plain linear layers (Sec. 4.1); the "
+                         "default run, which the headline number is quoted on, uses symmetric ones everywhere")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -49,7 +52,7 @@ def parse():
 def workload_name(args):
     if args.tokens > 0:
         return f"unet_linear_sweep_{args.table}_{args.tokens}tokens"
-    return f"unet_sweep_sdxl512_{args.table}_b{args.batch}"
+    return f"unet_sweep_sdxl512_{args.table}_b{args.batch}" + ("_asym_linear_acts" if args.act_asym else "")
 
 
 # ----------------------------------------------------------------------------- peaks
@@ -254,7 +257,7 @@ def run_ours(args):
 
     if args.tokens > 0 and args.table != "a16":
         raise SystemExit("--tokens needs --table a16 (the weight-only engine)")
-    sweep = UNetSweep(args.batch, args.table, seed=5 + rank, tokens=args.tokens)
+    sweep = UNetSweep(args.batch, args.table, seed=5 + rank, tokens=args.tokens, act_asym=args.act_asym)
     tc_layers = [pl for pl in sweep.layers if sweep.uses_tensor_int8(pl)]
     other_layers = [pl for pl in sweep.layers if not sweep.uses_tensor_int8(pl)]
     if args.table == "a16":
@@ -392,7 +395,7 @@ def run_ours(args):
         # DRAM bytes per step of these kernels from one ncu capture of this command at batch 4 (caches flushed
         # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.00 GB read by the quantization
         # passes (every layer's input once) + 2.96 GB by the GEMMs (weights and int8 activations once)
-        traffic = 5.97e9 if (args.batch == 4 and world == 1) else None
+        traffic = 5.97e9 if (args.batch == 4 and world == 1 and not args.act_asym) else None
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
                     "traffic": traffic,
                     "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
@@ -442,7 +445,7 @@ def run_ours(args):
             "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
             "device_status": status,
         }
-        if world == 1 and not args.no_cpu_baseline and args.tokens == 0:
+        if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym:
             out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
         print(json.dumps(out))
     if world > 1:

@@ -26,15 +26,19 @@ class PackedLayer:
     bos_out: Optional[torch.Tensor]
     x_key: tuple
     y_key: tuple
+    code_sums: Optional[torch.Tensor] = None   # asymmetric activations: per-channel sums of the weight codes
 
 
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
-                 layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0):
+                 layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
-        (whatever the image size), so that a layer is one stream over its packed weights."""
+        (whatever the image size), so that a layer is one stream over its packed weights.
+        act_asym: the 8-bit activations of the plain linear layers are asymmetric (Sec. 4.1); convolutions
+        and the BOS-aware K/V projections keep symmetric ones."""
         assert table in ("w4a8", "a16")
         self.batch = batch
+        self.act_asym = act_asym
         self.tokens = tokens
         self.table = table
         self.device = device
@@ -49,6 +53,7 @@ class UNetSweep:
         self.x: Dict[tuple, torch.Tensor] = {}
         self.y: Dict[tuple, torch.Tensor] = {}
         self.x_scale: Dict[tuple, torch.Tensor] = {}
+        self.x_asym: Dict[tuple, tuple] = {}
         self.layers: List[PackedLayer] = []
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self._build(seed)
@@ -100,7 +105,12 @@ class UNetSweep:
                 if l.a_bits == 8:
                     e0 = self.x[xk][0, 0].to(torch.float32)
                     bos = (W.to(torch.float32) @ e0).to(torch.float16).contiguous()
-            self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk))
+            sums = None
+            if self.act_asym and l.kind == "linear" and l.a_bits == 8:
+                sums = mixdq.weight_code_sums(packed, l.N, l.K, l.w_bits)
+                if xk not in self.x_asym:
+                    self.x_asym[xk] = mixdq.act_asym_params(self.x[xk].reshape(-1, xk[-1]))
+            self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk, sums))
             if l.kind == "conv3x3":
                 need = mixdq.conv3x3_workspace_bytes(self.batch, l.H, l.H, l.Cin, l.N, l.stride, l.w_bits, l.a_bits)
             else:
@@ -125,6 +135,10 @@ class UNetSweep:
             return mixdq.crossattn_kv(x, pl.packed, l.N, l.w_bits, pl.w_scale, sx, pl.bos_out, ws, self.status,
                                       out=y)
         x2 = x.reshape(-1, x.shape[-1])
+        if pl.code_sums is not None:
+            ax, az = self.x_asym[pl.x_key]
+            return mixdq.linear_a8_asym(x2, pl.packed, l.N, l.w_bits, pl.w_scale, pl.code_sums, ax, az, pl.bias, ws,
+                                        self.status, out=y.reshape(-1, l.N))
         return mixdq.linear(x2, pl.packed, l.N, l.w_bits, pl.w_scale, pl.w_zero, l.a_bits, sx, pl.bias, ws,
                             self.status, out=y.reshape(-1, l.N))
 
@@ -175,6 +189,7 @@ def _main(argv=None) -> int:
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--tokens", type=int, default=0, help="linear layers only: run on this many rows (weight-bound regime)")
+    ap.add_argument("--act-asym", action="store_true", help="asymmetric 8-bit activations (plain linear layers)")
     ap.add_argument("--eager", action="store_true", help="plain launches only, no graph and no timing")
     a = ap.parse_args(argv)
 
@@ -185,7 +200,7 @@ def _main(argv=None) -> int:
         raise SystemExit(f"no layer named {a.layer!r}")
     if a.w_bits is not None:
         pick[0].w_bits = a.w_bits
-    sw = UNetSweep(a.batch, a.table, layers=pick, tokens=a.tokens)
+    sw = UNetSweep(a.batch, a.table, layers=pick, tokens=a.tokens, act_asym=a.act_asym)
     pl = sw.layers[0]
     for _ in range(a.reps):
         sw.run_layer(pl)
