@@ -461,6 +461,41 @@ int orc_int_conv3x3(const int8_t *qx, const int16_t *qw, int64_t B, int64_t H, i
     return overflow ? ORC_ERR_OVERFLOW : ORC_OK;
 }
 
+/* The same direct convolution on centred codes of asymmetrically quantized activations (q - z, int16):
+ * a padded position holds the real value 0, whose code is z, so it contributes (z - z) * w = 0 and is
+ * skipped exactly as above. */
+int orc_int_conv3x3_i16(const int16_t *cx, const int16_t *qw, int64_t B, int64_t H, int64_t W, int64_t C,
+                        int64_t N, int stride, int32_t *acc_out)
+{
+    if (!cx || !qw || !acc_out || (stride != 1 && stride != 2)) return ORC_ERR_ARG;
+    int64_t Ho = (H + 2 - 3) / stride + 1, Wo = (W + 2 - 3) / stride + 1;
+    int overflow = 0;
+#pragma omp parallel for collapse(2) schedule(static) reduction(| : overflow)
+    for (int64_t b = 0; b < B; ++b) {
+        for (int64_t ho = 0; ho < Ho; ++ho) {
+            for (int64_t wo = 0; wo < Wo; ++wo) {
+                for (int64_t n = 0; n < N; ++n) {
+                    int64_t acc = 0;
+                    for (int kh = 0; kh < 3; ++kh) {
+                        int64_t hi = ho * stride + kh - 1;
+                        if (hi < 0 || hi >= H) continue;
+                        for (int kw = 0; kw < 3; ++kw) {
+                            int64_t wi = wo * stride + kw - 1;
+                            if (wi < 0 || wi >= W) continue;
+                            const int16_t *xp = cx + ((b * H + hi) * W + wi) * C;
+                            const int16_t *wp = qw + ((n * 3 + kh) * 3 + kw) * C;
+                            for (int64_t c = 0; c < C; ++c) acc += (int64_t)xp[c] * (int64_t)wp[c];
+                        }
+                    }
+                    if (acc > INT32_MAX || acc < INT32_MIN) overflow = 1;
+                    acc_out[((b * Ho + ho) * Wo + wo) * N + n] = (int32_t)acc;
+                }
+            }
+        }
+    }
+    return overflow ? ORC_ERR_OVERFLOW : ORC_OK;
+}
+
 /* Dequantize + bias: y = fp16( acc * s_x * s_w[n] + bias[n] ), in double. */
 int orc_dequant_epilogue(const int32_t *acc, int64_t M, int64_t N, float act_scale,
                          const float *w_scale, const uint16_t *bias, uint16_t *Y)

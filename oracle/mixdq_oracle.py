@@ -223,6 +223,20 @@ def int_conv3x3(qx, qw, stride: int = 1):
     return acc
 
 
+def int_conv3x3_i16(cx, qw, stride: int = 1):
+    """cx int16 NHWC [B,H,W,C] (centred codes q - z); qw int16 [N,3,3,C] -> int32 [B,Ho,Wo,N]."""
+    cx = np.ascontiguousarray(cx, np.int16)
+    qw = np.ascontiguousarray(qw, np.int16)
+    B, H, W, Cin = cx.shape
+    N = qw.shape[0]
+    assert qw.shape == (N, 3, 3, Cin)
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    acc = np.empty((B, Ho, Wo, N), np.int32)
+    _chk(lib().orc_int_conv3x3_i16(_p(cx), _p(qw), C.c_int64(B), C.c_int64(H), C.c_int64(W),
+                                   C.c_int64(Cin), C.c_int64(N), stride, _p(acc)), "int_conv3x3_i16")
+    return acc
+
+
 def dequant_epilogue(acc, act_scale_, w_scale, bias=None):
     acc = np.ascontiguousarray(acc, np.int32)
     N = acc.shape[-1]
@@ -304,6 +318,15 @@ def conv3x3_a8(X, codes, w_scale, act_scale_, bias=None, stride: int = 1):
     X = _f16(X)
     qx = quantize_acts(X, act_scale_, 8)
     acc = int_conv3x3(qx, codes, stride)
+    return acc, dequant_epilogue(acc, act_scale_, w_scale, bias)
+
+
+def conv3x3_a8_asym(X, codes, w_scale, act_scale_, act_zero: int, bias=None, stride: int = 1):
+    """3x3 convolution with asymmetric per-tensor activations (Sec. 4.1): X fp16 NHWC, codes int16
+    [N,3,3,C]; the zero padding is the real value 0, i.e. code z.  Returns (int32 acc, fp16 out), NHWC."""
+    X = _f16(X)
+    cx = quantize_acts_asym(X, act_scale_, act_zero)
+    acc = int_conv3x3_i16(cx, codes, stride)
     return acc, dequant_epilogue(acc, act_scale_, w_scale, bias)
 
 

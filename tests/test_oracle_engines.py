@@ -188,6 +188,51 @@ def test_int_conv_tap_counts_and_centre_kernel():
     assert np.array_equal(a2, a1[:, ::2, ::2, :])
 
 
+@pytest.mark.parametrize("stride", [1, 2])
+def test_int_conv_i16_padding_is_the_zero_point(stride):
+    # Explicitly padding the UNSIGNED codes with z and running a border-free brute force over the padded
+    # image gives the same sums: the padded ring is the real value 0.  (Padding with code 0 would not.)
+    rng = np.random.default_rng(17 + stride)
+    B, H, W, Cc, N, z = 2, 6, 4, 3, 2, 93
+    q = rng.integers(0, 256, size=(B, H, W, Cc))
+    qw = rng.integers(-127, 128, size=(N, 3, 3, Cc)).astype(np.int16)
+    acc = orc.int_conv3x3_i16((q - z).astype(np.int16), qw, stride)
+    qp = np.full((B, H + 2, W + 2, Cc), z, np.int64)
+    qp[:, 1:-1, 1:-1, :] = q
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    assert acc.shape == (B, Ho, Wo, N)
+    for b in range(B):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                win = qp[b, ho * stride:ho * stride + 3, wo * stride:wo * stride + 3, :] - z
+                for n in range(N):
+                    assert int(acc[b, ho, wo, n]) == int((win * qw[n].astype(np.int64)).sum())
+    # on codes that fit int8 it is the int8 engine
+    c8 = rng.integers(-127, 128, size=(B, H, W, Cc)).astype(np.int8)
+    assert np.array_equal(orc.int_conv3x3_i16(c8.astype(np.int16), qw, stride), orc.int_conv3x3(c8, qw, stride))
+
+
+def test_a8_asym_conv_equals_linear_on_im2col():
+    rng = np.random.default_rng(23)
+    X = synth.one_sided_f16((2, 5, 6, 8), seed=31)
+    W = synth.normal_f16((12, 72), 0.05, seed=32)
+    b = synth.normal_f16((12,), 0.1, seed=33)
+    ws, _ = orc.weight_minmax_params(W, 8, True)
+    codes = orc.quantize_weights(W, 8, ws, None)
+    sx, zx = orc.act_minmax_params(X)
+    for stride in (1, 2):
+        acc, y = orc.conv3x3_a8_asym(X, codes.reshape(12, 3, 3, 8), ws, sx, zx, b, stride)
+        # im2col of the fp16 image (zero padding = real zeros) through the linear layer of the same scheme
+        Xp = np.zeros((2, 7, 8, 8), np.float16)
+        Xp[:, 1:-1, 1:-1, :] = X
+        Ho, Wo = acc.shape[1:3]
+        cols = np.stack([Xp[:, ho * stride:ho * stride + 3, wo * stride:wo * stride + 3, :].reshape(2, 72)
+                         for ho in range(Ho) for wo in range(Wo)], axis=1).reshape(-1, 72)
+        acc_l, y_l = orc.linear_a8_asym(cols, codes, ws, sx, zx, b)
+        assert np.array_equal(acc.reshape(-1, 12), acc_l)
+        assert np.array_equal(y.reshape(-1, 12).view(np.uint16), y_l.view(np.uint16))
+
+
 # ------------------------------------------------ epilogue and layer identities
 
 def _tol(y_ref):
