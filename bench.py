@@ -42,7 +42,7 @@ def parse():
                     help="weight-bound regime: only the linear layers of the a16 table, each on this many rows "
                          "(e.g. 16); reports the weight stream in GB/s against the HBM roofline")
     ap.add_argument("--act-asym", action="store_true",
-                    help="w4a8 table: asymmetric 8-bit activations on the plain linear layers (Sec. 4.1); the "
+                    help="w4a8 table: asymmetric 8-bit activations on linear layers and 3x3 convolutions (Sec. 4.1); the "
                          "default run, which the headline number is quoted on, uses symmetric ones everywhere")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -52,7 +52,7 @@ def parse():
 def workload_name(args):
     if args.tokens > 0:
         return f"unet_linear_sweep_{args.table}_{args.tokens}tokens"
-    return f"unet_sweep_sdxl512_{args.table}_b{args.batch}" + ("_asym_linear_acts" if args.act_asym else "")
+    return f"unet_sweep_sdxl512_{args.table}_b{args.batch}" + ("_asym_acts" if args.act_asym else "")
 
 
 # ----------------------------------------------------------------------------- peaks

@@ -177,8 +177,7 @@ int mixdq_linear_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, const
  * (mixdq_weight_code_sums) restores the zero-point in the epilogue.  act_scale (fp32) and act_zero (int32)
  * are device scalars, e.g. from mixdq_act_asym_params_from_minmax.  Other arguments as in mixdq_linear.
  * Unlike mixdq_linear this call NEEDS the workspace (mixdq_workspace_bytes(M, N, K, w_bits, 8)) and
- * K % 16 == 0, ldx % 8 == 0, K <= 66000; it returns MIXDQ_ERR_UNSUPPORTED otherwise.  Linear layers only:
- * a zero-padded convolution would need the code sums per filter tap at the image border.
+ * K % 16 == 0, ldx % 8 == 0, K <= 66000; it returns MIXDQ_ERR_UNSUPPORTED otherwise.
  */
 int mixdq_linear_a8_asym(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
                          int w_bits, const float* w_scale, const int32_t* w_code_sums,
@@ -201,6 +200,27 @@ int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, c
                   int64_t Cout, int stride, int w_bits, const float* w_scale, const int32_t* w_zero,
                   int act_bits, const float* act_scale, const void* bias, void* Y, void* workspace,
                   size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * The 3x3 convolution with asymmetric per-tensor activations (as mixdq_linear_a8_asym; Sec. 4.1).  The zero
+ * padding is the real value 0, whose code is the zero-point: the call keeps the int8 image in the workspace
+ * with a one-pixel border of that code, so border outputs need no special case.  w_code_sums =
+ * mixdq_weight_code_sums(packed_W, Cout, 9 * Cin, w_bits).  NEEDS the workspace
+ * (mixdq_conv3x3_workspace_bytes) and a geometry the two-kernel path takes (Cin % 32 == 0; Wo a multiple of
+ * 128, or 128 / Wo a divisor or a multiple of Ho; stride 2 only on even H, W): MIXDQ_ERR_UNSUPPORTED otherwise.
+ */
+int mixdq_conv3x3_a8_asym(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                          int64_t Cout, int stride, int w_bits, const float* w_scale,
+                          const int32_t* w_code_sums, const float* act_scale, const int32_t* act_zero,
+                          const void* bias, void* Y, void* workspace, size_t workspace_bytes, int32_t* status,
+                          void* stream);
+
+/* Parity hook: acc[B, Ho, Wo, Cout] = sum over the window of (q - z) * qw as int32. */
+int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                                  const void* packed_W, int64_t Cout, int stride, int w_bits,
+                                  const int32_t* w_code_sums, const float* act_scale, const int32_t* act_zero,
+                                  int32_t* acc_out, void* workspace, size_t workspace_bytes, int32_t* status,
+                                  void* stream);
 
 /* Parity hook: int32 accumulators [B, Ho, Wo, Cout] of the int8 conv path. */
 int mixdq_conv3x3_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,

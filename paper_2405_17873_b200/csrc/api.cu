@@ -76,7 +76,8 @@ int linear_impl(const void* X, int64_t M, int64_t K, int64_t ldx, const void* pa
 int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
                int64_t Cout, int stride, int w_bits, const float* w_scale, const int32_t* w_zero,
                int act_bits, const float* act_scale, const void* bias, void* Y, int32_t* acc_out,
-               void* workspace, size_t ws_bytes, int32_t* status, void* stream)
+               void* workspace, size_t ws_bytes, int32_t* status, void* stream,
+               const int32_t* act_zero = nullptr, const int32_t* w_code_sums = nullptr)
 {
     if (!X || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
     if (!fits_int(B) || !fits_int(H) || !fits_int(W) || !fits_int(Cin) || !fits_int(Cout))
@@ -105,6 +106,8 @@ int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, cons
         p.stride = stride;
         p.batch = static_cast<int>(B);
         p.act_scale = act_scale;
+        p.act_zero = act_zero;
+        p.w_code_sums = w_code_sums;
         p.w_scale = w_scale;
         p.bias = static_cast<const __half*>(bias);
         p.Y = static_cast<__half*>(Y);
@@ -203,7 +206,8 @@ extern "C" int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, in
     if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
     if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
-    *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * H * W, Cin) : 0;
+    // room for the int8 image with a one-pixel border, which the asymmetric-activation call keeps
+    *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * (H + 2) * (W + 2), Cin) : 0;
     return MIXDQ_OK;
 }
 
@@ -251,6 +255,28 @@ extern "C" int mixdq_linear_a8_asym_acc_i32(const void* X, int64_t M, int64_t K,
     if (!acc_out || !asym_args_ok(K, act_scale, act_zero, w_code_sums)) return MIXDQ_ERR_INVALID_ARG;
     return linear_impl(X, M, K, ldx, packed_W, N, w_bits, nullptr, nullptr, 8, act_scale, nullptr, nullptr,
                        acc_out, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
+}
+
+extern "C" int mixdq_conv3x3_a8_asym(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                                     const void* packed_W, int64_t Cout, int stride, int w_bits,
+                                     const float* w_scale, const int32_t* w_code_sums, const float* act_scale,
+                                     const int32_t* act_zero, const void* bias, void* Y, void* workspace,
+                                     size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!Y || !asym_args_ok(9 * Cin, act_scale, act_zero, w_code_sums)) return MIXDQ_ERR_INVALID_ARG;
+    return conv3_impl(X, B, H, W, Cin, packed_W, Cout, stride, w_bits, w_scale, nullptr, 8, act_scale, bias, Y,
+                      nullptr, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
+}
+
+extern "C" int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                                             const void* packed_W, int64_t Cout, int stride, int w_bits,
+                                             const int32_t* w_code_sums, const float* act_scale,
+                                             const int32_t* act_zero, int32_t* acc_out, void* workspace,
+                                             size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!acc_out || !asym_args_ok(9 * Cin, act_scale, act_zero, w_code_sums)) return MIXDQ_ERR_INVALID_ARG;
+    return conv3_impl(X, B, H, W, Cin, packed_W, Cout, stride, w_bits, nullptr, nullptr, 8, act_scale, nullptr,
+                      nullptr, acc_out, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
 }
 
 extern "C" int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,

@@ -24,7 +24,7 @@ struct Params {
     int H = 0, W = 0, Cin = 0, Ho = 0, Wo = 0, stride = 1;  // conv geometry
     int batch = 0;                                          // prompts (BOS mode)
     const float* act_scale = nullptr;
-    // asymmetric activations (two-kernel path, linear rows only): zero-point and per-channel sums of
+    // asymmetric activations (two-kernel path; not the BOS-aware projection): zero-point and per-channel sums of
     // the weight codes; both nullptr for symmetric activations
     const int32_t* act_zero = nullptr;
     const int32_t* w_code_sums = nullptr;

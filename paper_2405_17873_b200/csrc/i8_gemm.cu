@@ -657,12 +657,14 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
 
     // two-kernel path: needs room for the int8 activations behind the split-reduction scratch
     const size_t split_bytes = split_scratch_bytes(p.M, p.N);
-    const int64_t in_rows = amode == A_CONV3 ? static_cast<int64_t>(p.batch) * p.H * p.W : p.M;
+    // an asymmetric convolution input is kept with its one-pixel border
+    const int pad = (amode == A_CONV3 && p.act_zero) ? 2 : 0;
+    const int64_t in_rows = amode == A_CONV3 ? static_cast<int64_t>(p.batch) * (p.H + pad) * (p.W + pad) : p.M;
     const int64_t row_len = amode == A_CONV3 ? p.Cin : p.K;
     const bool tma_room = workspace && ws_bytes >= split_bytes + tma_scratch_bytes(in_rows, row_len);
     if (p.act_zero) {
         // asymmetric activations exist in the two-kernel form only
-        if (amode != A_LINEAR || !p.w_code_sums || !tma_room || !tma_path_ok(p, amode, w_bits)) return MIXDQ_ERR_UNSUPPORTED;
+        if (amode == A_BOS || !p.w_code_sums || !tma_room || !tma_path_ok(p, amode, w_bits)) return MIXDQ_ERR_UNSUPPORTED;
         return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
     }
     if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1)

@@ -33,6 +33,27 @@ __device__ __forceinline__ uint32_t q4(float a, float b, float c, float d, float
     return __byte_perm(__byte_perm(qa, qb, 0x0040), __byte_perm(qc, qd, 0x0040), 0x5410);
 }
 
+// 16 consecutive fp16 values (16-byte aligned) to 16 code bytes.
+__device__ __forceinline__ uint4 quantize16(const __half* __restrict__ p, float inv, float lo, float hi, uint32_t zoff)
+{
+    const uint4* src = reinterpret_cast<const uint4*>(p);
+    const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
+    const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
+    const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
+    float2 f[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[j] = __half22float2(h0[j]);
+        f[4 + j] = __half22float2(h1[j]);
+    }
+    uint4 o;
+    o.x = q4(f[0].x, f[0].y, f[1].x, f[1].y, inv, lo, hi, zoff);
+    o.y = q4(f[2].x, f[2].y, f[3].x, f[3].y, inv, lo, hi, zoff);
+    o.z = q4(f[4].x, f[4].y, f[5].x, f[5].y, inv, lo, hi, zoff);
+    o.w = q4(f[6].x, f[6].y, f[7].x, f[7].y, inv, lo, hi, zoff);
+    return o;
+}
+
 // One thread per 16 consecutive elements of a row.  bos != 0: output row r reads input row
 // (r / 76) * 77 + r % 76 + 1, i.e. the BOS token of every prompt is left out.
 // act_zero != nullptr: asymmetric codes with that zero-point (see q4).
@@ -61,22 +82,40 @@ __global__ void quant_kernel(const __half* __restrict__ X, long long ldx, long l
         hi = kMagic + static_cast<float>(255 - z);
         zoff = static_cast<uint32_t>(z - 128);
     }
-    const uint4* src = reinterpret_cast<const uint4*>(X + src_row * ldx + c * 16);
-    const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
-    const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
-    const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
-    float2 f[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        f[j] = __half22float2(h0[j]);
-        f[4 + j] = __half22float2(h1[j]);
-    }
+    *reinterpret_cast<uint4*>(out + r * K + c * 16) = quantize16(X + src_row * ldx + c * 16, inv, lo, hi, zoff);
+}
+
+// The int8 image of an asymmetrically quantized convolution input, with its padding written out: X fp16 NHWC
+// [B, H, W, Cin] -> out int8 [B, H + 2, W + 2, Cin] whose one-pixel border holds the code of the real value
+// 0 (the zero-point; stored re-centred, as zero - 128).  The GEMM's A tiles then never leave the image, and
+// the padded positions cancel against the zero-point term like any other.  One thread per 16 channels.
+__global__ void quant_pad_kernel(const __half* __restrict__ X, int B, int H, int W, int Cin,
+                                 const float* __restrict__ act_scale, const int32_t* __restrict__ act_zero,
+                                 int8_t* __restrict__ out)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int cpr = Cin >> 4;
+    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    if (idx >= static_cast<long long>(B) * (H + 2) * (W + 2) * cpr) return;
+    const long long pix = idx / cpr;
+    const int c = static_cast<int>(idx - pix * cpr);
+    const int wp = static_cast<int>(pix % (W + 2));
+    const long long t = pix / (W + 2);
+    const int hp = static_cast<int>(t % (H + 2));
+    const long long b = t / (H + 2);
+    const int z = __ldg(act_zero);
     uint4 o;
-    o.x = q4(f[0].x, f[0].y, f[1].x, f[1].y, inv, lo, hi, zoff);
-    o.y = q4(f[2].x, f[2].y, f[3].x, f[3].y, inv, lo, hi, zoff);
-    o.z = q4(f[4].x, f[4].y, f[5].x, f[5].y, inv, lo, hi, zoff);
-    o.w = q4(f[6].x, f[6].y, f[7].x, f[7].y, inv, lo, hi, zoff);
-    *reinterpret_cast<uint4*>(out + r * K + c * 16) = o;
+    if (hp == 0 || hp == H + 1 || wp == 0 || wp == W + 1) {
+        const uint32_t word = (static_cast<uint32_t>(z - 128) & 0xffu) * 0x01010101u;
+        o = make_uint4(word, word, word, word);
+    } else {
+        const float inv = __fdiv_rn(1.f, __ldg(act_scale));
+        const __half* src = X + ((b * H + (hp - 1)) * W + (wp - 1)) * Cin + c * 16;
+        o = quantize16(src, inv, kMagic - static_cast<float>(z), kMagic + static_cast<float>(255 - z),
+                       static_cast<uint32_t>(z - 128));
+    }
+    *reinterpret_cast<uint4*>(out + pix * Cin + c * 16) = o;
 }
 
 // Barrier over all threads of all CTAs of the cluster (hardware barrier, not a spin).
@@ -103,6 +142,7 @@ __device__ __forceinline__ int4 ld_cluster_v4(uint32_t addr, int cta_rank)
 struct TmaParams {
     int M, N, k_blocks;
     int conv;     // 0: A is a [M, K] int8 matrix; 1: A is an int8 NHWC image gathered per filter tap
+    int pad;      // conv: 1 when the int8 image carries its one-pixel border (asymmetric activations)
     int cblocks;  // conv: k-blocks per filter tap = ceil(Cin / 128)
     int Cin, HoWo, Wo;
     int stride;   // conv: input pixels per output pixel along H and W (1 or 2)
@@ -436,7 +476,8 @@ __device__ __forceinline__ bool produce_a_tile(const CUtensorMap* tmap_a, const 
         const uint32_t full = bar0 + 8 * (L::FULL_A + s);
         mbar_arrive_expect_tx(full, L::A_BYTES);
         if (p.conv) {
-            tma_load_4d(a0 + s * L::A_BYTES, tmap_a, cb * BK, p.stride * wo0 + kw - 1, p.stride * ho0 + kh - 1, img_b, full);
+            tma_load_4d(a0 + s * L::A_BYTES, tmap_a, cb * BK, p.stride * wo0 + kw - 1 + p.pad,
+                        p.stride * ho0 + kh - 1 + p.pad, img_b, full);
             if (++cb == p.cblocks) {
                 cb = 0;
                 if (++kw == 3) {
@@ -1157,11 +1198,17 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
 
     // 1. quantize the activations once
     const bool conv = amode == A_CONV3;
-    const long long in_rows = conv ? static_cast<long long>(p.batch) * p.H * p.W : p.M;
+    const int pad = (conv && p.act_zero) ? 1 : 0;  // asymmetric conv input: the border is written out
+    const long long in_rows = conv ? static_cast<long long>(p.batch) * (p.H + 2 * pad) * (p.W + 2 * pad) : p.M;
     const int row_len = conv ? p.Cin : p.K;
     const long long ldx = conv ? p.Cin : p.ldx;
     const long long tasks = in_rows * (row_len / 16);
-    int rc = launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
+    int rc;
+    if (pad)
+        rc = launch_pdl(quant_pad_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
+                        p.X, p.batch, p.H, p.W, p.Cin, p.act_scale, p.act_zero, aq);
+    else
+        rc = launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
                         p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, p.act_zero, aq);
     if (rc != MIXDQ_OK) return rc;
 
@@ -1191,13 +1238,14 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     if (conv) {
         int Wb, Hb, Bb;
         if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
-        const uint64_t dims[4] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.W),
-                                  static_cast<uint64_t>(p.H), static_cast<uint64_t>(p.batch)};
-        const uint64_t strides[3] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.Cin) * p.W,
-                                     static_cast<uint64_t>(p.Cin) * p.W * p.H};
+        const uint64_t Wi = static_cast<uint64_t>(p.W + 2 * pad), Hi = static_cast<uint64_t>(p.H + 2 * pad);
+        const uint64_t dims[4] = {static_cast<uint64_t>(p.Cin), Wi, Hi, static_cast<uint64_t>(p.batch)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(p.Cin), static_cast<uint64_t>(p.Cin) * Wi,
+                                     static_cast<uint64_t>(p.Cin) * Wi * Hi};
         const uint32_t box[4] = {BK, static_cast<uint32_t>(Wb), static_cast<uint32_t>(Hb), static_cast<uint32_t>(Bb)};
         rc = encode_tmap_4d_u8(&ta, aq, dims, strides, box, static_cast<uint32_t>(p.stride));
         tp.conv = 1;
+        tp.pad = pad;
         tp.stride = p.stride;
         tp.cblocks = static_cast<int>(ceil_div(p.Cin, BK));
         tp.Cin = p.Cin;

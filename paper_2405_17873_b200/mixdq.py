@@ -38,6 +38,10 @@ _SIGNATURES = {
                                     _sz, _vp, _vp]),
     "mixdq_linear_a8_asym_acc_i32": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp,
                                             _sz, _vp, _vp]),
+    "mixdq_conv3x3_a8_asym": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp,
+                                     _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_conv3x3_a8_asym_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp,
+                                             _vp, _vp, _sz, _vp, _vp]),
     "mixdq_workspace_bytes": (_int, [_i64, _i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_conv3x3_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, _int, _int, _int, C.POINTER(_sz)]),
     "mixdq_linear": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp, _sz,
@@ -262,6 +266,30 @@ def conv3x3(X, packed_W, Cout: int, w_bits: int, w_scale, w_zero=None, act_bits:
                              _ptr(w_zero), act_bits, _ptr(act_scale), _ptr(bias), _ptr(Y), wp, wb,
                              _ptr(status), _stream()), "mixdq_conv3x3")
     return Y
+
+
+def conv3x3_a8_asym(X, packed_W, Cout: int, w_bits: int, w_scale, w_code_sums, act_scale, act_zero, bias=None,
+                    stride: int = 1, workspace=None, status=None, out=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    Y = out if out is not None else torch.empty((B, Ho, Wo, Cout), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3_a8_asym(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits, _ptr(w_scale),
+                                     _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(bias), _ptr(Y),
+                                     wp, wb, _ptr(status), _stream()), "mixdq_conv3x3_a8_asym")
+    return Y
+
+
+def conv3x3_a8_asym_acc_i32(X, packed_W, Cout: int, w_bits: int, w_code_sums, act_scale, act_zero,
+                            stride: int = 1, workspace=None, status=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    acc = torch.empty((B, Ho, Wo, Cout), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3_a8_asym_acc_i32(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits,
+                                             _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(acc), wp,
+                                             wb, _ptr(status), _stream()), "mixdq_conv3x3_a8_asym_acc_i32")
+    return acc
 
 
 def conv3x3_acc_i32(X, packed_W, Cout: int, w_bits: int, act_scale, stride: int = 1, workspace=None,

@@ -34,8 +34,8 @@ class UNetSweep:
                  layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
         (whatever the image size), so that a layer is one stream over its packed weights.
-        act_asym: the 8-bit activations of the plain linear layers are asymmetric (Sec. 4.1); convolutions
-        and the BOS-aware K/V projections keep symmetric ones."""
+        act_asym: the 8-bit activations of the linear layers and 3x3 convolutions are asymmetric (Sec. 4.1);
+        the BOS-aware K/V projections keep symmetric ones."""
         assert table in ("w4a8", "a16")
         self.batch = batch
         self.act_asym = act_asym
@@ -106,7 +106,8 @@ class UNetSweep:
                     e0 = self.x[xk][0, 0].to(torch.float32)
                     bos = (W.to(torch.float32) @ e0).to(torch.float16).contiguous()
             sums = None
-            if self.act_asym and l.kind == "linear" and l.a_bits == 8:
+            # convolutions whose geometry the two-kernel path does not take (conv_in: 4 channels) stay symmetric
+            if self.act_asym and l.a_bits == 8 and (l.kind in ("linear", "conv1x1") or (l.kind == "conv3x3" and l.Cin % 32 == 0)):
                 sums = mixdq.weight_code_sums(packed, l.N, l.K, l.w_bits)
                 if xk not in self.x_asym:
                     self.x_asym[xk] = mixdq.act_asym_params(self.x[xk].reshape(-1, xk[-1]))
@@ -128,6 +129,10 @@ class UNetSweep:
         x, y = self.x[pl.x_key], self.y[pl.y_key]
         sx = self.x_scale.get(pl.x_key) if l.a_bits == 8 else None
         ws = workspace if workspace is not None else self.workspace
+        if l.kind == "conv3x3" and pl.code_sums is not None:
+            ax, az = self.x_asym[pl.x_key]
+            return mixdq.conv3x3_a8_asym(x, pl.packed, l.N, l.w_bits, pl.w_scale, pl.code_sums, ax, az, pl.bias,
+                                         l.stride, ws, self.status, out=y)
         if l.kind == "conv3x3":
             return mixdq.conv3x3(x, pl.packed, l.N, l.w_bits, pl.w_scale, pl.w_zero, l.a_bits, sx, pl.bias,
                                  l.stride, ws, self.status, out=y)
@@ -189,7 +194,7 @@ def _main(argv=None) -> int:
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--tokens", type=int, default=0, help="linear layers only: run on this many rows (weight-bound regime)")
-    ap.add_argument("--act-asym", action="store_true", help="asymmetric 8-bit activations (plain linear layers)")
+    ap.add_argument("--act-asym", action="store_true", help="asymmetric 8-bit activations (linear layers and 3x3 convolutions)")
     ap.add_argument("--eager", action="store_true", help="plain launches only, no graph and no timing")
     a = ap.parse_args(argv)
 

@@ -95,3 +95,66 @@ def test_linear_asym_needs_the_workspace():
     sx, zx = mixdq.act_asym_params(dev(X))
     with pytest.raises(mixdq.MixdqError):
         mixdq.linear_a8_asym(dev(X), packed, N, 8, s, sums, sx, zx)
+
+
+# ----------------------------------------------------------------------------- 3x3 convolution
+
+def _run_conv(X, Wt, b, bits, stride):
+    B, H, W, Cin = X.shape
+    Cout = Wt.shape[0]
+    s_ref, _, codes = oracle_weights(Wt.reshape(Cout, -1), bits, True)
+    sx_ref, zx_ref = orc.act_minmax_params(X)
+    acc_ref, y_ref = orc.conv3x3_a8_asym(X, codes.reshape(Cout, 3, 3, Cin), s_ref, sx_ref, zx_ref, b, stride)
+
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt.reshape(Cout, -1), bits, True)
+    sums = mixdq.weight_code_sums(packed, Cout, 9 * Cin, bits)
+    sx, zx = mixdq.act_asym_params(Xd)
+    assert host(sx)[0] == sx_ref and int(host(zx)[0]) == zx_ref
+    st = status_word()
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, W, Cin, Cout, stride, bits, 8))
+    acc = mixdq.conv3x3_a8_asym_acc_i32(Xd, packed, Cout, bits, sums, sx, zx, stride, workspace=ws, status=st)
+    y = mixdq.conv3x3_a8_asym(Xd, packed, Cout, bits, s, sums, sx, zx, None if b is None else dev(b), stride,
+                              workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+    return zx_ref
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,W,Cin,Cout,stride", [(1, 16, 16, 320, 136, 1), (3, 8, 8, 32, 40, 1),
+                                                    (2, 32, 32, 160, 136, 1), (1, 64, 64, 32, 24, 1),
+                                                    (1, 16, 16, 640, 264, 1), (2, 16, 16, 64, 48, 2),
+                                                    (1, 64, 64, 64, 40, 2), (2, 32, 32, 160, 136, 2),
+                                                    # persistent kernel: 128- and 256-wide tiles
+                                                    (4, 64, 64, 64, 264, 1), (5, 64, 64, 32, 512, 1)])
+def test_conv3x3_asym_post_silu_input(bits, B, H, W, Cin, Cout, stride):
+    X = synth.one_sided_f16((B, H, W, Cin), seed=H * W + Cin + 1)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=Cout + Cin + 2)
+    b = synth.normal_f16((Cout,), 0.01, seed=Cout + 3)
+    assert 0 < _run_conv(X, Wt, b, bits, stride) < 40
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_conv3x3_asym_border_is_the_zero_point(bits):
+    # one-signed images put the zero-point at an end of the grid, where a border filled with any other code
+    # (0, or the re-centred 0) would show in every border pixel; positive weights make it add up
+    Wt = np.abs(synth.normal_f16((72, 3, 3, 64), 0.02, seed=41))
+    Xp = np.abs(synth.normal_f16((2, 16, 16, 64), 1.0, seed=42)) + np.float16(0.5)
+    assert _run_conv(Xp, Wt, None, bits, 1) == 0
+    assert _run_conv(-Xp, Wt, None, bits, 1) == 255
+    assert _run_conv(-Xp, Wt, None, bits, 2) == 255
+
+
+def test_conv3x3_asym_geometry_outside_the_two_kernel_path():
+    B, H, W, Cin, Cout = 2, 12, 10, 32, 48
+    X = synth.one_sided_f16((B, H, W, Cin), seed=1)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=2)
+    s, _, packed = device_weights(Wt.reshape(Cout, -1), 8, True)
+    sums = mixdq.weight_code_sums(packed, Cout, 9 * Cin, 8)
+    sx, zx = mixdq.act_asym_params(dev(X))
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, W, Cin, Cout, 1, 8, 8))
+    with pytest.raises(mixdq.MixdqError):
+        mixdq.conv3x3_a8_asym(dev(X), packed, Cout, 8, s, sums, sx, zx, workspace=ws)
