@@ -326,6 +326,9 @@ int orc_int_gemm_i16(const int16_t *cx, const int16_t *qw, int64_t M, int64_t N,
 /*          of code[32 g + j]; a ragged last group is padded with      */
 /*          pad_code (the row's zero-point, so padding dequantizes to  */
 /*          0); row pitch ceil(K/32) * 12.                             */
+/*   2-bit: the same with two planes P0,P1 (four codes per byte: the   */
+/*          paper's lowest candidate width, Sec. 3.3); pitch           */
+/*          ceil(K/32) * 8.                                            */
 /* ------------------------------------------------------------------ */
 
 int64_t orc_packed_row_bytes(int64_t K, int bits)
@@ -333,7 +336,7 @@ int64_t orc_packed_row_bytes(int64_t K, int bits)
     if (K <= 0) return -1;
     if (bits == 8) return K;
     if (bits == 4) return (K + 1) / 2;
-    if (bits == 3) return ((K + 31) / 32) * 12;
+    if (bits == 3 || bits == 2) return ((K + 31) / 32) * 4 * bits;
     return -1;
 }
 
@@ -359,13 +362,13 @@ int orc_pack_codes(const int16_t *codes, int64_t N, int64_t K, int bits, const i
                 for (int j = 0; j < 32; ++j) {
                     int64_t k = 32 * g + j;
                     int c = (k < K) ? codes[n * K + k] : (pad_code ? pad_code[n] : 0);
-                    if (c < 0 || c > 7) return ORC_ERR_ARG;
-                    for (int p = 0; p < 3; ++p)
+                    if (c < 0 || c >= (1 << bits)) return ORC_ERR_ARG;
+                    for (int p = 0; p < bits; ++p)
                         if ((c >> p) & 1) plane[p] |= (1u << j);
                 }
-                for (int p = 0; p < 3; ++p)
+                for (int p = 0; p < bits; ++p)
                     for (int b = 0; b < 4; ++b)
-                        row[g * 12 + p * 4 + b] = (uint8_t)((plane[p] >> (8 * b)) & 0xff);
+                        row[g * 4 * bits + p * 4 + b] = (uint8_t)((plane[p] >> (8 * b)) & 0xff);
             }
         }
     }
@@ -390,9 +393,9 @@ int orc_unpack_codes(const uint8_t *packed, int64_t N, int64_t K, int bits, int 
                 int64_t g = k / 32;
                 int j = (int)(k % 32);
                 c = 0;
-                for (int p = 0; p < 3; ++p) {
+                for (int p = 0; p < bits; ++p) {
                     uint32_t plane = 0;
-                    for (int b = 0; b < 4; ++b) plane |= (uint32_t)row[g * 12 + p * 4 + b] << (8 * b);
+                    for (int b = 0; b < 4; ++b) plane |= (uint32_t)row[g * 4 * bits + p * 4 + b] << (8 * b);
                     c |= (int)((plane >> j) & 1u) << p;
                 }
             }

@@ -36,6 +36,16 @@ def test_bitplane_golden_words():
     assert _planes_of([2] + [0] * 31) == g["first2"]
 
 
+def test_two_bit_plane_words_by_hand():
+    # the first two planes of the 3-bit words: a 2-bit code is a 3-bit code whose top plane is absent
+    g = _read_planes()
+    two = lambda codes: orc.pack_codes(np.asarray(codes, np.int16).reshape(1, 32), 2).view("<u4")[0].tolist()
+    assert two([j % 4 for j in range(32)]) == g["jmod8"][:2]
+    assert two([3] * 32) == g["all7"][:2]
+    assert two([2] + [0] * 31) == g["first2"][:2]
+    assert two([0] * 31 + [1]) == [0x80000000, 0]
+
+
 def test_nibble_and_byte_layout_by_hand():
     # 4-bit: even k in the low nibble; signed codes as two's-complement nibbles
     packed = orc.pack_codes(np.array([[1, 2, -1, -8 + 1, 7]], np.int16), 4)
@@ -44,21 +54,21 @@ def test_nibble_and_byte_layout_by_hand():
     assert packed[0].tolist() == [0x81, 0xFF, 0x00, 0x7F, 0xFF]
 
 
-@pytest.mark.parametrize("bits,signed", [(3, False), (4, False), (4, True), (8, False), (8, True)])
+@pytest.mark.parametrize("bits,signed", [(2, False), (3, False), (4, False), (4, True), (8, False), (8, True)])
 @pytest.mark.parametrize("K", [1, 31, 32, 33, 64, 77, 320])
 def test_pack_roundtrip_and_size_law(bits, signed, K):
     rng = np.random.default_rng(bits * 100 + K)
     lo, hi = (-(2 ** (bits - 1) - 1), 2 ** (bits - 1) - 1) if signed else (0, 2 ** bits - 1)
     codes = rng.integers(lo, hi + 1, size=(5, K)).astype(np.int16)
-    pad = rng.integers(0, 8, size=5).astype(np.int32)
+    pad = rng.integers(0, min(8, 2 ** bits), size=5).astype(np.int32)
     packed = orc.pack_codes(codes, bits, pad)
-    want = {8: K, 4: (K + 1) // 2, 3: ((K + 31) // 32) * 12}[bits]
+    want = {8: K, 4: (K + 1) // 2, 3: ((K + 31) // 32) * 12, 2: ((K + 31) // 32) * 8}[bits]
     assert packed.shape == (5, want)
     assert np.array_equal(orc.unpack_codes(packed, K, bits, signed), codes)
-    if bits == 3 and K % 32:
+    if bits <= 3 and K % 32:
         # the ragged tail holds the pad code (the row's zero-point)
         Kp = ((K + 31) // 32) * 32
-        full = orc.unpack_codes(packed, Kp, 3, False)
+        full = orc.unpack_codes(packed, Kp, bits, False)
         assert np.array_equal(full[:, K:], np.repeat(pad[:, None], Kp - K, 1))
 
 
@@ -69,6 +79,14 @@ def test_every_value_in_every_position():
             codes[0, pos] = val
             planes = orc.pack_codes(codes, 3).view("<u4")[0]
             for p in range(3):
+                assert int(planes[p]) == (((val >> p) & 1) << pos)
+    for pos in range(32):
+        for val in range(4):
+            codes = np.zeros((1, 32), np.int16)
+            codes[0, pos] = val
+            planes = orc.pack_codes(codes, 2).view("<u4")[0]
+            assert planes.shape == (2,)
+            for p in range(2):
                 assert int(planes[p]) == (((val >> p) & 1) << pos)
     for pos in range(2):
         for val in range(-7, 8):
@@ -83,7 +101,7 @@ def test_storage_saving_matches_table1():
     # size ratio to fp16 is 16 / average-bits: compare with the values the paper prints
     rows = np.loadtxt(os.path.join(GOLDEN, "table1_storage_opt.txt"))
     K = 1280
-    for bits in (3, 4, 8):
+    for bits in (2, 3, 4, 8):
         assert orc.packed_row_bytes(K, bits) * 8 == K * bits
     for avg_bits, printed in rows:
         assert abs(16.0 / avg_bits - printed) <= 0.05 + 1e-9
@@ -312,7 +330,7 @@ def test_a8_asym_equals_fake_quant_matmul(bits):
         assert ea < 0.75 * es
 
 
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 def test_weight_only_equals_fake_quant_matmul(bits):
     X = synth.normal_f16((33, 70), 1.0, seed=21)
     W = synth.normal_f16((19, 70), 0.02, seed=22)

@@ -79,7 +79,7 @@ def test_act_codes_clamp_to_restricted_range():
     assert got.tolist() == [127, -127, 127, -127, 127, -127]
 
 
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("symmetric", [True, False])
 def test_weight_quant_error_bound_extremes_and_idempotence(bits, symmetric):
     W = synth.normal_f16((48, 200), 0.02, seed=11 + bits)
@@ -133,7 +133,7 @@ def test_weight_quant_error_bound_extremes_and_idempotence(bits, symmetric):
 
 def test_weight_codes_vs_exact_rationals_asymmetric():
     W = synth.normal_f16((6, 64), 0.02, seed=77)
-    for bits in (3, 4, 8):
+    for bits in (2, 3, 4, 8):
         scale, zero = orc.weight_minmax_params(W, bits, False)
         codes = orc.quantize_weights(W, bits, scale, zero)
         L = 2 ** bits - 1
@@ -151,11 +151,12 @@ def test_sqnr_rises_six_db_per_bit():
     W = synth.normal_f16((64, 1024), 0.02, seed=5)
     w = W.astype(np.float64)
     sq = {}
-    for bits in (3, 4, 8):
+    for bits in (2, 3, 4, 8):
         scale, zero = orc.weight_minmax_params(W, bits, False)
         deq = orc.dequantize_weights(orc.quantize_weights(W, bits, scale, zero), scale, zero)
         sq[bits] = 10 * np.log10((w ** 2).sum() / ((deq - w) ** 2).sum())
     assert 4.5 < sq[4] - sq[3] < 8.0
+    assert 3.0 < sq[3] - sq[2] < 9.0     # a 4-level min-max grid on a Gaussian row is far from uniform-noise theory
     assert 22.0 < sq[8] - sq[4] < 26.5   # four more bits: ~24 dB
 
 
