@@ -63,12 +63,14 @@ const char* mixdq_strerror(int code);
  * Bytes of a packed [N, K] weight matrix.  `out` is a HOST pointer.
  * Canonical layout: row pitch K (8-bit), ceil(K/2) (4-bit, even k in the low nibble),
  * ceil(K/32)*12 (3-bit: per group of 32 codes three little-endian u32 bit-planes, bit j of
- * plane p = bit p of code 32g+j; a ragged last group is padded with the row's zero-point).
+ * plane p = bit p of code 32g+j; a ragged last group is padded with the row's zero-point),
+ * ceil(K/32)*8 (2-bit, the lowest candidate width of Sec. 3.3: the same with two planes).
  * Device layout: 8-bit rows padded to a multiple of 16 bytes; 4-bit rows padded to a
  * multiple of 32 codes with, inside every group of 8 codes, byte j holding code j in the
  * low nibble and code j+4 in the high nibble; 3-bit rows padded to a multiple of 128
  * codes, each block of 128 codes stored as three 16-byte bit-planes whose bits are
- * interleaved for the register decode (mixdq_unpack_weights undoes it).
+ * interleaved for the register decode (mixdq_unpack_weights undoes it); 2-bit rows alike with
+ * two planes per block (32 bytes per 128 codes).
  */
 int mixdq_packed_bytes(int64_t N, int64_t K, int bits, int layout, size_t* out);
 
@@ -84,8 +86,8 @@ int mixdq_weight_minmax_params(const void* W, int64_t N, int64_t K, int bits, in
 
 /*
  * Quantize W (fp16 [N, K]) with the given per-channel scale (and zero-point) and pack the
- * codes.  bits in {3, 4, 8}.  zero == NULL selects symmetric signed codes (not available
- * for 3 bits).  `packed_out` must hold mixdq_packed_bytes(N, K, bits, layout) bytes and be
+ * codes.  bits in {2, 3, 4, 8}.  zero == NULL selects symmetric signed codes (not available
+ * for 2 and 3 bits).  `packed_out` must hold mixdq_packed_bytes(N, K, bits, layout) bytes and be
  * 16-byte aligned.  This is the offline step of the path: it runs once per layer.
  */
 int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits, const float* scale,
@@ -152,7 +154,7 @@ int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t Cin, 
  *                   inside the kernel, multiplied with the integer weight codes in int32
  *                   and dequantized as  y = fp16(acc * act_scale * w_scale[n] + bias[n]).
  *                   Weights must be symmetric (w_zero == NULL), w_bits in {4, 8}.
- *   act_bits == 16: weight-only W3/W4/W8-A16 (Table 1 "weight only" rows): X stays fp16,
+ *   act_bits == 16: weight-only W2/W3/W4/W8-A16 (Table 1 "weight only" rows): X stays fp16,
  *                   y = fp16(w_scale[n] * sum_k x[k] * (q[n,k] - w_zero[n]) + bias[n]).
  *                   act_scale is ignored.  w_zero == NULL means signed codes, zero-point 0.
  * packed_W is in MIXDQ_LAYOUT_DEVICE.  ldx is the row stride of X in elements (>= K,

@@ -16,8 +16,8 @@ int check_widths(int w_bits, int act_bits, const int32_t* w_zero)
         return MIXDQ_OK;
     }
     if (act_bits == 16) {
-        if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
-        if (w_bits == 3 && !w_zero) return MIXDQ_ERR_UNSUPPORTED;
+        if (w_bits != 2 && w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+        if (w_bits <= 3 && !w_zero) return MIXDQ_ERR_UNSUPPORTED;
         return MIXDQ_OK;
     }
     return MIXDQ_ERR_UNSUPPORTED;
@@ -193,7 +193,7 @@ extern "C" int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_b
 {
     if (!out || rows <= 0 || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
-    if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits != 2 && w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     *out = (act_bits == 8) ? i8::workspace_bytes(rows, N, rows, K) : 0;
     return MIXDQ_OK;
 }
@@ -204,7 +204,7 @@ extern "C" int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, in
     if (!out || B <= 0 || H <= 0 || W <= 0 || Cin <= 0 || Cout <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (stride != 1 && stride != 2) return MIXDQ_ERR_INVALID_ARG;
     if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
-    if (w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits != 2 && w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
     // room for the int8 image with a one-pixel border, which the asymmetric-activation call keeps
     *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * (H + 2) * (W + 2), Cin) : 0;

@@ -24,11 +24,11 @@ inline int64_t row_pitch_bytes(int64_t K, int bits, int layout)
     if (layout == MIXDQ_LAYOUT_CANONICAL) {
         if (bits == 8) return K;
         if (bits == 4) return (K + 1) / 2;
-        if (bits == 3) return ceil_div(K, 32) * 12;
+        if (bits == 3 || bits == 2) return ceil_div(K, 32) * 4 * bits;
     } else if (layout == MIXDQ_LAYOUT_DEVICE) {
         if (bits == 8) return round_up(K, 16);
         if (bits == 4) return round_up(K, 32) / 2;
-        if (bits == 3) return ceil_div(K, 128) * 48;
+        if (bits == 3 || bits == 2) return ceil_div(K, 128) * 16 * bits;
     }
     return -1;
 }

@@ -109,24 +109,24 @@ __global__ void pack_kernel(const __half* __restrict__ W, int64_t N, int64_t K, 
                 word |= (lo | (hi << 4)) << (8 * j);
             }
         }
-    } else {  // 3-bit planes
+    } else {  // bit-planes: `bits` (3 or 2) planes per group
         if (layout == MIXDQ_LAYOUT_CANONICAL) {
-            const int64_t k0 = 32 * (w / 3);  // group g: words 3g .. 3g+2 are planes 0..2
-            const int plane = static_cast<int>(w % 3);
+            const int64_t k0 = 32 * (w / bits);  // group g: words bits*g .. are planes 0..bits-1
+            const int plane = static_cast<int>(w % bits);
             for (int j = 0; j < 32; ++j)
-                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << j;
+                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, bits, inv, hz, z) >> plane) & 1) << j;
         } else {
             // block of 128 codes: planes in order, 4 words each; word t of a plane covers codes
             // 32t .. 32t+31 with bit 4f + s = code 8s + (f even ? f/2 : 4 + f/2), which is the
             // field order of the 4-bit device layout spread over four shifts of the word
-            const int64_t blk = w / 12;
-            const int r = static_cast<int>(w % 12);
+            const int64_t blk = w / (4 * bits);
+            const int r = static_cast<int>(w % (4 * bits));
             const int plane = r / 4;
             const int64_t k0 = 128 * blk + 32 * (r % 4);
             for (int pos = 0; pos < 32; ++pos) {
                 const int f = pos >> 2, sft = pos & 3;
                 const int j = 8 * sft + ((f & 1) ? 4 + (f >> 1) : (f >> 1));
-                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, 3, inv, hz, z) >> plane) & 1) << pos;
+                word |= static_cast<uint32_t>((code_at(W, n, k0 + j, K, bits, inv, hz, z) >> plane) & 1) << pos;
             }
         }
     }
@@ -155,11 +155,11 @@ __device__ __forceinline__ int decode_code(const uint8_t* __restrict__ row, int6
         c = (is_signed && nib >= 8) ? nib - 16 : nib;
     } else {
         c = 0;
-        for (int p = 0; p < 3; ++p) {
+        for (int p = 0; p < bits; ++p) {
             int64_t byte;
             int bit;
             if (layout == MIXDQ_LAYOUT_CANONICAL) {
-                byte = (k / 32) * 12 + p * 4 + ((k % 32) >> 3);
+                byte = (k / 32) * 4 * bits + p * 4 + ((k % 32) >> 3);
                 bit = static_cast<int>(k & 7);
             } else {
                 const int64_t blk = k / 128;
@@ -167,7 +167,7 @@ __device__ __forceinline__ int decode_code(const uint8_t* __restrict__ row, int6
                 const int t = r >> 5, sft = (r & 31) >> 3, j = r & 7;
                 const int f = (j < 4) ? 2 * j : 2 * (j - 4) + 1;
                 const int pos = 4 * f + sft;
-                byte = blk * 48 + p * 16 + t * 4 + (pos >> 3);
+                byte = blk * 16 * bits + p * 16 + t * 4 + (pos >> 3);
                 bit = pos & 7;
             }
             c |= ((row[byte] >> bit) & 1) << p;
@@ -322,7 +322,7 @@ __global__ void act_scale_kernel(const float* __restrict__ amax, float* __restri
     scale_out[0] = (a == 0.f) ? 1.f : __fdiv_rn(a, 127.f);
 }
 
-bool width_ok(int bits) { return bits == 3 || bits == 4 || bits == 8; }
+bool width_ok(int bits) { return bits == 2 || bits == 3 || bits == 4 || bits == 8; }
 
 }  // namespace
 
@@ -361,7 +361,7 @@ extern "C" int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits,
     if (!W || !scale || !packed_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (layout != MIXDQ_LAYOUT_CANONICAL && layout != MIXDQ_LAYOUT_DEVICE) return MIXDQ_ERR_INVALID_ARG;
     if (!width_ok(bits)) return MIXDQ_ERR_UNSUPPORTED;
-    if (bits == 3 && !zero) return MIXDQ_ERR_UNSUPPORTED;  // 3-bit codes are unsigned only
+    if (bits <= 3 && !zero) return MIXDQ_ERR_UNSUPPORTED;  // bit-plane codes are unsigned only
     if (reinterpret_cast<uintptr_t>(packed_out) & 15) return MIXDQ_ERR_ALIGNMENT;
     const int64_t pitch = row_pitch_bytes(K, bits, layout);
     const int64_t words = N * ((pitch + 3) / 4);
@@ -377,7 +377,7 @@ extern "C" int mixdq_unpack_weights(const void* packed, int64_t N, int64_t K, in
     if (!packed || !codes_out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (layout != MIXDQ_LAYOUT_CANONICAL && layout != MIXDQ_LAYOUT_DEVICE) return MIXDQ_ERR_INVALID_ARG;
     if (!width_ok(bits)) return MIXDQ_ERR_UNSUPPORTED;
-    if (bits == 3 && is_signed) return MIXDQ_ERR_UNSUPPORTED;
+    if (bits <= 3 && is_signed) return MIXDQ_ERR_UNSUPPORTED;
     const int64_t pitch = row_pitch_bytes(K, bits, layout);
     unpack_kernel<<<static_cast<unsigned>(ceil_div(N * K, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(packed), N, K, bits, is_signed, layout, pitch, codes_out);

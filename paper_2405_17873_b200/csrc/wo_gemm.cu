@@ -88,10 +88,11 @@ __device__ __forceinline__ void load_unit(UnitRegs<BITS>& u, const uint8_t* __re
             u.w[4] = v.x; u.w[5] = v.y; u.w[6] = v.z; u.w[7] = v.w;
         }
     } else {
-        const long long off = static_cast<long long>(unit) * 48 + t * 4;
+        // bit-planes (3 or 2 of them; the decode reads an absent top plane as zeros)
+        const long long off = static_cast<long long>(unit) * (16 * BITS) + t * 4;
         if (off < pitch) {
 #pragma unroll
-            for (int p = 0; p < 3; ++p) u.w[p] = __ldg(reinterpret_cast<const uint32_t*>(row + off + 16 * p));
+            for (int p = 0; p < BITS; ++p) u.w[p] = __ldg(reinterpret_cast<const uint32_t*>(row + off + 16 * p));
         }
     }
 }
@@ -106,7 +107,7 @@ __device__ __forceinline__ void decode_substep(const UnitRegs<BITS>& u, int s, _
         uint32_t w = u.w[s];
         if (SIGNED) w ^= 0x88888888u;
         decode_fields<0xFu>(w, z_lo, z_hi, f);
-    } else if (BITS == 3) {
+    } else if (BITS <= 3) {
         // bit 4n + s of plane p is bit p of field n of sub-step s: gather the three planes
         // into one word of 4-bit-spaced fields (bit 3 of each field is ignored by the mask)
         const uint32_t a = u.w[0] >> s;
@@ -540,8 +541,9 @@ int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream
         return MIXDQ_ERR_ALIGNMENT;
     const long long pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
     const bool is_signed = p.w_zero == nullptr;
-    if (tc_path_ok(p, amode, w_bits) && !(w_bits == 3 && is_signed)) return run_tc(p, amode, packed, w_bits, p.batch, stream);
+    if (tc_path_ok(p, amode, w_bits) && !(w_bits <= 3 && is_signed)) return run_tc(p, amode, packed, w_bits, p.batch, stream);
     if (w_bits == 3) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_nt<3, false>(p, amode, packed, pitch, stream);
+    if (w_bits == 2) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_nt<2, false>(p, amode, packed, pitch, stream);
     if (w_bits == 4)
         return is_signed ? launch_nt<4, true>(p, amode, packed, pitch, stream)
                          : launch_nt<4, false>(p, amode, packed, pitch, stream);

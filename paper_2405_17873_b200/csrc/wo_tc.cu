@@ -103,10 +103,11 @@ __device__ __forceinline__ void load_codes32(Codes32<BITS>& c, const uint8_t* __
         }
     } else {
         // 128-code blocks of three 16-byte planes; word (k32 % 4) of each plane holds this run
-        const long long off = static_cast<long long>(k32 >> 2) * 48 + (k32 & 3) * 4;
+        // (two planes for 2-bit codes: the decode reads the absent top plane as zeros)
+        const long long off = static_cast<long long>(k32 >> 2) * (16 * BITS) + (k32 & 3) * 4;
         if (off < pitch) {
 #pragma unroll
-            for (int p = 0; p < 3; ++p) c.w[p] = __ldg(reinterpret_cast<const uint32_t*>(row + off + 16 * p));
+            for (int p = 0; p < BITS; ++p) c.w[p] = __ldg(reinterpret_cast<const uint32_t*>(row + off + 16 * p));
         }
     }
 }
@@ -119,7 +120,7 @@ __device__ __forceinline__ uint4 decode8(const Codes32<BITS>& c, int s, __half2 
         uint32_t w = c.w[s];
         if (SIGNED) w ^= 0x88888888u;
         return decode_word<0xFu>(w, z_lo, z_hi);
-    } else if (BITS == 3) {
+    } else if (BITS <= 3) {
         const uint32_t a = c.w[0] >> s;
         const uint32_t b = (s == 0) ? (c.w[1] << 1) : (c.w[1] >> (s - 1));
         const uint32_t d = (s <= 1) ? (c.w[2] << (2 - s)) : (c.w[2] >> (s - 2));
@@ -484,6 +485,7 @@ int run_tc(const Params& p, int amode, const void* packed, int w_bits, int batch
     if (rc != MIXDQ_OK) return rc;
     const bool is_signed = p.w_zero == nullptr;
     if (w_bits == 3) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_tc<3, false>(tx, tp, stream);
+    if (w_bits == 2) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_tc<2, false>(tx, tp, stream);
     if (w_bits == 4) return is_signed ? launch_tc<4, true>(tx, tp, stream) : launch_tc<4, false>(tx, tp, stream);
     if (w_bits == 8) return is_signed ? launch_tc<8, true>(tx, tp, stream) : launch_tc<8, false>(tx, tp, stream);
     return MIXDQ_ERR_UNSUPPORTED;

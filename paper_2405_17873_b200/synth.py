@@ -185,11 +185,13 @@ def unet_layers() -> List[LayerSpec]:
 
 
 def assign_bits_weight_only(layers: List[LayerSpec], seed: int = 5, target: float = 3.66,
-                            frac8: float = 0.02) -> None:
+                            frac8: float = 0.02, low: int = 3) -> None:
     """Seeded A16 table whose parameter-weighted mean weight width is ~3.66 bits
     (the W3.66A16 row of Table 1): a shuffled ~2% of parameters at 8 bits, then a
-    3-vs-4 split chosen to land on the target.  conv_in / conv_out stay at 8 bits
-    (Sec. 5 lists them as the sensitive convolutions)."""
+    `low`-vs-4 split chosen to land on the target (low = 3, or 2 for the paper's own candidate
+    widths {2, 4, 8}, Sec. 3.3).  conv_in / conv_out stay at 8 bits (Sec. 5 lists them as the
+    sensitive convolutions)."""
+    assert low in (2, 3)
     rng = np.random.default_rng(seed)
     order = rng.permutation(len(layers))
     total = sum(l.params for l in layers)
@@ -207,12 +209,12 @@ def assign_bits_weight_only(layers: List[LayerSpec], seed: int = 5, target: floa
             l.w_bits = 8
             p8 += l.params
     rest = [l for l in rest if l.w_bits == 0]
-    # choose params at 3 bits so that (8*p8 + 3*p3 + 4*(total-p8-p3)) / total == target
-    want_p3 = 8 * p8 + 4 * (total - p8) - target * total
+    # choose params at `low` bits so that (8*p8 + low*p3 + 4*(total-p8-p3)) / total == target
+    want_p3 = (8 * p8 + 4 * (total - p8) - target * total) / (4 - low)
     p3 = 0
     for l in rest:
         if p3 + l.params <= want_p3:
-            l.w_bits = 3
+            l.w_bits = low
             p3 += l.params
         else:
             l.w_bits = 4

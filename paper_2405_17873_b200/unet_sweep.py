@@ -31,11 +31,13 @@ class PackedLayer:
 
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
-                 layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False):
+                 layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False,
+                 low_bits: int = 3):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
         (whatever the image size), so that a layer is one stream over its packed weights.
         act_asym: the 8-bit activations of the linear layers and 3x3 convolutions are asymmetric (Sec. 4.1);
-        the BOS-aware K/V projections keep symmetric ones."""
+        the BOS-aware K/V projections keep symmetric ones.
+        low_bits: lowest width of the a16 table (3, or 2 for the paper's candidate widths {2, 4, 8})."""
         assert table in ("w4a8", "a16")
         self.batch = batch
         self.act_asym = act_asym
@@ -49,7 +51,7 @@ class UNetSweep:
             if table == "w4a8":
                 synth.assign_bits_w4a8(self.specs, seed)
             else:
-                synth.assign_bits_weight_only(self.specs, seed)
+                synth.assign_bits_weight_only(self.specs, seed, low=low_bits)
         self.x: Dict[tuple, torch.Tensor] = {}
         self.y: Dict[tuple, torch.Tensor] = {}
         self.x_scale: Dict[tuple, torch.Tensor] = {}

@@ -18,7 +18,7 @@ def _weights(N, K, seed):
     return W
 
 
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("symmetric", [True, False])
 @pytest.mark.parametrize("N,K", [(37, 77), (64, 320), (130, 1000)])
 def test_minmax_params_bit_exact(bits, symmetric, N, K):
@@ -29,7 +29,7 @@ def test_minmax_params_bit_exact(bits, symmetric, N, K):
     assert np.array_equal(host(z), z_ref)
 
 
-@pytest.mark.parametrize("bits,symmetric", [(3, False), (4, False), (4, True), (8, False), (8, True)])
+@pytest.mark.parametrize("bits,symmetric", [(2, False), (3, False), (4, False), (4, True), (8, False), (8, True)])
 @pytest.mark.parametrize("N,K", [(5, 1), (37, 77), (64, 320), (33, 1000), (16, 2048)])
 def test_packed_bytes_and_codes_bit_exact(bits, symmetric, N, K):
     W = _weights(max(N, 4), K, 200 + bits + K)[:N] if N >= 4 else _weights(4, K, 200 + bits + K)[:N]
@@ -51,7 +51,7 @@ def test_packed_bytes_and_codes_bit_exact(bits, symmetric, N, K):
 
 def test_unpack_reads_oracle_packed_bytes():
     rng = np.random.default_rng(3)
-    for bits, signed in ((3, False), (4, True), (4, False), (8, True), (8, False)):
+    for bits, signed in ((2, False), (3, False), (4, True), (4, False), (8, True), (8, False)):
         lo, hi = (-(2 ** (bits - 1) - 1), 2 ** (bits - 1) - 1) if signed else (0, 2 ** bits - 1)
         codes = rng.integers(lo, hi + 1, size=(9, 75)).astype(np.int16)
         packed = orc.pack_codes(codes, bits, np.zeros(9, np.int32))

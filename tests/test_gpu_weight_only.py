@@ -27,7 +27,7 @@ def test_mixed_bitwidth_trio(idx, M):
     _run(X, W, b, bits)
 
 
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("M,K,N", [(1, 128, 16), (5, 136, 40), (16, 1280, 96), (33, 2560, 72), (8, 4224, 48),
                                    (77, 320, 330)])
 def test_ragged_shapes(bits, M, K, N):
@@ -38,7 +38,7 @@ def test_ragged_shapes(bits, M, K, N):
 
 
 # 64 tokens or more: the tensor-memory (tcgen05) form of the engine, one or several tiles per CTA
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("M,K,N", [(64, 64, 16), (300, 2880, 136), (2100, 320, 1300), (130, 200, 264), (4096, 320, 320)])
 def test_many_token_shapes(bits, M, K, N):
     X = synth.normal_f16((M, K), 1.0, seed=M * 7 + K)
@@ -61,7 +61,7 @@ def test_symmetric_codes_at_a16(bits):
     _run(X, W, None, bits, symmetric=True)
 
 
-@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("geom", [(2, 6, 5, 32, 40, 1), (2, 6, 5, 32, 40, 2), (2, 16, 16, 64, 40, 1),
                                   (1, 8, 8, 128, 48, 1), (3, 32, 32, 192, 136, 1)])
 def test_weight_only_conv3x3(bits, geom):
