@@ -499,6 +499,25 @@ int orc_int_conv3x3_i16(const int16_t *cx, const int16_t *qw, int64_t B, int64_t
     return overflow ? ORC_ERR_OVERFLOW : ORC_OK;
 }
 
+/* Shortcut-splitting (Sec. 4.1, after Q-Diffusion): the reduction range of a layer fed by a concatenation
+ * [hidden | skip] is cut at the seam, each part has its own per-tensor activation scale and its own int32
+ * accumulator, and the two meet only after dequantization:
+ *   y = fp16( (acc_lo * s_lo + acc_hi * s_hi) * s_w[n] + bias[n] ), in double. */
+int orc_dequant_epilogue_split(const int32_t *acc_lo, const int32_t *acc_hi, int64_t M, int64_t N, float s_lo,
+                               float s_hi, const float *w_scale, const uint16_t *bias, uint16_t *Y)
+{
+    if (!acc_lo || !acc_hi || !w_scale || !Y) return ORC_ERR_ARG;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double y = ((double)acc_lo[m * N + n] * (double)s_lo + (double)acc_hi[m * N + n] * (double)s_hi) *
+                       (double)w_scale[n];
+            if (bias) y += half_to_double(bias[n]);
+            Y[m * N + n] = double_to_half(y);
+        }
+    return ORC_OK;
+}
+
 /* Dequantize + bias: y = fp16( acc * s_x * s_w[n] + bias[n] ), in double. */
 int orc_dequant_epilogue(const int32_t *acc, int64_t M, int64_t N, float act_scale,
                          const float *w_scale, const uint16_t *bias, uint16_t *Y)

@@ -249,6 +249,21 @@ def dequant_epilogue(acc, act_scale_, w_scale, bias=None):
     return Y
 
 
+def dequant_epilogue_split(acc_lo, acc_hi, s_lo, s_hi, w_scale, bias=None):
+    acc_lo = np.ascontiguousarray(acc_lo, np.int32)
+    acc_hi = np.ascontiguousarray(acc_hi, np.int32)
+    assert acc_lo.shape == acc_hi.shape
+    N = acc_lo.shape[-1]
+    M = acc_lo.size // N
+    w_scale = np.ascontiguousarray(w_scale, np.float32)
+    bias = None if bias is None else _f16(bias)
+    Y = np.empty(acc_lo.shape, np.float16)
+    _chk(lib().orc_dequant_epilogue_split(_p(acc_lo), _p(acc_hi), C.c_int64(M), C.c_int64(N),
+                                          C.c_float(float(s_lo)), C.c_float(float(s_hi)), _p(w_scale), _p(bias),
+                                          _p(Y)), "dequant_epilogue_split")
+    return Y
+
+
 # --------------------------------------------------------------- weight-only
 
 def weight_only_linear(X, codes, scale, zero=None, bias=None):
@@ -328,6 +343,30 @@ def conv3x3_a8_asym(X, codes, w_scale, act_scale_, act_zero: int, bias=None, str
     cx = quantize_acts_asym(X, act_scale_, act_zero)
     acc = int_conv3x3_i16(cx, codes, stride)
     return acc, dequant_epilogue(acc, act_scale_, w_scale, bias)
+
+
+def linear_a8_split(X, codes, w_scale, s_lo, s_hi, split_at: int, bias=None):
+    """Shortcut-splitting on a linear layer (Sec. 4.1): columns [0, split_at) of X are quantized with s_lo,
+    the rest with s_hi; returns (acc_lo, acc_hi, fp16 out)."""
+    X = _f16(X)
+    codes = np.ascontiguousarray(codes, np.int16)
+    q_lo = quantize_acts(np.ascontiguousarray(X[:, :split_at]), s_lo, 8)
+    q_hi = quantize_acts(np.ascontiguousarray(X[:, split_at:]), s_hi, 8)
+    acc_lo = int_gemm(q_lo, np.ascontiguousarray(codes[:, :split_at]))
+    acc_hi = int_gemm(q_hi, np.ascontiguousarray(codes[:, split_at:]))
+    return acc_lo, acc_hi, dequant_epilogue_split(acc_lo, acc_hi, s_lo, s_hi, w_scale, bias)
+
+
+def conv3x3_a8_split(X, codes, w_scale, s_lo, s_hi, split_at: int, bias=None, stride: int = 1):
+    """The same on a 3x3 convolution: X fp16 NHWC whose channels [0, split_at) and [split_at, C) come from
+    the two concatenated tensors; codes int16 [N,3,3,C]."""
+    X = _f16(X)
+    codes = np.ascontiguousarray(codes, np.int16)
+    q_lo = quantize_acts(np.ascontiguousarray(X[..., :split_at]), s_lo, 8)
+    q_hi = quantize_acts(np.ascontiguousarray(X[..., split_at:]), s_hi, 8)
+    acc_lo = int_conv3x3(q_lo, np.ascontiguousarray(codes[..., :split_at]), stride)
+    acc_hi = int_conv3x3(q_hi, np.ascontiguousarray(codes[..., split_at:]), stride)
+    return acc_lo, acc_hi, dequant_epilogue_split(acc_lo, acc_hi, s_lo, s_hi, w_scale, bias)
 
 
 def linear_a16(X, codes, scale, zero=None, bias=None):

@@ -373,6 +373,86 @@ def test_a8_conv_equals_linear_on_im2col():
     assert np.array_equal(y.reshape(-1, 5).view(np.uint16), y2.view(np.uint16))
 
 
+# ------------------------------------------------------- shortcut-splitting (Sec. 4.1)
+
+def _concat_input(M, C_lo, C_hi, seed, ratio=12.0):
+    """[hidden | skip]: two tensors of very different ranges side by side."""
+    lo = synth.normal_f16((M, C_lo), 1.0, seed=seed)
+    hi = synth.normal_f16((M, C_hi), 1.0 / ratio, seed=seed + 1)
+    return np.concatenate([lo, hi], axis=1)
+
+
+def test_split_epilogue_by_hand_and_reduction_to_unsplit():
+    a = np.array([[100, -3]], np.int32)
+    b = np.array([[7, 50]], np.int32)
+    ws = np.array([0.5, 2.0], np.float32)
+    y = orc.dequant_epilogue_split(a, b, 0.25, 0.125, ws, np.array([1.0, -1.0], np.float16))
+    # (100*0.25 + 7*0.125)*0.5 + 1 = 13.9375 ; (-3*0.25 + 50*0.125)*2 - 1 = 10
+    assert y.astype(np.float64).tolist() == [[13.9375, 10.0]]
+    # equal scales: the split layer is the unsplit one, accumulators and outputs
+    X, W, bias = synth.single_linear(seed=9, M=40, K=96, N=24)
+    ws, _ = orc.weight_minmax_params(W, 8, True)
+    codes = orc.quantize_weights(W, 8, ws, None)
+    sx = orc.act_scale(orc.act_absmax(X), 8)
+    acc, y = orc.linear_a8(X, codes, ws, sx, bias)
+    a_lo, a_hi, ys = orc.linear_a8_split(X, codes, ws, sx, sx, 32, bias)
+    assert np.array_equal(a_lo.astype(np.int64) + a_hi, acc)
+    assert np.abs(ys.astype(np.float64) - y.astype(np.float64)).max() <= 2.0 ** -10 * np.abs(y.astype(np.float64)).max()
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_split_linear_equals_fake_quant_matmul_and_gains(bits):
+    X = _concat_input(64, 80, 48, seed=50)
+    _, W, b = synth.single_linear(seed=3, M=8, K=128, N=40)
+    ws, _ = orc.weight_minmax_params(W, bits, True)
+    codes = orc.quantize_weights(W, bits, ws, None)
+    s_lo = orc.act_scale(orc.act_absmax(X[:, :80]), 8)
+    s_hi = orc.act_scale(orc.act_absmax(X[:, 80:]), 8)
+    a_lo, a_hi, y = orc.linear_a8_split(X, codes, ws, s_lo, s_hi, 80, b)
+    # brute force of one accumulator pair
+    q = np.concatenate([orc.quantize_acts(X[:, :80], s_lo, 8), orc.quantize_acts(X[:, 80:], s_hi, 8)], axis=1)
+    assert int(a_lo[5, 7]) == sum(int(q[5, k]) * int(codes[7, k]) for k in range(80))
+    assert int(a_hi[5, 7]) == sum(int(q[5, k]) * int(codes[7, k]) for k in range(80, 128))
+    xq = np.concatenate([q[:, :80] * float(s_lo), q[:, 80:] * float(s_hi)], axis=1).astype(np.float64)
+    wq = codes.astype(np.float64) * ws.astype(np.float64)[:, None]
+    ref = xq @ wq.T + b.astype(np.float64)
+    assert np.all(np.abs(y.astype(np.float64) - ref) <= 2.0 ** -10 * np.abs(ref) + 1e-7)
+    if bits == 8:
+        # one scale over the concatenation leaves the small-range half with a few levels only
+        full = X.astype(np.float64) @ wq.T + b.astype(np.float64)
+        s_all = orc.act_scale(orc.act_absmax(X), 8)
+        _, y1 = orc.linear_a8(X, codes, ws, s_all, b)
+        e_split = np.abs(y.astype(np.float64) - full).mean()
+        e_one = np.abs(y1.astype(np.float64) - full).mean()
+        # rounding noise per element ~ step^2 / 12: the hi half's step shrinks 12x, the lo half's stays
+        predicted = np.sqrt((80 + 48 / 12.0 ** 2) / 128)
+        assert abs(e_split / e_one - predicted) < 0.08
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_split_conv_equals_split_linear_on_im2col(stride):
+    B, H, W_, C_lo, C_hi, N = 2, 5, 6, 16, 8, 10
+    X = _concat_input(B * H * W_, C_lo, C_hi, seed=60).reshape(B, H, W_, C_lo + C_hi)
+    Wt = synth.normal_f16((N, 3, 3, C_lo + C_hi), 0.05, seed=61)
+    b = synth.normal_f16((N,), 0.1, seed=62)
+    ws, _ = orc.weight_minmax_params(Wt.reshape(N, -1), 8, True)
+    codes = orc.quantize_weights(Wt.reshape(N, -1), 8, ws, None).reshape(N, 3, 3, C_lo + C_hi)
+    s_lo = orc.act_scale(orc.act_absmax(X[..., :C_lo].reshape(-1, C_lo)), 8)
+    s_hi = orc.act_scale(orc.act_absmax(X[..., C_lo:].reshape(-1, C_hi)), 8)
+    a_lo, a_hi, y = orc.conv3x3_a8_split(X, codes, ws, s_lo, s_hi, C_lo, b, stride)
+    # im2col with the columns regrouped as [all lo channels of the 9 taps | all hi channels]
+    Xp = np.zeros((B, H + 2, W_ + 2, C_lo + C_hi), np.float16)
+    Xp[:, 1:-1, 1:-1, :] = X
+    Ho, Wo = a_lo.shape[1:3]
+    win = np.stack([Xp[:, ho * stride:ho * stride + 3, wo * stride:wo * stride + 3, :]
+                    for ho in range(Ho) for wo in range(Wo)], axis=1)          # [B, Ho*Wo, 3, 3, C]
+    cols = np.concatenate([win[..., :C_lo].reshape(B * Ho * Wo, -1), win[..., C_lo:].reshape(B * Ho * Wo, -1)], axis=1)
+    wcols = np.concatenate([codes[..., :C_lo].reshape(N, -1), codes[..., C_lo:].reshape(N, -1)], axis=1)
+    l_lo, l_hi, y_l = orc.linear_a8_split(cols, wcols, ws, s_lo, s_hi, 9 * C_lo, b)
+    assert np.array_equal(a_lo.reshape(-1, N), l_lo) and np.array_equal(a_hi.reshape(-1, N), l_hi)
+    assert np.array_equal(y.reshape(-1, N).view(np.uint16), y_l.view(np.uint16))
+
+
 # ----------------------------------------------------------------------- BOS
 
 def _sqnr(ref, y):
