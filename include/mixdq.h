@@ -224,6 +224,56 @@ int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H, int64_t W
                                   int32_t* acc_out, void* workspace, size_t workspace_bytes, int32_t* status,
                                   void* stream);
 
+/*
+ * Shortcut-splitting (Sec. 4.1, "Quantization Scheme"): a layer whose input is a concatenation of two
+ * branches with different ranges (the skip connections of the UNet's up path) keeps one per-tensor
+ * activation scale per branch.  Row elements [0, split_at) of X (channels, for a convolution) are
+ * quantized with *act_scale_lo, elements [split_at, K) with *act_scale_hi; each part is multiplied with its
+ * own part of the weights into an exact int32 sum, and
+ *     y[m, n] = fp16( (s_lo * acc_lo[m, n] + s_hi * acc_hi[m, n]) * w_scale[n] + bias[n] ).
+ * The weights arrive as two packed matrices made offline with mixdq_pack_weights from the two column
+ * ranges of W and the SAME per-output-channel scale (taken over the whole row): packed_W_lo is
+ * [N, split_at] and packed_W_hi [N, K - split_at]; for a convolution W[..., :split_at] and
+ * W[..., split_at:] flattened to [Cout, 9 * split_at] and [Cout, 9 * (Cin - split_at)] in (kh, kw, cin) order.
+ * Symmetric weights, w_bits in {4, 8}; symmetric activations.  NEEDS a workspace of
+ * mixdq_split_workspace_bytes(in_rows, row_len, split_at, out_rows, N) bytes, where (in_rows, row_len,
+ * out_rows) = (M, K, M) for a linear layer and (B*H*W, Cin, B*Ho*Wo) for a convolution; it holds the two
+ * int8 copies and the two int32 sums, needs no initial content, and calls sharing it must not overlap.
+ * split_at and K - split_at (Cin - split_at) must suit the two-kernel path: multiples of 16 (convolution:
+ * of 32, with an image geometry as for mixdq_conv3x3_a8_asym), ldx % 8 == 0, X 16-byte aligned;
+ * MIXDQ_ERR_UNSUPPORTED otherwise, MIXDQ_ERR_WORKSPACE when the workspace is missing or too small.
+ */
+int mixdq_split_workspace_bytes(int64_t in_rows, int64_t row_len, int64_t split_at, int64_t out_rows, int64_t N,
+                                size_t* out);
+
+int mixdq_linear_a8_split(const void* X, int64_t M, int64_t K, int64_t ldx, int64_t split_at,
+                          const void* packed_W_lo, const void* packed_W_hi, int64_t N, int w_bits,
+                          const float* w_scale, const float* act_scale_lo, const float* act_scale_hi,
+                          const void* bias, void* Y, void* workspace, size_t workspace_bytes, int32_t* status,
+                          void* stream);
+
+/* Parity hook: the two int32 sums [M, N] of a shortcut-split linear layer, before the epilogue. */
+int mixdq_linear_a8_split_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, int64_t split_at,
+                                  const void* packed_W_lo, const void* packed_W_hi, int64_t N, int w_bits,
+                                  const float* act_scale_lo, const float* act_scale_hi, int32_t* acc_lo_out,
+                                  int32_t* acc_hi_out, void* workspace, size_t workspace_bytes, int32_t* status,
+                                  void* stream);
+
+/* Shortcut-splitting on a 3x3 convolution (NHWC input whose channels [0, split_at) and [split_at, Cin) come
+ * from the two branches); other arguments as in mixdq_conv3x3 and mixdq_linear_a8_split. */
+int mixdq_conv3x3_a8_split(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, int64_t split_at,
+                           const void* packed_W_lo, const void* packed_W_hi, int64_t Cout, int stride, int w_bits,
+                           const float* w_scale, const float* act_scale_lo, const float* act_scale_hi,
+                           const void* bias, void* Y, void* workspace, size_t workspace_bytes, int32_t* status,
+                           void* stream);
+
+/* Parity hook: the two int32 sums [B, Ho, Wo, Cout] of a shortcut-split convolution. */
+int mixdq_conv3x3_a8_split_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, int64_t split_at,
+                                   const void* packed_W_lo, const void* packed_W_hi, int64_t Cout, int stride,
+                                   int w_bits, const float* act_scale_lo, const float* act_scale_hi,
+                                   int32_t* acc_lo_out, int32_t* acc_hi_out, void* workspace,
+                                   size_t workspace_bytes, int32_t* status, void* stream);
+
 /* Parity hook: int32 accumulators [B, Ho, Wo, Cout] of the int8 conv path. */
 int mixdq_conv3x3_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
                           const void* packed_W, int64_t Cout, int stride, int w_bits,

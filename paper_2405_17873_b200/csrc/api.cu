@@ -279,6 +279,137 @@ extern "C" int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H
                       nullptr, acc_out, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
 }
 
+// ---------------------------------------------------------------- shortcut-splitting (Sec. 4.1)
+
+namespace {
+
+int split_common(i8::Params& p, int amode, int64_t in_rows, int64_t row_len, int64_t split_at, const void* packed_lo,
+                 const void* packed_hi, int w_bits, const float* act_scale_lo, const float* act_scale_hi,
+                 int32_t* acc_lo_out, int32_t* acc_hi_out, void* workspace, size_t ws_bytes, void* stream)
+{
+    if (!p.X || !packed_lo || !packed_hi || !act_scale_lo || !act_scale_hi) return MIXDQ_ERR_INVALID_ARG;
+    if (p.Y ? !p.w_scale : (!acc_lo_out || !acc_hi_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (split_at <= 0 || split_at >= row_len) return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (!aligned16(packed_lo) || !aligned16(packed_hi)) return MIXDQ_ERR_ALIGNMENT;
+    if (!i8::split_path_ok(p, amode, static_cast<int>(split_at), w_bits)) return MIXDQ_ERR_UNSUPPORTED;
+    if (!workspace || ws_bytes < i8::split_layer_scratch_bytes(in_rows, row_len, split_at, p.M, p.N))
+        return MIXDQ_ERR_WORKSPACE;
+    return i8::run_tma_split(p, amode, static_cast<int>(split_at), packed_lo, packed_hi, w_bits, act_scale_lo,
+                             act_scale_hi, acc_lo_out, acc_hi_out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int linear_split_impl(const void* X, int64_t M, int64_t K, int64_t ldx, int64_t split_at, const void* packed_lo,
+                      const void* packed_hi, int64_t N, int w_bits, const float* w_scale, const float* act_scale_lo,
+                      const float* act_scale_hi, const void* bias, void* Y, int32_t* acc_lo_out,
+                      int32_t* acc_hi_out, void* workspace, size_t ws_bytes, int32_t* status, void* stream)
+{
+    if (!fits_int(M) || !fits_int(K) || !fits_int(N) || ldx < K) return MIXDQ_ERR_INVALID_ARG;
+    i8::Params p;
+    p.X = static_cast<const __half*>(X);
+    p.ldx = ldx;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.w_scale = w_scale;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = N;
+    p.status = status;
+    return split_common(p, A_LINEAR, M, K, split_at, packed_lo, packed_hi, w_bits, act_scale_lo, act_scale_hi,
+                        acc_lo_out, acc_hi_out, workspace, ws_bytes, stream);
+}
+
+int conv3_split_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, int64_t split_at,
+                     const void* packed_lo, const void* packed_hi, int64_t Cout, int stride, int w_bits,
+                     const float* w_scale, const float* act_scale_lo, const float* act_scale_hi, const void* bias,
+                     void* Y, int32_t* acc_lo_out, int32_t* acc_hi_out, void* workspace, size_t ws_bytes,
+                     int32_t* status, void* stream)
+{
+    if (!fits_int(B) || !fits_int(H) || !fits_int(W) || !fits_int(Cin) || !fits_int(Cout))
+        return MIXDQ_ERR_INVALID_ARG;
+    if (stride != 1 && stride != 2) return MIXDQ_ERR_INVALID_ARG;
+    const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    if (!fits_int(B * Ho * Wo) || !fits_int(9 * Cin) || !fits_int(B * H * W * Cin)) return MIXDQ_ERR_INVALID_ARG;
+    i8::Params p;
+    p.X = static_cast<const __half*>(X);
+    p.ldx = 8;
+    p.M = static_cast<int>(B * Ho * Wo);
+    p.N = static_cast<int>(Cout);
+    p.K = static_cast<int>(9 * Cin);
+    p.H = static_cast<int>(H);
+    p.W = static_cast<int>(W);
+    p.Cin = static_cast<int>(Cin);
+    p.Ho = static_cast<int>(Ho);
+    p.Wo = static_cast<int>(Wo);
+    p.stride = stride;
+    p.batch = static_cast<int>(B);
+    p.w_scale = w_scale;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = Cout;
+    p.status = status;
+    return split_common(p, A_CONV3, B * H * W, Cin, split_at, packed_lo, packed_hi, w_bits, act_scale_lo,
+                        act_scale_hi, acc_lo_out, acc_hi_out, workspace, ws_bytes, stream);
+}
+
+}  // namespace
+
+extern "C" int mixdq_split_workspace_bytes(int64_t in_rows, int64_t row_len, int64_t split_at, int64_t out_rows,
+                                           int64_t N, size_t* out)
+{
+    if (!out || in_rows <= 0 || out_rows <= 0 || N <= 0 || split_at <= 0 || split_at >= row_len)
+        return MIXDQ_ERR_INVALID_ARG;
+    *out = i8::split_layer_scratch_bytes(in_rows, row_len, split_at, out_rows, N);
+    return MIXDQ_OK;
+}
+
+extern "C" int mixdq_linear_a8_split(const void* X, int64_t M, int64_t K, int64_t ldx, int64_t split_at,
+                                     const void* packed_W_lo, const void* packed_W_hi, int64_t N, int w_bits,
+                                     const float* w_scale, const float* act_scale_lo, const float* act_scale_hi,
+                                     const void* bias, void* Y, void* workspace, size_t workspace_bytes,
+                                     int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return linear_split_impl(X, M, K, ldx, split_at, packed_W_lo, packed_W_hi, N, w_bits, w_scale, act_scale_lo,
+                             act_scale_hi, bias, Y, nullptr, nullptr, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int mixdq_linear_a8_split_acc_i32(const void* X, int64_t M, int64_t K, int64_t ldx, int64_t split_at,
+                                             const void* packed_W_lo, const void* packed_W_hi, int64_t N,
+                                             int w_bits, const float* act_scale_lo, const float* act_scale_hi,
+                                             int32_t* acc_lo_out, int32_t* acc_hi_out, void* workspace,
+                                             size_t workspace_bytes, int32_t* status, void* stream)
+{
+    return linear_split_impl(X, M, K, ldx, split_at, packed_W_lo, packed_W_hi, N, w_bits, nullptr, act_scale_lo,
+                             act_scale_hi, nullptr, nullptr, acc_lo_out, acc_hi_out, workspace, workspace_bytes,
+                             status, stream);
+}
+
+extern "C" int mixdq_conv3x3_a8_split(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, int64_t split_at,
+                                      const void* packed_W_lo, const void* packed_W_hi, int64_t Cout, int stride,
+                                      int w_bits, const float* w_scale, const float* act_scale_lo,
+                                      const float* act_scale_hi, const void* bias, void* Y, void* workspace,
+                                      size_t workspace_bytes, int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return conv3_split_impl(X, B, H, W, Cin, split_at, packed_W_lo, packed_W_hi, Cout, stride, w_bits, w_scale,
+                            act_scale_lo, act_scale_hi, bias, Y, nullptr, nullptr, workspace, workspace_bytes,
+                            status, stream);
+}
+
+extern "C" int mixdq_conv3x3_a8_split_acc_i32(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin,
+                                              int64_t split_at, const void* packed_W_lo, const void* packed_W_hi,
+                                              int64_t Cout, int stride, int w_bits, const float* act_scale_lo,
+                                              const float* act_scale_hi, int32_t* acc_lo_out, int32_t* acc_hi_out,
+                                              void* workspace, size_t workspace_bytes, int32_t* status,
+                                              void* stream)
+{
+    return conv3_split_impl(X, B, H, W, Cin, split_at, packed_W_lo, packed_W_hi, Cout, stride, w_bits, nullptr,
+                            act_scale_lo, act_scale_hi, nullptr, nullptr, acc_lo_out, acc_hi_out, workspace,
+                            workspace_bytes, status, stream);
+}
+
 extern "C" int mixdq_conv3x3(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
                              int64_t Cout, int stride, int w_bits, const float* w_scale,
                              const int32_t* w_zero, int act_bits, const float* act_scale, const void* bias,

@@ -51,6 +51,14 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
 // Two-kernel path (quantize once, then a TMA-fed GEMM); see i8_tma.cu.
 bool tma_path_ok(const Params& p, int amode, int w_bits);
 int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream);
+// Shortcut-splitting (one activation scale per branch of a concatenated input): row elements [0, split_at)
+// and [split_at, row_len) are quantized, multiplied and summed separately and meet in a two-scale epilogue.
+// Linear layers and 3x3 convolutions whose halves both suit the two-kernel path.
+size_t split_layer_scratch_bytes(int64_t in_rows, int64_t row_len, int64_t split_at, int64_t out_rows, int64_t N);
+bool split_path_ok(const Params& p, int amode, int split_at, int w_bits);
+int run_tma_split(const Params& p, int amode, int split_at, const void* packed_lo, const void* packed_hi, int w_bits,
+                  const float* scale_lo, const float* scale_hi, int32_t* acc_lo_out, int32_t* acc_hi_out,
+                  void* scratch, cudaStream_t stream);
 
 }  // namespace i8
 

@@ -118,6 +118,69 @@ __global__ void quant_pad_kernel(const __half* __restrict__ X, int B, int H, int
     *reinterpret_cast<uint4*>(out + pix * Cin + c * 16) = o;
 }
 
+// Shortcut-splitting (Sec. 4.1): the input of a layer fed by a concatenation keeps one scale per branch.
+// Columns [0, split) of every row are quantized with *scale_lo into the dense matrix out_lo [rows, split],
+// columns [split, K) with *scale_hi into out_hi [rows, K - split].  split and K are multiples of 16, so a
+// thread's 16 elements lie on one side.
+__global__ void quant_split_kernel(const __half* __restrict__ X, long long ldx, long long rows, int K, int split,
+                                   const float* __restrict__ scale_lo, const float* __restrict__ scale_hi,
+                                   int8_t* __restrict__ out_lo, int8_t* __restrict__ out_hi)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int cpr = K >> 4;
+    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    if (idx >= rows * cpr) return;
+    const long long r = idx / cpr;
+    const int c = static_cast<int>(idx - r * cpr) * 16;
+    const bool hi_side = c >= split;
+    const float inv = __fdiv_rn(1.f, __ldg(hi_side ? scale_hi : scale_lo));
+    const uint4 q = quantize16(X + r * ldx + c, inv, kMagic - 127.f, kMagic + 127.f, 0u);
+    int8_t* dst = hi_side ? out_hi + r * (K - split) + (c - split) : out_lo + r * split + c;
+    *reinterpret_cast<uint4*>(dst) = q;
+}
+
+// The epilogue of a shortcut-split layer: y = fp16((s_lo * acc_lo + s_hi * acc_hi) * s_w[n] + bias[n]) from the
+// two branches' exact int32 sums.  One thread per four consecutive columns (N % 4 == 0) or per element.
+__global__ void combine_split_kernel(const int32_t* __restrict__ acc_lo, const int32_t* __restrict__ acc_hi,
+                                     long long M, int N, const float* __restrict__ scale_lo,
+                                     const float* __restrict__ scale_hi, const float* __restrict__ w_scale,
+                                     const __half* __restrict__ bias, __half* __restrict__ Y, long long ldy)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const float s_lo = __ldg(scale_lo), s_hi = __ldg(scale_hi);
+    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    if ((N & 3) == 0 && (ldy & 3) == 0) {
+        const int gpr = N >> 2;
+        if (idx >= M * gpr) return;
+        const long long m = idx / gpr;
+        const int n = static_cast<int>(idx - m * gpr) * 4;
+        const int4 a = *reinterpret_cast<const int4*>(acc_lo + m * N + n);
+        const int4 b = *reinterpret_cast<const int4*>(acc_hi + m * N + n);
+        const float4 w = __ldg(reinterpret_cast<const float4*>(w_scale + n));
+        float bs[4] = {0.f, 0.f, 0.f, 0.f};
+        if (bias) {
+            const uint2 raw = __ldg(reinterpret_cast<const uint2*>(bias + n));
+            const __half2* hb = reinterpret_cast<const __half2*>(&raw);
+            const float2 b0 = __half22float2(hb[0]), b1 = __half22float2(hb[1]);
+            bs[0] = b0.x; bs[1] = b0.y; bs[2] = b1.x; bs[3] = b1.y;
+        }
+        __half2 h[2];
+        h[0] = __floats2half2_rn(fmaf(fmaf(static_cast<float>(a.x), s_lo, static_cast<float>(b.x) * s_hi), w.x, bs[0]),
+                                 fmaf(fmaf(static_cast<float>(a.y), s_lo, static_cast<float>(b.y) * s_hi), w.y, bs[1]));
+        h[1] = __floats2half2_rn(fmaf(fmaf(static_cast<float>(a.z), s_lo, static_cast<float>(b.z) * s_hi), w.z, bs[2]),
+                                 fmaf(fmaf(static_cast<float>(a.w), s_lo, static_cast<float>(b.w) * s_hi), w.w, bs[3]));
+        *reinterpret_cast<uint2*>(Y + m * ldy + n) = *reinterpret_cast<const uint2*>(h);
+        return;
+    }
+    if (idx >= M * N) return;
+    const long long m = idx / N;
+    const int n = static_cast<int>(idx - m * N);
+    const float v = fmaf(static_cast<float>(acc_lo[idx]), s_lo, static_cast<float>(acc_hi[idx]) * s_hi);
+    Y[m * ldy + n] = __float2half_rn(fmaf(v, __ldg(w_scale + n), bias ? __half2float(bias[n]) : 0.f));
+}
+
 // Barrier over all threads of all CTAs of the cluster (hardware barrier, not a spin).
 __device__ __forceinline__ void cluster_sync_all()
 {
@@ -1190,10 +1253,12 @@ bool tma_path_ok(const Params& p, int amode, int w_bits)
     return p.K % 16 == 0 && p.ldx % 8 == 0 && (reinterpret_cast<uintptr_t>(p.X) & 15) == 0;
 }
 
+// Step 2 of the two-kernel path: the TMA-fed GEMM (or implicit-GEMM convolution) on int8 activations `aq`
+// that an earlier kernel of the stream has written ([M, K] dense, or the NHWC image, padded when p.act_zero).
+static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bits, int8_t* aq, cudaStream_t stream);
+
 int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream)
 {
-    const bool w4 = w_bits == 4;
-    const int64_t pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
     int8_t* aq = static_cast<int8_t*>(scratch);
 
     // 1. quantize the activations once
@@ -1211,6 +1276,16 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
         rc = launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
                         p.X, ldx, in_rows, row_len, amode == A_BOS ? 1 : 0, p.act_scale, p.act_zero, aq);
     if (rc != MIXDQ_OK) return rc;
+    return run_tma_gemm(p, amode, packed, w_bits, aq, stream);
+}
+
+static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bits, int8_t* aq, cudaStream_t stream)
+{
+    const bool w4 = w_bits == 4;
+    const int64_t pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
+    const bool conv = amode == A_CONV3;
+    const int pad = (conv && p.act_zero) ? 1 : 0;
+    int rc;
 
     // 2. tensor maps
     CUtensorMap ta, tw, ty{};
@@ -1296,6 +1371,84 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
     if (wide) return launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
     return w4 ? launch_tma<128, 6, true>(ta, tw, ty, tp, splits, stream)
               : launch_tma<128, 6, false>(ta, tw, ty, tp, splits, stream);
+}
+
+// Layout of the shortcut-split scratch: [int8 lo | int8 hi | int32 sums lo | int32 sums hi], each 256-byte aligned.
+size_t split_layer_scratch_bytes(int64_t in_rows, int64_t row_len, int64_t split_at, int64_t out_rows, int64_t N)
+{
+    return static_cast<size_t>(round_up(in_rows * split_at, 256) + round_up(in_rows * (row_len - split_at), 256) +
+                               2 * round_up(out_rows * N * 4, 256));
+}
+
+bool split_path_ok(const Params& p, int amode, int split_at, int w_bits)
+{
+    if (amode != A_LINEAR && amode != A_CONV3) return false;
+    const int row_len = amode == A_CONV3 ? p.Cin : p.K;
+    if (split_at <= 0 || split_at >= row_len || split_at % 16 != 0 || row_len % 16 != 0) return false;
+    if ((reinterpret_cast<uintptr_t>(p.X) & 15) != 0) return false;
+    Params lo = p, hi = p;
+    if (amode == A_CONV3) {
+        lo.Cin = split_at;
+        hi.Cin = row_len - split_at;
+        lo.K = 9 * lo.Cin;
+        hi.K = 9 * hi.Cin;
+    } else {
+        if (p.ldx % 8 != 0) return false;
+        lo.K = split_at;
+        hi.K = row_len - split_at;
+    }
+    return tma_path_ok(lo, amode, w_bits) && tma_path_ok(hi, amode, w_bits);
+}
+
+// Shortcut-splitting (Sec. 4.1): one quantization pass with a scale per branch, one int8 GEMM (or implicit-GEMM
+// convolution) per branch into exact int32 sums, and the two-scale epilogue.  acc_lo_out / acc_hi_out: where
+// the sums go (nullptr: into the scratch); p.Y == nullptr: sums only.
+int run_tma_split(const Params& p, int amode, int split_at, const void* packed_lo, const void* packed_hi, int w_bits,
+                  const float* scale_lo, const float* scale_hi, int32_t* acc_lo_out, int32_t* acc_hi_out,
+                  void* scratch, cudaStream_t stream)
+{
+    const bool conv = amode == A_CONV3;
+    const long long in_rows = conv ? static_cast<long long>(p.batch) * p.H * p.W : p.M;
+    const int row_len = conv ? p.Cin : p.K;
+    const long long ldx = conv ? p.Cin : p.ldx;
+    uint8_t* base = static_cast<uint8_t*>(scratch);
+    int8_t* aq_lo = reinterpret_cast<int8_t*>(base);
+    base += round_up(in_rows * split_at, 256);
+    int8_t* aq_hi = reinterpret_cast<int8_t*>(base);
+    base += round_up(in_rows * (row_len - split_at), 256);
+    const long long acc_bytes = round_up(static_cast<long long>(p.M) * p.N * 4, 256);
+    int32_t* acc_lo = acc_lo_out ? acc_lo_out : reinterpret_cast<int32_t*>(base);
+    int32_t* acc_hi = acc_hi_out ? acc_hi_out : reinterpret_cast<int32_t*>(base + acc_bytes);
+
+    const long long tasks = in_rows * (row_len / 16);
+    int rc = launch_pdl(quant_split_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
+                        p.X, ldx, in_rows, row_len, split_at, scale_lo, scale_hi, aq_lo, aq_hi);
+    if (rc != MIXDQ_OK) return rc;
+
+    Params q = p;
+    q.Y = nullptr;
+    q.bias = nullptr;
+    q.act_zero = nullptr;
+    q.w_code_sums = nullptr;
+    q.force_splits = 0;
+    q.acc_out = acc_lo;
+    q.act_scale = scale_lo;
+    q.Cin = conv ? split_at : 0;
+    q.K = conv ? 9 * split_at : split_at;
+    rc = run_tma_gemm(q, amode, packed_lo, w_bits, aq_lo, stream);
+    if (rc != MIXDQ_OK) return rc;
+    q.acc_out = acc_hi;
+    q.act_scale = scale_hi;
+    q.Cin = conv ? row_len - split_at : 0;
+    q.K = conv ? 9 * (row_len - split_at) : row_len - split_at;
+    rc = run_tma_gemm(q, amode, packed_hi, w_bits, aq_hi, stream);
+    if (rc != MIXDQ_OK || !p.Y) return rc;
+
+    const bool vec = p.N % 4 == 0 && p.ldy % 4 == 0;
+    const long long work = static_cast<long long>(p.M) * (vec ? p.N / 4 : p.N);
+    const long long M = p.M;
+    return launch_pdl(combine_split_kernel, dim3(static_cast<unsigned>(ceil_div(work, 256))), dim3(256), 0, stream, 1,
+                      acc_lo, acc_hi, M, p.N, scale_lo, scale_hi, p.w_scale, p.bias, p.Y, p.ldy);
 }
 
 }  // namespace i8

@@ -42,6 +42,15 @@ _SIGNATURES = {
                                      _vp, _vp, _sz, _vp, _vp]),
     "mixdq_conv3x3_a8_asym_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp,
                                              _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_split_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, C.POINTER(_sz)]),
+    "mixdq_linear_a8_split": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp,
+                                     _sz, _vp, _vp]),
+    "mixdq_linear_a8_split_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _vp, _vp, _vp, _vp,
+                                             _vp, _sz, _vp, _vp]),
+    "mixdq_conv3x3_a8_split": (_int, [_vp, _i64, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _int, _vp, _vp, _vp,
+                                      _vp, _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_conv3x3_a8_split_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _int, _vp, _vp,
+                                              _vp, _vp, _vp, _sz, _vp, _vp]),
     "mixdq_workspace_bytes": (_int, [_i64, _i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_conv3x3_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, _int, _int, _int, C.POINTER(_sz)]),
     "mixdq_linear": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _int, _vp, _vp, _vp, _vp, _sz,
@@ -290,6 +299,64 @@ def conv3x3_a8_asym_acc_i32(X, packed_W, Cout: int, w_bits: int, w_code_sums, ac
                                              _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(acc), wp,
                                              wb, _ptr(status), _stream()), "mixdq_conv3x3_a8_asym_acc_i32")
     return acc
+
+
+def split_workspace_bytes(in_rows: int, row_len: int, split_at: int, out_rows: int, N: int) -> int:
+    out = _sz(0)
+    _chk(lib().mixdq_split_workspace_bytes(in_rows, row_len, split_at, out_rows, N, C.byref(out)),
+         "mixdq_split_workspace_bytes")
+    return out.value
+
+
+def linear_a8_split(X, split_at: int, packed_W_lo, packed_W_hi, N: int, w_bits: int, w_scale, act_scale_lo,
+                    act_scale_hi, bias=None, workspace=None, status=None, out=None):
+    M, K = X.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear_a8_split(_ptr(X), M, K, X.stride(0), split_at, _ptr(packed_W_lo), _ptr(packed_W_hi), N,
+                                     w_bits, _ptr(w_scale), _ptr(act_scale_lo), _ptr(act_scale_hi), _ptr(bias),
+                                     _ptr(Y), wp, wb, _ptr(status), _stream()), "mixdq_linear_a8_split")
+    return Y
+
+
+def linear_a8_split_acc_i32(X, split_at: int, packed_W_lo, packed_W_hi, N: int, w_bits: int, act_scale_lo,
+                            act_scale_hi, workspace=None, status=None):
+    M, K = X.shape
+    lo = torch.empty((M, N), dtype=torch.int32, device=X.device)
+    hi = torch.empty((M, N), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_linear_a8_split_acc_i32(_ptr(X), M, K, X.stride(0), split_at, _ptr(packed_W_lo),
+                                             _ptr(packed_W_hi), N, w_bits, _ptr(act_scale_lo), _ptr(act_scale_hi),
+                                             _ptr(lo), _ptr(hi), wp, wb, _ptr(status), _stream()),
+         "mixdq_linear_a8_split_acc_i32")
+    return lo, hi
+
+
+def conv3x3_a8_split(X, split_at: int, packed_W_lo, packed_W_hi, Cout: int, w_bits: int, w_scale, act_scale_lo,
+                     act_scale_hi, bias=None, stride: int = 1, workspace=None, status=None, out=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    Y = out if out is not None else torch.empty((B, Ho, Wo, Cout), dtype=torch.float16, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3_a8_split(_ptr(X), B, H, W, Cin, split_at, _ptr(packed_W_lo), _ptr(packed_W_hi), Cout,
+                                      stride, w_bits, _ptr(w_scale), _ptr(act_scale_lo), _ptr(act_scale_hi),
+                                      _ptr(bias), _ptr(Y), wp, wb, _ptr(status), _stream()),
+         "mixdq_conv3x3_a8_split")
+    return Y
+
+
+def conv3x3_a8_split_acc_i32(X, split_at: int, packed_W_lo, packed_W_hi, Cout: int, w_bits: int, act_scale_lo,
+                             act_scale_hi, stride: int = 1, workspace=None, status=None):
+    B, H, W, Cin = X.shape
+    Ho, Wo = _out_hw(H, W, stride)
+    lo = torch.empty((B, Ho, Wo, Cout), dtype=torch.int32, device=X.device)
+    hi = torch.empty((B, Ho, Wo, Cout), dtype=torch.int32, device=X.device)
+    wp, wb = _ws(workspace)
+    _chk(lib().mixdq_conv3x3_a8_split_acc_i32(_ptr(X), B, H, W, Cin, split_at, _ptr(packed_W_lo),
+                                              _ptr(packed_W_hi), Cout, stride, w_bits, _ptr(act_scale_lo),
+                                              _ptr(act_scale_hi), _ptr(lo), _ptr(hi), wp, wb, _ptr(status),
+                                              _stream()), "mixdq_conv3x3_a8_split_acc_i32")
+    return lo, hi
 
 
 def conv3x3_acc_i32(X, packed_W, Cout: int, w_bits: int, act_scale, stride: int = 1, workspace=None,

@@ -184,6 +184,22 @@ def unet_layers() -> List[LayerSpec]:
     return L
 
 
+# hidden-state channels of the layers fed by [hidden | skip] concatenations in the up path, by input width
+_CONCAT_HIDDEN = {2560: 1280, 1920: 1280, 1280: 640, 960: 640, 640: 320}
+
+
+def shortcut_split_at(l: LayerSpec) -> int:
+    """Channel at which the input of a resnet convolution (3x3 or its 1x1 shortcut) of the up path splits into
+    the hidden state and the skip connection it was concatenated with (Sec. 4.1, shortcut-splitting); 0 for a
+    layer that is not fed by a concatenation.  In this architecture those are the resnet layers that narrow
+    their input (Cin > Cout)."""
+    if l.kind not in ("conv3x3", "conv1x1") or not (l.name.startswith("res") or l.name.startswith("sc")):
+        return 0
+    if l.Cin <= l.N:
+        return 0
+    return _CONCAT_HIDDEN.get(l.Cin, 0)
+
+
 def assign_bits_weight_only(layers: List[LayerSpec], seed: int = 5, target: float = 3.66,
                             frac8: float = 0.02, low: int = 3) -> None:
     """Seeded A16 table whose parameter-weighted mean weight width is ~3.66 bits

@@ -27,18 +27,24 @@ class PackedLayer:
     x_key: tuple
     y_key: tuple
     code_sums: Optional[torch.Tensor] = None   # asymmetric activations: per-channel sums of the weight codes
+    split_at: int = 0                          # shortcut-splitting: `packed` holds input channels [0, split_at) ...
+    packed_hi: Optional[torch.Tensor] = None   # ... and this the rest
 
 
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
                  layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False,
-                 low_bits: int = 3):
+                 low_bits: int = 3, shortcut_split: bool = False):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
         (whatever the image size), so that a layer is one stream over its packed weights.
         act_asym: the 8-bit activations of the linear layers and 3x3 convolutions are asymmetric (Sec. 4.1);
         the BOS-aware K/V projections keep symmetric ones.
-        low_bits: lowest width of the a16 table (3, or 2 for the paper's candidate widths {2, 4, 8})."""
+        low_bits: lowest width of the a16 table (3, or 2 for the paper's candidate widths {2, 4, 8}).
+        shortcut_split: the A8 resnet convolutions (3x3 and 1x1) of the up path, whose input is a concatenation
+        [hidden | skip], keep one activation scale per branch (Sec. 4.1); symmetric activations."""
         assert table in ("w4a8", "a16")
+        assert not (act_asym and shortcut_split)
+        self.shortcut_split = shortcut_split
         self.batch = batch
         self.act_asym = act_asym
         self.tokens = tokens
@@ -56,6 +62,7 @@ class UNetSweep:
         self.y: Dict[tuple, torch.Tensor] = {}
         self.x_scale: Dict[tuple, torch.Tensor] = {}
         self.x_asym: Dict[tuple, tuple] = {}
+        self.x_split_scale: Dict[tuple, tuple] = {}
         self.layers: List[PackedLayer] = []
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self._build(seed)
@@ -113,8 +120,24 @@ class UNetSweep:
                 sums = mixdq.weight_code_sums(packed, l.N, l.K, l.w_bits)
                 if xk not in self.x_asym:
                     self.x_asym[xk] = mixdq.act_asym_params(self.x[xk].reshape(-1, xk[-1]))
-            self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk, sums))
-            if l.kind == "conv3x3":
+            split_at = synth.shortcut_split_at(l) if (self.shortcut_split and l.a_bits == 8) else 0
+            packed_hi = None
+            if split_at:
+                # the two channel ranges of the weights, packed apart with the scale of the whole row
+                taps = l.K // l.Cin
+                W3 = W.view(l.N, taps, l.Cin)
+                packed = mixdq.pack_weights(W3[:, :, :split_at].reshape(l.N, -1).contiguous(), l.w_bits, s)
+                packed_hi = mixdq.pack_weights(W3[:, :, split_at:].reshape(l.N, -1).contiguous(), l.w_bits, s)
+                if (xk, split_at) not in self.x_split_scale:
+                    x2 = self.x[xk].reshape(-1, l.Cin)
+                    self.x_split_scale[(xk, split_at)] = (mixdq.act_scale(x2[:, :split_at].contiguous()),
+                                                          mixdq.act_scale(x2[:, split_at:].contiguous()))
+            self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk, sums, split_at,
+                                           packed_hi))
+            if split_at:
+                out_rows = yk[0] * yk[1] * yk[2]
+                need = mixdq.split_workspace_bytes(self.batch * l.H * l.H, l.Cin, split_at, out_rows, l.N)
+            elif l.kind == "conv3x3":
                 need = mixdq.conv3x3_workspace_bytes(self.batch, l.H, l.H, l.Cin, l.N, l.stride, l.w_bits, l.a_bits)
             else:
                 rows = yk[0] * (yk[1] if len(yk) > 2 else 1) * (yk[2] if len(yk) > 3 else 1)
@@ -131,6 +154,13 @@ class UNetSweep:
         x, y = self.x[pl.x_key], self.y[pl.y_key]
         sx = self.x_scale.get(pl.x_key) if l.a_bits == 8 else None
         ws = workspace if workspace is not None else self.workspace
+        if pl.split_at:
+            s_lo, s_hi = self.x_split_scale[(pl.x_key, pl.split_at)]
+            if l.kind == "conv3x3":
+                return mixdq.conv3x3_a8_split(x, pl.split_at, pl.packed, pl.packed_hi, l.N, l.w_bits, pl.w_scale, s_lo,
+                                              s_hi, pl.bias, l.stride, ws, self.status, out=y)
+            return mixdq.linear_a8_split(x.reshape(-1, l.Cin), pl.split_at, pl.packed, pl.packed_hi, l.N, l.w_bits,
+                                         pl.w_scale, s_lo, s_hi, pl.bias, ws, self.status, out=y.reshape(-1, l.N))
         if l.kind == "conv3x3" and pl.code_sums is not None:
             ax, az = self.x_asym[pl.x_key]
             return mixdq.conv3x3_a8_asym(x, pl.packed, l.N, l.w_bits, pl.w_scale, pl.code_sums, ax, az, pl.bias,
@@ -161,14 +191,14 @@ class UNetSweep:
         return sum(pl.spec.ops(self.batch) for pl in group)
 
     def packed_weight_bytes(self) -> int:
-        return sum(pl.packed.numel() for pl in self.layers)
+        return sum(pl.packed.numel() + (0 if pl.packed_hi is None else pl.packed_hi.numel()) for pl in self.layers)
 
     def algorithmic_bytes(self, pl: PackedLayer) -> int:
         """Packed weights + per-channel params + input once + output once + bias."""
         l = pl.spec
         x, y = self.x[pl.x_key], self.y[pl.y_key]
         params = l.N * (4 if pl.w_zero is None else 8)
-        return pl.packed.numel() + params + x.numel() * 2 + y.numel() * 2 + (0 if pl.bias is None else l.N * 2)
+        return pl.packed.numel() + (0 if pl.packed_hi is None else pl.packed_hi.numel()) + params + x.numel() * 2 + y.numel() * 2 + (0 if pl.bias is None else l.N * 2)
 
     def uses_tensor_int8(self, pl: PackedLayer) -> bool:
         """True when the layer runs on the tcgen05 int8 engine (not the plain corner kernel)."""
@@ -197,6 +227,8 @@ def _main(argv=None) -> int:
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--tokens", type=int, default=0, help="linear layers only: run on this many rows (weight-bound regime)")
     ap.add_argument("--act-asym", action="store_true", help="asymmetric 8-bit activations (linear layers and 3x3 convolutions)")
+    ap.add_argument("--shortcut-split", action="store_true",
+                    help="one activation scale per branch for the concatenation-fed resnet convolutions of the up path")
     ap.add_argument("--eager", action="store_true", help="plain launches only, no graph and no timing")
     a = ap.parse_args(argv)
 
@@ -207,7 +239,8 @@ def _main(argv=None) -> int:
         raise SystemExit(f"no layer named {a.layer!r}")
     if a.w_bits is not None:
         pick[0].w_bits = a.w_bits
-    sw = UNetSweep(a.batch, a.table, layers=pick, tokens=a.tokens, act_asym=a.act_asym)
+    sw = UNetSweep(a.batch, a.table, layers=pick, tokens=a.tokens, act_asym=a.act_asym,
+                   shortcut_split=a.shortcut_split)
     pl = sw.layers[0]
     for _ in range(a.reps):
         sw.run_layer(pl)
