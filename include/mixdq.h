@@ -225,6 +225,30 @@ int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H, int64_t W
                                   void* stream);
 
 /*
+ * Activations stored as int8 between layers (the activation-memory saving of Sec. 4.3 / Table 2: an 8-bit
+ * activation tensor is kept as its codes plus one scale).  The two steps of mixdq_linear with act_bits = 8
+ * as calls of their own:
+ *   mixdq_quantize_acts: Xq_out[r, k] = clamp(rne(X[r, k] / *act_scale), -127, 127) as a dense int8
+ *     [rows, K] matrix (the symmetric per-tensor activation quantizer of Sec. 4.1; the paper's separate
+ *     quantization kernel).  K % 16 == 0, ldx % 8 == 0 (MIXDQ_ERR_UNSUPPORTED otherwise), both pointers
+ *     16-byte aligned.
+ *   mixdq_linear_q8: Y = fp16(*act_scale * w_scale[n] * sum_k Xq[m, k] * qw[n, k] + bias[n]) on such codes
+ *     (dense [M, K], 16-byte aligned, K % 16 == 0).  Several layers that read the same tensor (the q, k and v
+ *     projections of self-attention) then share one quantization pass.  Needs no workspace.  Symmetric
+ *     weights, w_bits in {4, 8}.
+ */
+int mixdq_quantize_acts(const void* X, int64_t rows, int64_t K, int64_t ldx, const float* act_scale, void* Xq_out,
+                        void* stream);
+
+int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
+                    const float* w_scale, const float* act_scale, const void* bias, void* Y, int32_t* status,
+                    void* stream);
+
+/* Parity hook: int32 accumulators [M, N] of mixdq_linear_q8. */
+int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
+                            int32_t* acc_out, int32_t* status, void* stream);
+
+/*
  * Shortcut-splitting (Sec. 4.1, "Quantization Scheme"): a layer whose input is a concatenation of two
  * branches with different ranges (the skip connections of the UNet's up path) keeps one per-tensor
  * activation scale per branch.  Row elements [0, split_at) of X (channels, for a convolution) are

@@ -279,6 +279,63 @@ extern "C" int mixdq_conv3x3_a8_asym_acc_i32(const void* X, int64_t B, int64_t H
                       nullptr, acc_out, workspace, workspace_bytes, status, stream, act_zero, w_code_sums);
 }
 
+// ---------------------------------------------------------------- int8 activations kept between layers
+
+extern "C" int mixdq_quantize_acts(const void* X, int64_t rows, int64_t K, int64_t ldx, const float* act_scale,
+                                   void* Xq_out, void* stream)
+{
+    if (!X || !act_scale || !Xq_out || !fits_int(rows) || !fits_int(K) || ldx < K) return MIXDQ_ERR_INVALID_ARG;
+    if (K % 16 != 0 || ldx % 8 != 0) return MIXDQ_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(Xq_out)) return MIXDQ_ERR_ALIGNMENT;
+    return i8::run_quant(static_cast<const __half*>(X), ldx, rows, static_cast<int>(K), act_scale,
+                         static_cast<int8_t*>(Xq_out), static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+
+int linear_q8_impl(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
+                   const float* w_scale, const float* act_scale, const void* bias, void* Y, int32_t* acc_out,
+                   int32_t* status, void* stream)
+{
+    if (!Xq || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(M) || !fits_int(K) || !fits_int(N)) return MIXDQ_ERR_INVALID_ARG;
+    if (Y && (!w_scale || !act_scale)) return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (K % 16 != 0) return MIXDQ_ERR_UNSUPPORTED;
+    if (!aligned16(packed_W) || !aligned16(Xq)) return MIXDQ_ERR_ALIGNMENT;
+    i8::Params p;
+    p.ldx = K;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.act_scale = act_scale;
+    p.w_scale = w_scale;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = N;
+    p.acc_out = acc_out;
+    p.status = status;
+    return i8::run_tma_prequantized(p, A_LINEAR, packed_W, w_bits, static_cast<const int8_t*>(Xq),
+                                    static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+
+extern "C" int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
+                               const float* w_scale, const float* act_scale, const void* bias, void* Y,
+                               int32_t* status, void* stream)
+{
+    if (!Y) return MIXDQ_ERR_INVALID_ARG;
+    return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, w_scale, act_scale, bias, Y, nullptr, status, stream);
+}
+
+extern "C" int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N,
+                                       int w_bits, int32_t* acc_out, int32_t* status, void* stream)
+{
+    if (!acc_out) return MIXDQ_ERR_INVALID_ARG;
+    return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, nullptr, nullptr, nullptr, nullptr, acc_out, status, stream);
+}
+
 // ---------------------------------------------------------------- shortcut-splitting (Sec. 4.1)
 
 namespace {

@@ -51,6 +51,12 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
 // Two-kernel path (quantize once, then a TMA-fed GEMM); see i8_tma.cu.
 bool tma_path_ok(const Params& p, int amode, int w_bits);
 int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream);
+// The two steps as calls of their own, for activations that are stored as int8 between layers: the codes of
+// X [rows, K] into a dense int8 matrix, and the GEMM / implicit-GEMM convolution on such codes (p.X unused).
+int run_quant(const __half* X, long long ldx, long long rows, int K, const float* act_scale, int8_t* out,
+              cudaStream_t stream);
+int run_tma_prequantized(const Params& p, int amode, const void* packed, int w_bits, const int8_t* aq,
+                         cudaStream_t stream);
 // Shortcut-splitting (one activation scale per branch of a concatenated input): row elements [0, split_at)
 // and [split_at, row_len) are quantized, multiplied and summed separately and meet in a two-scale epilogue.
 // Linear layers and 3x3 convolutions whose halves both suit the two-kernel path.

@@ -781,7 +781,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             // -------------------------------------------------------- epilogue warps
             // while the main loop runs: per-column dequantization factors of this tile, and the
             // stored BOS rows
-            const float sx = __ldg(p.act_scale);
+            const float sx = p.act_scale ? __ldg(p.act_scale) : 0.f;  // absent: accumulators only
             const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
             for (int j = tid - 64; j < BN; j += 128) {
                 const int n = n0 + j;
@@ -1072,7 +1072,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         const int lg = warp & 3;
         const int half = warp < 6 ? 0 : 1;
         const int et = tid - 64;  // epilogue warps only: 0..127
-        const float sx = __ldg(p.act_scale);
+        const float sx = p.act_scale ? __ldg(p.act_scale) : 0.f;  // absent: accumulators only
         const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
         bool ok = true;
         for (int t = 0; t < my_tiles; ++t) {
@@ -1121,9 +1121,15 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                 continue;
             }
             const uint32_t acc = tmem_base + buf * L::ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
-            if (p.acc_out && half == 0) {
-                // parity hook: raw accumulators, one row per thread
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+            if (p.acc_out) {
+                // raw int32 sums (parity hook; the branches of a shortcut-split layer): each half of the warps takes
+                // its half of the columns, 16 at a time through the warp's staging tile (64-byte rows, 80 bytes
+                // apart), so that four lanes store one row's 64 contiguous bytes
+                const int cbeg = half * (BN / 2);
+                uint8_t* stage = smem + L::OFF_EPI + (half * 4 + lg) * EPI32_TILE;
+                const bool vec = ((p.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
+                if (p.tma_store && lane == 0) tma_store_wait_read();  // an output store may still read the tile
+                for (int c0 = cbeg; c0 < cbeg + BN / 2; c0 += 32) {
                     if (n0 + c0 >= p.N) break;  // uniform across the warp
                     uint32_t r[32];
                     tmem_ld_32x32(acc + c0, r);
@@ -1136,16 +1142,40 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
                     } else {
                         tmem_ld_wait();
                     }
-                    const int m = m0 + lg * 32 + lane;
-                    if (m >= p.M) continue;
-                    const int n = n0 + c0;
-                    int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (n + j < p.N)
-                            dst[j] = (W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j])) +
-                                     (p.act_zero ? zshift * __ldg(p.w_code_sums + n + j) : 0);
+                    for (int j = 0; j < 32; ++j) {
+                        int32_t v = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
+                        if (p.act_zero && n0 + c0 + j < p.N) v += zshift * __ldg(p.w_code_sums + n0 + c0 + j);
+                        r[j] = static_cast<uint32_t>(v);
+                    }
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        __syncwarp();  // the previous pass has been read out
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4*>(stage + lane * EPI32_ROW + q * 16) =
+                                make_uint4(r[16 * hh + 4 * q], r[16 * hh + 4 * q + 1], r[16 * hh + 4 * q + 2],
+                                           r[16 * hh + 4 * q + 3]);
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const int rl = it * 8 + (lane >> 2), seg = lane & 3;
+                            const int m = m0 + lg * 32 + rl;
+                            const int n = n0 + c0 + 16 * hh + seg * 4;
+                            if (m >= p.M || n >= p.N) continue;
+                            const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI32_ROW + seg * 16);
+                            int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
+                            if (vec) {  // n % 4 == 0 and N % 4 == 0: the four columns exist and are aligned
+                                *reinterpret_cast<uint4*>(dst) = v;
+                            } else {
+                                const uint32_t a[4] = {v.x, v.y, v.z, v.w};
+                                for (int j = 0; j < 4; ++j)
+                                    if (n + j < p.N) dst[j] = static_cast<int32_t>(a[j]);
+                            }
+                        }
+                    }
                 }
+                __syncwarp();
             }
             if (p.Y) {
                 const int cbeg = half * (BN / 2);
@@ -1371,6 +1401,22 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     if (wide) return launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
     return w4 ? launch_tma<128, 6, true>(ta, tw, ty, tp, splits, stream)
               : launch_tma<128, 6, false>(ta, tw, ty, tp, splits, stream);
+}
+
+// Step 1 alone: the int8 codes of X [rows, K] (row stride ldx) as a dense [rows, K] matrix.
+int run_quant(const __half* X, long long ldx, long long rows, int K, const float* act_scale, int8_t* out,
+              cudaStream_t stream)
+{
+    const long long tasks = rows * (K / 16);
+    return launch_pdl(quant_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1, X, ldx,
+                      rows, K, 0, act_scale, static_cast<const int32_t*>(nullptr), out);
+}
+
+// Step 2 alone, on int8 activations the caller keeps (the stored form of an activation tensor).
+int run_tma_prequantized(const Params& p, int amode, const void* packed, int w_bits, const int8_t* aq,
+                         cudaStream_t stream)
+{
+    return run_tma_gemm(p, amode, packed, w_bits, const_cast<int8_t*>(aq), stream);
 }
 
 // Layout of the shortcut-split scratch: [int8 lo | int8 hi | int32 sums lo | int32 sums hi], each 256-byte aligned.

@@ -42,6 +42,9 @@ _SIGNATURES = {
                                      _vp, _vp, _sz, _vp, _vp]),
     "mixdq_conv3x3_a8_asym_acc_i32": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp,
                                              _vp, _vp, _sz, _vp, _vp]),
+    "mixdq_quantize_acts": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "mixdq_linear_q8": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "mixdq_linear_q8_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp]),
     "mixdq_split_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, C.POINTER(_sz)]),
     "mixdq_linear_a8_split": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp,
                                      _sz, _vp, _vp]),
@@ -298,6 +301,32 @@ def conv3x3_a8_asym_acc_i32(X, packed_W, Cout: int, w_bits: int, w_code_sums, ac
     _chk(lib().mixdq_conv3x3_a8_asym_acc_i32(_ptr(X), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits,
                                              _ptr(w_code_sums), _ptr(act_scale), _ptr(act_zero), _ptr(acc), wp,
                                              wb, _ptr(status), _stream()), "mixdq_conv3x3_a8_asym_acc_i32")
+    return acc
+
+
+def quantize_acts(X, act_scale, out=None):
+    """int8 codes [rows, K] of X fp16 [rows, K] with the per-tensor scale *act_scale (device)."""
+    rows, K = X.shape
+    Xq = out if out is not None else torch.empty((rows, K), dtype=torch.int8, device=X.device)
+    assert X.stride(1) == 1
+    _chk(lib().mixdq_quantize_acts(C.c_void_p(X.data_ptr()), rows, K, X.stride(0), _ptr(act_scale), _ptr(Xq),
+                                   _stream()), "mixdq_quantize_acts")
+    return Xq
+
+
+def linear_q8(Xq, packed_W, N: int, w_bits: int, w_scale, act_scale, bias=None, status=None, out=None):
+    M, K = Xq.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib().mixdq_linear_q8(_ptr(Xq), M, K, _ptr(packed_W), N, w_bits, _ptr(w_scale), _ptr(act_scale),
+                               _ptr(bias), _ptr(Y), _ptr(status), _stream()), "mixdq_linear_q8")
+    return Y
+
+
+def linear_q8_acc_i32(Xq, packed_W, N: int, w_bits: int, status=None):
+    M, K = Xq.shape
+    acc = torch.empty((M, N), dtype=torch.int32, device=Xq.device)
+    _chk(lib().mixdq_linear_q8_acc_i32(_ptr(Xq), M, K, _ptr(packed_W), N, w_bits, _ptr(acc), _ptr(status),
+                                       _stream()), "mixdq_linear_q8_acc_i32")
     return acc
 
 
