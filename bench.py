@@ -50,6 +50,9 @@ def parse():
     ap.add_argument("--shortcut-split", action="store_true",
                     help="w4a8 table: the resnet convolutions of the up path that read a [hidden | skip] concatenation keep "
                          "one activation scale per branch (Sec. 4.1, shortcut-splitting); not part of the default run")
+    ap.add_argument("--share-qkv-quant", action="store_true",
+                    help="w4a8 table: the q, k and v projections of every self-attention block share one quantization "
+                         "pass of their common input (int8 codes kept, three GEMMs on them); not part of the default run")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -59,7 +62,7 @@ def workload_name(args):
     if args.tokens > 0:
         return f"unet_linear_sweep_{args.table}_{args.tokens}tokens" + ("_w248" if args.low_bits == 2 else "")
     return f"unet_sweep_sdxl512_{args.table}_b{args.batch}" + ("_asym_acts" if args.act_asym else "") + \
-        ("_shortcut_split" if args.shortcut_split else "") + \
+        ("_shortcut_split" if args.shortcut_split else "") + ("_shared_qkv_quant" if args.share_qkv_quant else "") + \
         ("_w248" if (args.low_bits == 2 and args.table == "a16") else "")
 
 
@@ -266,7 +269,7 @@ def run_ours(args):
     if args.tokens > 0 and args.table != "a16":
         raise SystemExit("--tokens needs --table a16 (the weight-only engine)")
     sweep = UNetSweep(args.batch, args.table, seed=5 + rank, tokens=args.tokens, act_asym=args.act_asym, low_bits=args.low_bits,
-                      shortcut_split=args.shortcut_split)
+                      shortcut_split=args.shortcut_split, share_qkv_quant=args.share_qkv_quant)
     tc_layers = [pl for pl in sweep.layers if sweep.uses_tensor_int8(pl)]
     other_layers = [pl for pl in sweep.layers if not sweep.uses_tensor_int8(pl)]
     if args.table == "a16":
@@ -402,9 +405,9 @@ def run_ours(args):
         achieved = tc_ops / (tc_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL
         # DRAM bytes per step of these kernels from one ncu capture of this command at batch 4 (caches flushed
-        # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.00 GB read by the quantization
-        # passes (every layer's input once) + 2.96 GB by the GEMMs (weights and int8 activations once)
-        traffic = 5.97e9 if (args.batch == 4 and world == 1 and not args.act_asym and not args.shortcut_split) else None
+        # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.01 GB read by the quantization
+        # passes (every layer's input once) + 3.00 GB by the GEMMs (weights and int8 activations once)
+        traffic = 6.01e9 if (args.batch == 4 and world == 1 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant) else None
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
                     "traffic": traffic,
                     "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
@@ -454,7 +457,7 @@ def run_ours(args):
             "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
             "device_status": status,
         }
-        if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and args.low_bits == 3:
+        if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and args.low_bits == 3:
             out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
         print(json.dumps(out))
     if world > 1:

@@ -184,6 +184,18 @@ def unet_layers() -> List[LayerSpec]:
     return L
 
 
+def self_attention_role(l: LayerSpec) -> int:
+    """0, 1, 2 for the q, k and v projections of a self-attention block -- three layers that read the same
+    tensor -- and -1 for every other layer.  The census lists six 1280x1280 (640x640) projections per
+    transformer block (self q, k, v, out; cross q, out) before the per-transformer proj_in / proj_out."""
+    base, _, idx = l.name.partition("#")
+    blocks = {"attn_1280": 60, "attn_640": 10}.get(base)
+    if blocks is None or int(idx) >= 6 * blocks:
+        return -1
+    role = int(idx) % 6
+    return role if role < 3 else -1
+
+
 # hidden-state channels of the layers fed by [hidden | skip] concatenations in the up path, by input width
 _CONCAT_HIDDEN = {2560: 1280, 1920: 1280, 1280: 640, 960: 640, 640: 320}
 

@@ -29,21 +29,26 @@ class PackedLayer:
     code_sums: Optional[torch.Tensor] = None   # asymmetric activations: per-channel sums of the weight codes
     split_at: int = 0                          # shortcut-splitting: `packed` holds input channels [0, split_at) ...
     packed_hi: Optional[torch.Tensor] = None   # ... and this the rest
+    qkv_role: int = -1                         # shared quantization: 0 quantizes the tensor, 1 and 2 reuse the codes
 
 
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
                  layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False,
-                 low_bits: int = 3, shortcut_split: bool = False):
+                 low_bits: int = 3, shortcut_split: bool = False, share_qkv_quant: bool = False):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
         (whatever the image size), so that a layer is one stream over its packed weights.
         act_asym: the 8-bit activations of the linear layers and 3x3 convolutions are asymmetric (Sec. 4.1);
         the BOS-aware K/V projections keep symmetric ones.
         low_bits: lowest width of the a16 table (3, or 2 for the paper's candidate widths {2, 4, 8}).
         shortcut_split: the A8 resnet convolutions (3x3 and 1x1) of the up path, whose input is a concatenation
-        [hidden | skip], keep one activation scale per branch (Sec. 4.1); symmetric activations."""
+        [hidden | skip], keep one activation scale per branch (Sec. 4.1); symmetric activations.
+        share_qkv_quant: the q, k and v projections of a self-attention block read one tensor; it is quantized
+        once (by q's call) and the three GEMMs run on the stored int8 codes (symmetric activations)."""
         assert table in ("w4a8", "a16")
-        assert not (act_asym and shortcut_split)
+        assert not (act_asym and shortcut_split) and not (act_asym and share_qkv_quant)
+        self.share_qkv_quant = share_qkv_quant and table == "w4a8" and tokens == 0
+        self.xq: Dict[tuple, torch.Tensor] = {}
         self.shortcut_split = shortcut_split
         self.batch = batch
         self.act_asym = act_asym
@@ -132,8 +137,11 @@ class UNetSweep:
                     x2 = self.x[xk].reshape(-1, l.Cin)
                     self.x_split_scale[(xk, split_at)] = (mixdq.act_scale(x2[:, :split_at].contiguous()),
                                                           mixdq.act_scale(x2[:, split_at:].contiguous()))
+            role = synth.self_attention_role(l) if (self.share_qkv_quant and l.a_bits == 8) else -1
+            if role >= 0 and xk not in self.xq:
+                self.xq[xk] = torch.empty((xk[1], xk[2]), dtype=torch.int8, device=self.device)
             self.layers.append(PackedLayer(l, packed, s, None if symmetric else z, bias, bos, xk, yk, sums, split_at,
-                                           packed_hi))
+                                           packed_hi, role))
             if split_at:
                 out_rows = yk[0] * yk[1] * yk[2]
                 need = mixdq.split_workspace_bytes(self.batch * l.H * l.H, l.Cin, split_at, out_rows, l.N)
@@ -172,6 +180,12 @@ class UNetSweep:
             return mixdq.crossattn_kv(x, pl.packed, l.N, l.w_bits, pl.w_scale, sx, pl.bos_out, ws, self.status,
                                       out=y)
         x2 = x.reshape(-1, x.shape[-1])
+        if pl.qkv_role >= 0:
+            xq = self.xq[pl.x_key]
+            if pl.qkv_role == 0:
+                mixdq.quantize_acts(x2, sx, out=xq)
+            return mixdq.linear_q8(xq, pl.packed, l.N, l.w_bits, pl.w_scale, sx, pl.bias, self.status,
+                                   out=y.reshape(-1, l.N))
         if pl.code_sums is not None:
             ax, az = self.x_asym[pl.x_key]
             return mixdq.linear_a8_asym(x2, pl.packed, l.N, l.w_bits, pl.w_scale, pl.code_sums, ax, az, pl.bias, ws,
