@@ -91,3 +91,66 @@ def test_argument_errors_come_back_before_any_launch(lib):
     assert lib.mixdq_crossattn_kv(fake, 1, 2048, fake, 640, 8, fake, fake, null, fake, null, 0, null, null) == -1
     assert lib.mixdq_pack_weights(fake, 4, 32, 3, fake, null, 1, fake, null) == -2
     assert lib.mixdq_pack_weights(fake, 4, 32, 4, fake, null, 1, odd, null) == -3
+
+
+def test_split_and_q8_argument_errors_come_back_before_any_launch(lib):
+    out = C.c_size_t(0)
+    null = None
+    fake = C.c_void_p(0x1000)       # never dereferenced: the checks below fail first
+    odd = C.c_void_p(0x1008)
+    # scratch of a shortcut-split layer: two int8 copies + two int32 sums, each rounded up to 256 bytes
+    assert lib.mixdq_split_workspace_bytes(64, 96, 32, 64, 48, C.byref(out)) == 0
+    assert out.value == 64 * 32 + 64 * 64 + 2 * 64 * 48 * 4
+    assert lib.mixdq_split_workspace_bytes(64, 96, 96, 64, 48, C.byref(out)) == -1    # nothing on the hi side
+    assert lib.mixdq_split_workspace_bytes(64, 96, 0, 64, 48, C.byref(out)) == -1
+    assert lib.mixdq_split_workspace_bytes(64, 96, 32, 64, 48, None) == -1
+    big = C.c_size_t(1 << 30)
+    split = lambda *a: lib.mixdq_linear_a8_split(*a)
+    #            X     M   K   ldx at  Wlo   Whi   N   b  ws    slo   shi   bias  Y     wsp   bytes st    stream
+    assert split(null, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -1
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, null, fake, big, null, null) == -1
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, null, fake, null, fake, fake, big, null, null) == -1
+    assert split(fake, 64, 96, 96, 96, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -1
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 3, fake, fake, fake, null, fake, fake, big, null, null) == -2
+    assert split(fake, 64, 96, 96, 24, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -2
+    assert split(fake, 64, 96, 96, 32, odd, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -3
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, null, big, null, null) == -4
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, 100, null, null) == -4
+    conv = lambda *a: lib.mixdq_conv3x3_a8_split(*a)
+    #           X     B  H  W  Cin at  Wlo   Whi   Co  s  b  ws    slo   shi   bias  Y     wsp   bytes st    stream
+    assert conv(fake, 1, 8, 8, 64, 32, fake, fake, 16, 3, 8, fake, fake, fake, null, fake, fake, big, null, null) == -1
+    assert conv(fake, 1, 8, 8, 64, 16, fake, fake, 16, 1, 8, fake, fake, fake, null, fake, fake, big, null, null) == -2
+    assert conv(fake, 1, 6, 6, 64, 32, fake, fake, 16, 1, 8, fake, fake, fake, null, fake, fake, big, null, null) == -2
+    # int8 activations kept between layers
+    assert lib.mixdq_quantize_acts(null, 4, 32, 32, fake, fake, null) == -1
+    assert lib.mixdq_quantize_acts(fake, 4, 32, 16, fake, fake, null) == -1       # row stride below K
+    assert lib.mixdq_quantize_acts(fake, 4, 40, 40, fake, fake, null) == -2       # K % 16
+    assert lib.mixdq_quantize_acts(fake, 4, 32, 32, fake, odd, null) == -3
+    assert lib.mixdq_linear_q8(null, 4, 32, fake, 16, 8, fake, fake, null, fake, null, null) == -1
+    assert lib.mixdq_linear_q8(fake, 4, 32, fake, 16, 8, fake, null, null, fake, null, null) == -1   # no scale
+    assert lib.mixdq_linear_q8(fake, 4, 32, fake, 16, 3, fake, fake, null, fake, null, null) == -2
+    assert lib.mixdq_linear_q8(fake, 4, 40, fake, 16, 8, fake, fake, null, fake, null, null) == -2
+    assert lib.mixdq_linear_q8(odd, 4, 32, fake, 16, 8, fake, fake, null, fake, null, null) == -3
+    assert lib.mixdq_linear_q8_acc_i32(fake, 4, 32, fake, 16, 8, null, null, null) == -1
+
+
+def test_census_helpers_for_split_and_shared_quantization():
+    from paper_2405_17873_b200 import synth
+    layers = synth.unet_layers()
+    split = {l.name: synth.shortcut_split_at(l) for l in layers if synth.shortcut_split_at(l)}
+    # the nine concatenation-fed resnets of the up path (3 per level), each with its 3x3 and its 1x1 shortcut conv
+    assert len(split) == 18
+    assert split["res16_2560_1280#0"] == 1280 and split["res16_1920_1280#0"] == 1280
+    assert split["res32_1920_640#0"] == 1280 and split["res32_1280_640#0"] == 640 and split["res32_960_640#0"] == 640
+    assert split["res64_960_320#0"] == 640 and split["res64_640_320#1"] == 320 and split["sc64_640#0"] == 320
+    for l in layers:
+        s = synth.shortcut_split_at(l)
+        assert s == 0 or (0 < s < l.Cin and s % 32 == 0 and (l.Cin - s) % 32 == 0)
+    # down-path resnets widen their input, the upsampler convs keep it: never split
+    assert not any(synth.shortcut_split_at(l) for l in layers if l.Cin <= l.N)
+    roles = [synth.self_attention_role(l) for l in layers]
+    assert roles.count(0) == roles.count(1) == roles.count(2) == 70     # 60 + 10 transformer blocks
+    by_name = {l.name: synth.self_attention_role(l) for l in layers}
+    assert [by_name[f"attn_1280#{i}"] for i in range(8)] == [0, 1, 2, -1, -1, -1, 0, 1]
+    assert by_name["attn_1280#360"] == -1 and by_name["attn_640#60"] == -1     # proj_in / proj_out
+    assert by_name["ffn1_1280#0"] == -1 and by_name["kv_1280#0"] == -1
