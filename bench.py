@@ -35,7 +35,9 @@ def parse():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "fp16_library"],
+                    help="ours: the CUDA library; reference: the CPU oracle; fp16_library: the same layers at fp16 through "
+                         "torch's vendor libraries, as context for the paper's speed-up over FP16")
     ap.add_argument("--batch", type=int, default=4)
     ap.add_argument("--table", default="w4a8", choices=["w4a8", "a16"])
     ap.add_argument("--tokens", type=int, default=0,
@@ -53,6 +55,10 @@ def parse():
     ap.add_argument("--share-qkv-quant", action="store_true",
                     help="w4a8 table: the q, k and v projections of every self-attention block share one quantization "
                          "pass of their common input (int8 codes kept, three GEMMs on them); not part of the default run")
+    ap.add_argument("--fuse-projections", action="store_true",
+                    help="q, k, v of every self-attention block and K, V of every cross-attention block run as one stacked "
+                         "layer where the bit table gives them equal widths (same operations, fewer layers); not part of "
+                         "the default run")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -62,7 +68,7 @@ def workload_name(args):
     if args.tokens > 0:
         return f"unet_linear_sweep_{args.table}_{args.tokens}tokens" + ("_w248" if args.low_bits == 2 else "")
     return f"unet_sweep_sdxl512_{args.table}_b{args.batch}" + ("_asym_acts" if args.act_asym else "") + \
-        ("_shortcut_split" if args.shortcut_split else "") + ("_shared_qkv_quant" if args.share_qkv_quant else "") + \
+        ("_shortcut_split" if args.shortcut_split else "") + ("_shared_qkv_quant" if args.share_qkv_quant else "") + ("_fused_projections" if args.fuse_projections else "") + \
         ("_w248" if (args.low_bits == 2 and args.table == "a16") else "")
 
 
@@ -249,6 +255,75 @@ def run_reference(args):
     }))
 
 
+# ----------------------------------------------------------------------------- fp16 library comparator
+
+def run_fp16_library(args):
+    """Context for the paper's speed-up over FP16 (Sec. 4.3): the same 794 layers at fp16 through the vendor
+    libraries (torch.nn.functional.linear / conv2d, channels-last), one step as a CUDA graph.  Not part of the
+    product path and not the benchmark's arm: it prints its own line with "impl": "fp16_library"."""
+    import torch
+    import torch.nn.functional as F
+    from paper_2405_17873_b200 import synth
+
+    torch.cuda.set_device(0)
+    B = args.batch
+    layers = synth.unet_layers()
+    g = torch.Generator(device="cuda").manual_seed(5)
+    xs, work, ops = {}, [], 0
+    for l in layers:
+        if l.kind in ("conv3x3", "conv1x1"):
+            k = 3 if l.kind == "conv3x3" else 1
+            key = ("img", l.H, l.Cin)
+            if key not in xs:
+                x = torch.randn((B, l.Cin, l.H, l.H), generator=g, device="cuda", dtype=torch.float16)
+                xs[key] = x.contiguous(memory_format=torch.channels_last)
+            w = (torch.randn((l.N, l.Cin, k, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).half()
+            w = w.contiguous(memory_format=torch.channels_last)
+            bias = (torch.randn((l.N,), generator=g, device="cuda") * 0.01).half()
+            work.append(("conv", xs[key], w, bias, l.stride, k // 2))
+        else:
+            rows = B * synth.TOKENS_PER_PROMPT if l.kind == "bos_kv" else l.M * B
+            key = ("rows", rows, l.K)
+            if key not in xs:
+                xs[key] = torch.randn((rows, l.K), generator=g, device="cuda", dtype=torch.float16)
+            w = (torch.randn((l.N, l.K), generator=g, device="cuda", dtype=torch.float32) * 0.02).half()
+            bias = None if l.kind == "bos_kv" else (torch.randn((l.N,), generator=g, device="cuda") * 0.01).half()
+            work.append(("lin", xs[key], w, bias, 1, 0))
+        ops += l.ops(B)
+
+    def step():
+        for kind, x, w, b, stride, pad in work:
+            if kind == "conv":
+                F.conv2d(x, w, b, stride=stride, padding=pad)
+            else:
+                F.linear(x, w, b)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream), torch.no_grad():
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step()
+        for _ in range(max(args.warmup, 3)):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"impl": "fp16_library", "metric": METRIC, "value": ops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "dtype": "f16", "data": "synthetic",
+                      "config": {"workload": f"unet_sweep_sdxl512_fp16_b{B}", "layers": len(layers), "ops_per_step": ops,
+                                 "launch": "CUDA graph replay", "library": "torch " + torch.__version__ +
+                                 " (cuBLAS / cuDNN), fp16 weights distinct per layer"}}))
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def run_ours(args):
@@ -269,7 +344,8 @@ def run_ours(args):
     if args.tokens > 0 and args.table != "a16":
         raise SystemExit("--tokens needs --table a16 (the weight-only engine)")
     sweep = UNetSweep(args.batch, args.table, seed=5 + rank, tokens=args.tokens, act_asym=args.act_asym, low_bits=args.low_bits,
-                      shortcut_split=args.shortcut_split, share_qkv_quant=args.share_qkv_quant)
+                      shortcut_split=args.shortcut_split, share_qkv_quant=args.share_qkv_quant,
+                      fuse_projections=args.fuse_projections)
     tc_layers = [pl for pl in sweep.layers if sweep.uses_tensor_int8(pl)]
     other_layers = [pl for pl in sweep.layers if not sweep.uses_tensor_int8(pl)]
     if args.table == "a16":
@@ -407,7 +483,7 @@ def run_ours(args):
         # DRAM bytes per step of these kernels from one ncu capture of this command at batch 4 (caches flushed
         # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.01 GB read by the quantization
         # passes (every layer's input once) + 3.00 GB by the GEMMs (weights and int8 activations once)
-        traffic = 6.01e9 if (args.batch == 4 and world == 1 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant) else None
+        traffic = 6.01e9 if (args.batch == 4 and world == 1 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections) else None
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
                     "traffic": traffic,
                     "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
@@ -457,7 +533,7 @@ def run_ours(args):
             "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
             "device_status": status,
         }
-        if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and args.low_bits == 3:
+        if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections and args.low_bits == 3:
             out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
         print(json.dumps(out))
     if world > 1:
@@ -468,6 +544,8 @@ def main():
     args = parse()
     if args.impl == "reference":
         run_reference(args)
+    elif args.impl == "fp16_library":
+        run_fp16_library(args)
     else:
         run_ours(args)
 

@@ -196,6 +196,37 @@ def self_attention_role(l: LayerSpec) -> int:
     return role if role < 3 else -1
 
 
+def fuse_projections(layers: List[LayerSpec]) -> List[LayerSpec]:
+    """The census with projections that read the same tensor stacked into one layer where their widths agree:
+    q, k and v of a self-attention block (N -> 3N) and the K and V projections of a cross-attention block
+    (consecutive pairs of the BOS-aware layers, N -> 2N).  Per-output-channel weight scales and a shared
+    activation scale make the stacked layer compute exactly what the separate ones do; the operation count
+    is unchanged."""
+    out: List[LayerSpec] = []
+    i = 0
+    while i < len(layers):
+        l = layers[i]
+        group = 1
+        if self_attention_role(l) == 0 and i + 2 < len(layers):
+            group = 3
+        elif l.kind == "bos_kv" and int(l.name.partition("#")[2]) % 2 == 0 and i + 1 < len(layers):
+            group = 2
+        members = layers[i:i + group]
+        same = all(m.kind == l.kind and (m.N, m.K, m.M, m.w_bits, m.a_bits) == (l.N, l.K, l.M, l.w_bits, l.a_bits)
+                   for m in members)
+        if group > 1 and same:
+            base, _, idx = l.name.partition("#")
+            out.append(LayerSpec(name=f"{'qkv' if group == 3 else 'kv2'}_{base}#{idx}", kind=l.kind, M=l.M,
+                                 N=group * l.N, K=l.K, per_batch=l.per_batch, w_bits=l.w_bits, a_bits=l.a_bits))
+            i += group
+        else:
+            out.append(l)
+            i += 1
+    for j, l in enumerate(out):
+        l.index = j
+    return out
+
+
 # hidden-state channels of the layers fed by [hidden | skip] concatenations in the up path, by input width
 _CONCAT_HIDDEN = {2560: 1280, 1920: 1280, 1280: 640, 960: 640, 640: 320}
 

@@ -35,7 +35,8 @@ class PackedLayer:
 class UNetSweep:
     def __init__(self, batch: int, table: str = "w4a8", seed: int = 5, device: str = "cuda",
                  layers: Optional[List[synth.LayerSpec]] = None, tokens: int = 0, act_asym: bool = False,
-                 low_bits: int = 3, shortcut_split: bool = False, share_qkv_quant: bool = False):
+                 low_bits: int = 3, shortcut_split: bool = False, share_qkv_quant: bool = False,
+                 fuse_projections: bool = False):
         """tokens > 0: the weight-bound regime -- only the linear layers, each on `tokens` rows in all
         (whatever the image size), so that a layer is one stream over its packed weights.
         act_asym: the 8-bit activations of the linear layers and 3x3 convolutions are asymmetric (Sec. 4.1);
@@ -44,7 +45,9 @@ class UNetSweep:
         shortcut_split: the A8 resnet convolutions (3x3 and 1x1) of the up path, whose input is a concatenation
         [hidden | skip], keep one activation scale per branch (Sec. 4.1); symmetric activations.
         share_qkv_quant: the q, k and v projections of a self-attention block read one tensor; it is quantized
-        once (by q's call) and the three GEMMs run on the stored int8 codes (symmetric activations)."""
+        once (by q's call) and the three GEMMs run on the stored int8 codes (symmetric activations).
+        fuse_projections: q, k, v of self-attention and K, V of cross-attention run as one stacked layer each where
+        the bit table gives them the same widths (synth.fuse_projections)."""
         assert table in ("w4a8", "a16")
         assert not (act_asym and shortcut_split) and not (act_asym and share_qkv_quant)
         self.share_qkv_quant = share_qkv_quant and table == "w4a8" and tokens == 0
@@ -63,6 +66,8 @@ class UNetSweep:
                 synth.assign_bits_w4a8(self.specs, seed)
             else:
                 synth.assign_bits_weight_only(self.specs, seed, low=low_bits)
+        if fuse_projections:
+            self.specs = synth.fuse_projections(self.specs)
         self.x: Dict[tuple, torch.Tensor] = {}
         self.y: Dict[tuple, torch.Tensor] = {}
         self.x_scale: Dict[tuple, torch.Tensor] = {}

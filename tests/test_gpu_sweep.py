@@ -52,6 +52,12 @@ def _check_layer(sw, pl, B):
         return
     codes = _codes(pl.packed, l.N, l.K, l.w_bits)
     sx = np.float32(host(sw.x_scale[pl.x_key])[0])
+    if l.kind == "bos_kv":
+        bos = host(pl.bos_out)
+        _, y_ref = orc.crossattn_kv(x, codes, ws, sx, bos)
+        assert np.array_equal(y[:, 0].view(np.uint16), np.broadcast_to(bos.view(np.uint16), y[:, 0].shape))
+        assert_close(y, y_ref)
+        return
     if l.kind == "conv3x3":
         _, y_ref = orc.conv3x3_a8(x, codes.reshape(l.N, 3, 3, l.Cin), ws, sx, b, l.stride)
     else:
@@ -88,3 +94,21 @@ def test_shared_quantization_gives_identical_bits():
         torch.cuda.synchronize()
         assert torch.equal(a.x[pa.x_key], b.x[pb.x_key])
         assert torch.equal(a.y[pa.y_key], b.y[pb.y_key])
+
+
+def test_fused_projections_against_oracle():
+    # q, k, v with equal widths become one 3N-wide layer, K and V one 2N-wide BOS-aware layer; a triple with
+    # mixed widths stays apart
+    L = [synth.LayerSpec(name=f"attn_640#{i}", kind="linear", M=192, N=96, K=160, w_bits=4) for i in range(3)]
+    L += [synth.LayerSpec(name=f"attn_640#{i}", kind="linear", M=192, N=96, K=160, w_bits=8 if i == 7 else 4)
+          for i in range(3, 9)]
+    L += [synth.LayerSpec(name=f"kv_640#{i}", kind="bos_kv", M=synth.TOKENS_PER_PROMPT, N=48, K=synth.TEXT_DIM, w_bits=8)
+          for i in range(2)]
+    ops = sum(l.ops(2) for l in L)
+    sw = UNetSweep(2, "w4a8", layers=L, fuse_projections=True)
+    assert [pl.spec.name for pl in sw.layers] == ["qkv_attn_640#0", "attn_640#3", "attn_640#4", "attn_640#5",
+                                                  "attn_640#6", "attn_640#7", "attn_640#8", "kv2_kv_640#0"]
+    assert [pl.spec.N for pl in sw.layers] == [288, 96, 96, 96, 96, 96, 96, 96]
+    assert sw.total_ops() == ops
+    for pl in sw.layers:
+        _check_layer(sw, pl, 2)
