@@ -138,3 +138,58 @@ def test_weight_only_layers_full_size(name, w_bits):
                                          ("attn_1280#0", 8)])
 def test_weight_only_sixteen_tokens_full_width(name, w_bits):
     _check_layer(name, w_bits, 16, rows_override=16)
+
+
+@pytest.mark.parametrize("name,w_bits", [("res16_2560_1280#0", 4), ("res32_1920_640#0", 8), ("res64_640_320#0", 4),
+                                         ("sc64_960#0", 4), ("sc16_2560#0", 8)])
+def test_shortcut_split_layers_full_size(name, w_bits):
+    """The concatenation-fed resnet convolutions at image batch 4 with one activation scale per branch
+    (Sec. 4.1): both int32 sums of the sampled output pixels bit-exact, outputs within tolerance."""
+    l = _SPECS[name]
+    split = synth.shortcut_split_at(l)
+    assert split > 0
+    X, W, b = synth.layer_inputs(l, B, seed=7000 + l.index)
+    X = X.copy()
+    X[..., split:] = (X[..., split:].astype(np.float32) / 8.0).astype(np.float16)   # the skip branch: a smaller range
+    taps = l.K // l.Cin
+    W3 = np.ascontiguousarray(W.reshape(l.N, taps, l.Cin))
+    W2 = W3.reshape(l.N, -1)
+    s_ref, _ = orc.weight_minmax_params(W2, w_bits, True)
+    codes = orc.quantize_weights(W2, w_bits, s_ref, None).reshape(l.N, taps, l.Cin)
+    x2 = X.reshape(-1, l.Cin)
+    s_lo_ref = orc.act_scale(orc.act_absmax(np.ascontiguousarray(x2[:, :split])), 8)
+    s_hi_ref = orc.act_scale(orc.act_absmax(np.ascontiguousarray(x2[:, split:])), 8)
+
+    Xd = dev(X)
+    s, _ = mixdq.weight_minmax_params(dev(W2), w_bits, True)
+    p_lo = mixdq.pack_weights(dev(W3[:, :, :split].reshape(l.N, -1)), w_bits, s)
+    p_hi = mixdq.pack_weights(dev(W3[:, :, split:].reshape(l.N, -1)), w_bits, s)
+    xd2 = Xd.reshape(-1, l.Cin)
+    s_lo, s_hi = mixdq.act_scale(xd2[:, :split].contiguous()), mixdq.act_scale(xd2[:, split:].contiguous())
+    assert host(s_lo)[0] == s_lo_ref and host(s_hi)[0] == s_hi_ref
+    Ho = (l.H - 1) // l.stride + 1
+    out_rows = B * Ho * Ho
+    ws = mixdq.new_workspace(mixdq.split_workspace_bytes(B * l.H * l.H, l.Cin, split, out_rows, l.N))
+    st = status_word()
+    if l.kind == "conv3x3":
+        a_lo, a_hi = mixdq.conv3x3_a8_split_acc_i32(Xd, split, p_lo, p_hi, l.N, w_bits, s_lo, s_hi, l.stride, ws, st)
+        y = mixdq.conv3x3_a8_split(Xd, split, p_lo, p_hi, l.N, w_bits, s, s_lo, s_hi, dev(b), l.stride, ws, st)
+    else:
+        a_lo, a_hi = mixdq.linear_a8_split_acc_i32(xd2, split, p_lo, p_hi, l.N, w_bits, s_lo, s_hi, ws, st)
+        y = mixdq.linear_a8_split(xd2, split, p_lo, p_hi, l.N, w_bits, s, s_lo, s_hi, dev(b), ws, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    a_lo, a_hi, y = (host(t).reshape(-1, l.N) for t in (a_lo, a_hi, y))
+    rows = _sample_rows(out_rows, seed=l.index)
+    if l.kind == "conv3x3":
+        win = _window_rows(X, rows, l.stride).reshape(len(rows), 9, l.Cin)
+    else:
+        win = x2[rows].reshape(len(rows), 1, l.Cin)
+    # the sampled pixels as a split linear layer on [all lo channels of the taps | all hi channels]
+    cols = np.ascontiguousarray(np.concatenate([win[:, :, :split].reshape(len(rows), -1),
+                                                win[:, :, split:].reshape(len(rows), -1)], axis=1))
+    wcols = np.ascontiguousarray(np.concatenate([codes[:, :, :split].reshape(l.N, -1),
+                                                 codes[:, :, split:].reshape(l.N, -1)], axis=1))
+    lo_ref, hi_ref, y_ref = orc.linear_a8_split(cols, wcols, s_ref, s_lo_ref, s_hi_ref, taps * split, b)
+    assert np.array_equal(a_lo[rows], lo_ref) and np.array_equal(a_hi[rows], hi_ref)
+    _close(y[rows], y_ref)
