@@ -262,7 +262,8 @@ int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* pa
  * Symmetric weights, w_bits in {4, 8}; symmetric activations.  NEEDS a workspace of
  * mixdq_split_workspace_bytes(in_rows, row_len, split_at, out_rows, N) bytes, where (in_rows, row_len,
  * out_rows) = (M, K, M) for a linear layer and (B*H*W, Cin, B*Ho*Wo) for a convolution; it holds the two
- * int8 copies and the two int32 sums, needs no initial content, and calls sharing it must not overlap.
+ * int8 copies and the first branch's int32 sums (the second branch's kernel reads them in its epilogue), must be
+ * 16-byte aligned, needs no initial content, and calls sharing it must not overlap.
  * split_at and K - split_at (Cin - split_at) must suit the two-kernel path: multiples of 16 (convolution:
  * of 32, with an image geometry as for mixdq_conv3x3_a8_asym), ldx % 8 == 0, X 16-byte aligned;
  * MIXDQ_ERR_UNSUPPORTED otherwise, MIXDQ_ERR_WORKSPACE when the workspace is missing or too small.

@@ -348,7 +348,7 @@ int split_common(i8::Params& p, int amode, int64_t in_rows, int64_t row_len, int
     if (p.Y ? !p.w_scale : (!acc_lo_out || !acc_hi_out)) return MIXDQ_ERR_INVALID_ARG;
     if (split_at <= 0 || split_at >= row_len) return MIXDQ_ERR_INVALID_ARG;
     if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
-    if (!aligned16(packed_lo) || !aligned16(packed_hi)) return MIXDQ_ERR_ALIGNMENT;
+    if (!aligned16(packed_lo) || !aligned16(packed_hi) || !aligned16(workspace)) return MIXDQ_ERR_ALIGNMENT;
     if (!i8::split_path_ok(p, amode, static_cast<int>(split_at), w_bits)) return MIXDQ_ERR_UNSUPPORTED;
     if (!workspace || ws_bytes < i8::split_layer_scratch_bytes(in_rows, row_len, split_at, p.M, p.N))
         return MIXDQ_ERR_WORKSPACE;

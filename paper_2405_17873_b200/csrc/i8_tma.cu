@@ -140,47 +140,6 @@ __global__ void quant_split_kernel(const __half* __restrict__ X, long long ldx, 
     *reinterpret_cast<uint4*>(dst) = q;
 }
 
-// The epilogue of a shortcut-split layer: y = fp16((s_lo * acc_lo + s_hi * acc_hi) * s_w[n] + bias[n]) from the
-// two branches' exact int32 sums.  One thread per four consecutive columns (N % 4 == 0) or per element.
-__global__ void combine_split_kernel(const int32_t* __restrict__ acc_lo, const int32_t* __restrict__ acc_hi,
-                                     long long M, int N, const float* __restrict__ scale_lo,
-                                     const float* __restrict__ scale_hi, const float* __restrict__ w_scale,
-                                     const __half* __restrict__ bias, __half* __restrict__ Y, long long ldy)
-{
-    pdl_launch_dependents();
-    pdl_wait();
-    const float s_lo = __ldg(scale_lo), s_hi = __ldg(scale_hi);
-    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-    if ((N & 3) == 0 && (ldy & 3) == 0) {
-        const int gpr = N >> 2;
-        if (idx >= M * gpr) return;
-        const long long m = idx / gpr;
-        const int n = static_cast<int>(idx - m * gpr) * 4;
-        const int4 a = *reinterpret_cast<const int4*>(acc_lo + m * N + n);
-        const int4 b = *reinterpret_cast<const int4*>(acc_hi + m * N + n);
-        const float4 w = __ldg(reinterpret_cast<const float4*>(w_scale + n));
-        float bs[4] = {0.f, 0.f, 0.f, 0.f};
-        if (bias) {
-            const uint2 raw = __ldg(reinterpret_cast<const uint2*>(bias + n));
-            const __half2* hb = reinterpret_cast<const __half2*>(&raw);
-            const float2 b0 = __half22float2(hb[0]), b1 = __half22float2(hb[1]);
-            bs[0] = b0.x; bs[1] = b0.y; bs[2] = b1.x; bs[3] = b1.y;
-        }
-        __half2 h[2];
-        h[0] = __floats2half2_rn(fmaf(fmaf(static_cast<float>(a.x), s_lo, static_cast<float>(b.x) * s_hi), w.x, bs[0]),
-                                 fmaf(fmaf(static_cast<float>(a.y), s_lo, static_cast<float>(b.y) * s_hi), w.y, bs[1]));
-        h[1] = __floats2half2_rn(fmaf(fmaf(static_cast<float>(a.z), s_lo, static_cast<float>(b.z) * s_hi), w.z, bs[2]),
-                                 fmaf(fmaf(static_cast<float>(a.w), s_lo, static_cast<float>(b.w) * s_hi), w.w, bs[3]));
-        *reinterpret_cast<uint2*>(Y + m * ldy + n) = *reinterpret_cast<const uint2*>(h);
-        return;
-    }
-    if (idx >= M * N) return;
-    const long long m = idx / N;
-    const int n = static_cast<int>(idx - m * N);
-    const float v = fmaf(static_cast<float>(acc_lo[idx]), s_lo, static_cast<float>(acc_hi[idx]) * s_hi);
-    Y[m * ldy + n] = __float2half_rn(fmaf(v, __ldg(w_scale + n), bias ? __half2float(bias[n]) : 0.f));
-}
-
 // Barrier over all threads of all CTAs of the cluster (hardware barrier, not a spin).
 __device__ __forceinline__ void cluster_sync_all()
 {
@@ -221,6 +180,10 @@ struct TmaParams {
     long long ldy;
     int32_t* acc_out;
     int32_t* status;
+    // second branch of a shortcut-split layer: the first branch's int32 sums [M, N] and its activation scale;
+    // the epilogue adds addend * (*addend_scale) * w_scale[n] to every output (ADD instances of the kernels)
+    const int32_t* addend;
+    const float* addend_scale;
     int small_acc;  // every |accumulator| (W4: after the >> 4) stays below 2^22
     int tma_store;  // Y is written through its tensor map (row-contiguous output, 16-byte aligned rows)
 };
@@ -436,6 +399,105 @@ __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t ac
                 const __half* hs = reinterpret_cast<const __half*>(&v);
                 for (int q = 0; q < 8; ++q)
                     if (n + q < p.N) dst[q] = hs[q];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// The 32-column passes for the second branch of a shortcut-split layer: y = acc * comb[c] + addend * ratio *
+// comb[c] + bias[c], where comb[c] = s_hi * s_w and ratio = s_lo / s_hi.  The first branch's sums come in through
+// the warp's staging tile, 16 columns at a time with four lanes along each row (coalesced), and the fp16 results
+// leave through the same tile with two lanes along each row.
+template <bool W4>
+__device__ __forceinline__ void store_rows32_add_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                           const float* bias, uint8_t* stage, const TmaParams& p,
+                                                           float ratio, int m_first, int n0, int lane)
+{
+    const bool yvec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
+    const bool avec = (p.N & 3) == 0;
+    for (int c0 = 0; c0 < ncols; c0 += 32) {
+        if (n0 + c0 >= p.N) break;  // uniform across the warp
+        uint32_t r[32];
+        tmem_ld_32x32(acc + c0, r);
+        if (acc2_off) {
+            uint32_t r2[32];
+            tmem_ld_32x32(acc + acc2_off + c0, r2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] += r2[j];
+        } else {
+            tmem_ld_wait();
+        }
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            __syncwarp();  // the tile's previous contents have been read out
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const int rl = it * 8 + (lane >> 2), seg = lane & 3;
+                const int mm = m_first + rl;
+                const int n = n0 + c0 + 16 * hh + seg * 4;
+                int4 a = make_int4(0, 0, 0, 0);
+                if (mm < p.M && n < p.N) {
+                    const int32_t* ap = p.addend + static_cast<long long>(mm) * p.N + n;
+                    // (read through L2: the sums were written by the previous kernel of the stream)
+                    if (avec) {  // N % 4 == 0 and n % 4 == 0: four existing, 16-byte aligned columns
+                        a = __ldcg(reinterpret_cast<const int4*>(ap));
+                    } else {
+                        a.x = __ldcg(ap);
+                        if (n + 1 < p.N) a.y = __ldcg(ap + 1);
+                        if (n + 2 < p.N) a.z = __ldcg(ap + 2);
+                        if (n + 3 < p.N) a.w = __ldcg(ap + 3);
+                    }
+                }
+                *reinterpret_cast<int4*>(stage + rl * EPI32_ROW + seg * 16) = a;
+            }
+            __syncwarp();
+            uint4 out[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int j = 16 * hh + 8 * q;  // column of the pass
+                const int c = c0 + j;
+                const int4 a0 = *reinterpret_cast<const int4*>(stage + lane * EPI32_ROW + q * 32);
+                const int4 a1 = *reinterpret_cast<const int4*>(stage + lane * EPI32_ROW + q * 32 + 16);
+                const float4 ca = *reinterpret_cast<const float4*>(comb + c);
+                const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
+                const float4 ba = *reinterpret_cast<const float4*>(bias + c);
+                const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+                __half2 hv[4];
+                hv[0] = __floats2half2_rn(
+                    fmaf(acc_to_float<W4, false>(r[j]), ca.x, fmaf(static_cast<float>(a0.x), ca.x * ratio, ba.x)),
+                    fmaf(acc_to_float<W4, false>(r[j + 1]), ca.y, fmaf(static_cast<float>(a0.y), ca.y * ratio, ba.y)));
+                hv[1] = __floats2half2_rn(
+                    fmaf(acc_to_float<W4, false>(r[j + 2]), ca.z, fmaf(static_cast<float>(a0.z), ca.z * ratio, ba.z)),
+                    fmaf(acc_to_float<W4, false>(r[j + 3]), ca.w, fmaf(static_cast<float>(a0.w), ca.w * ratio, ba.w)));
+                hv[2] = __floats2half2_rn(
+                    fmaf(acc_to_float<W4, false>(r[j + 4]), cb.x, fmaf(static_cast<float>(a1.x), cb.x * ratio, bb.x)),
+                    fmaf(acc_to_float<W4, false>(r[j + 5]), cb.y, fmaf(static_cast<float>(a1.y), cb.y * ratio, bb.y)));
+                hv[3] = __floats2half2_rn(
+                    fmaf(acc_to_float<W4, false>(r[j + 6]), cb.z, fmaf(static_cast<float>(a1.z), cb.z * ratio, bb.z)),
+                    fmaf(acc_to_float<W4, false>(r[j + 7]), cb.w, fmaf(static_cast<float>(a1.w), cb.w * ratio, bb.w)));
+                out[q] = *reinterpret_cast<const uint4*>(hv);
+            }
+            __syncwarp();  // every lane has read its row of sums
+            *reinterpret_cast<uint4*>(stage + lane * EPI32_ROW) = out[0];
+            *reinterpret_cast<uint4*>(stage + lane * EPI32_ROW + 16) = out[1];
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int rl = it * 16 + (lane >> 1), seg = lane & 1;
+                const int mm = m_first + rl;
+                const int n = n0 + c0 + 16 * hh + seg * 8;
+                if (mm >= p.M || n >= p.N) continue;
+                const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI32_ROW + seg * 16);
+                __half* dst = p.Y + static_cast<long long>(mm) * p.ldy + n;
+                if (yvec && n + 8 <= p.N) {
+                    *reinterpret_cast<uint4*>(dst) = v;
+                } else {
+                    const __half* hs = reinterpret_cast<const __half*>(&v);
+                    for (int q = 0; q < 8; ++q)
+                        if (n + q < p.N) dst[q] = hs[q];
+                }
             }
         }
         __syncwarp();
@@ -705,7 +767,7 @@ struct TmaSmem : Rings<BN, STAGES, W4, false> {
     static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
 };
 
-template <int BN, int STAGES, bool W4>
+template <int BN, int STAGES, bool W4, bool ADD = false>
 __global__ void __maxnreg__(96)
 tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                 const __grid_constant__ CUtensorMap tmap_y, const TmaParams p)
@@ -731,7 +793,8 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (rank + 1)) / splits);
     const int nkb = kb_end - kb_begin;
     // an unsplit tile needs no pass through shared memory: its epilogue warps store it themselves
-    const bool direct = splits == 1 && p.Y != nullptr && p.acc_out == nullptr;
+    // (nor does the second branch of a shortcut-split layer, whose epilogue reads the first branch's sums row-wise)
+    const bool direct = splits == 1 && p.Y != nullptr && p.acc_out == nullptr && !ADD;
     const bool dual = L::DUAL && nkb >= 2;  // two MMA issuers, two accumulators
 
     const uint32_t bar0 = smem_u32(bars);  // ring barriers, see Rings
@@ -879,6 +942,14 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         const bool vec = ((p.ldy & 3) == 0) && n + 4 <= p.N;
         const float4 cb = *reinterpret_cast<const float4*>(s_comb + chunk * 4);
         const float4 bb = *reinterpret_cast<const float4*>(s_bias + chunk * 4);
+        float4 cl = make_float4(0.f, 0.f, 0.f, 0.f);  // ADD: factors of the first branch's sums
+        if (ADD && n < p.N && p.w_scale) {
+            const float sl = __ldg(p.addend_scale);
+            cl.x = sl * __ldg(p.w_scale + n);
+            if (n + 1 < p.N) cl.y = sl * __ldg(p.w_scale + n + 1);
+            if (n + 2 < p.N) cl.z = sl * __ldg(p.w_scale + n + 2);
+            if (n + 3 < p.N) cl.w = sl * __ldg(p.w_scale + n + 3);
+        }
         if (n < p.N && tid < L::WORK_THREADS) {
 #pragma unroll 2
             for (int rl = tid / CHUNKS; rl < rows_per; rl += RSTEP) {
@@ -918,11 +989,29 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                         out_row = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
                                   (m - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
                     }
+                    float4 b4 = bb;
+                    if (ADD) {
+                        const int32_t* ap = p.addend + static_cast<long long>(m) * p.N + n;
+                        int4 a = make_int4(0, 0, 0, 0);
+                        // (read through L2: the sums were written by the previous kernel of the stream)
+                        if (((p.N & 3) == 0) && n + 4 <= p.N) {
+                            a = __ldcg(reinterpret_cast<const int4*>(ap));
+                        } else {
+                            a.x = __ldcg(ap);
+                            if (n + 1 < p.N) a.y = __ldcg(ap + 1);
+                            if (n + 2 < p.N) a.z = __ldcg(ap + 2);
+                            if (n + 3 < p.N) a.w = __ldcg(ap + 3);
+                        }
+                        b4.x = fmaf(static_cast<float>(a.x), cl.x, bb.x);
+                        b4.y = fmaf(static_cast<float>(a.y), cl.y, bb.y);
+                        b4.z = fmaf(static_cast<float>(a.z), cl.z, bb.z);
+                        b4.w = fmaf(static_cast<float>(a.w), cl.w, bb.w);
+                    }
                     __half2 h[2];
-                    h[0] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.x), cb.x, bb.x),
-                                             fmaf(acc_to_float<W4, false>(acc.y), cb.y, bb.y));
-                    h[1] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.z), cb.z, bb.z),
-                                             fmaf(acc_to_float<W4, false>(acc.w), cb.w, bb.w));
+                    h[0] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.x), cb.x, b4.x),
+                                             fmaf(acc_to_float<W4, false>(acc.y), cb.y, b4.y));
+                    h[1] = __floats2half2_rn(fmaf(acc_to_float<W4, false>(acc.z), cb.z, b4.z),
+                                             fmaf(acc_to_float<W4, false>(acc.w), cb.w, b4.w));
                     __half* dst = p.Y + out_row * p.ldy + n;
                     if (vec) {
                         *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
@@ -972,7 +1061,7 @@ struct PersistSmem : Rings<BN, STAGES, W4, true> {
     static constexpr int ACC_COLS = DUAL ? 2 * BN : BN;   // tensor-memory columns of one tile's accumulator(s)
 };
 
-template <int BN, int STAGES, bool W4>
+template <int BN, int STAGES, bool W4, bool ADD = false>
 __global__ void __launch_bounds__(PersistSmem<BN, STAGES, W4>::THREADS, 1)
 tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                            const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, int n_tiles,
@@ -1180,8 +1269,12 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
             if (p.Y) {
                 const int cbeg = half * (BN / 2);
                 uint8_t* stage = smem + L::OFF_EPI + (half * 4 + lg) * EPI32_TILE;
-                store_rows32_dispatch<W4>(acc + cbeg, dual ? BN : 0, BN / 2, comb + cbeg, bias + cbeg, stage, p, &tmap_y,
-                                          m0 + lg * 32, n0 + cbeg, lane);
+                if (ADD)
+                    store_rows32_add_from_tmem<W4>(acc + cbeg, dual ? BN : 0, BN / 2, comb + cbeg, bias + cbeg, stage, p,
+                                                   __ldg(p.addend_scale) / sx, m0 + lg * 32, n0 + cbeg, lane);
+                else
+                    store_rows32_dispatch<W4>(acc + cbeg, dual ? BN : 0, BN / 2, comb + cbeg, bias + cbeg, stage, p,
+                                              &tmap_y, m0 + lg * 32, n0 + cbeg, lane);
             }
             // the accumulator may be overwritten once every epilogue warp has read it
             tc_fence_before_sync();
@@ -1204,12 +1297,12 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     if (warp == 1) tmem_dealloc(tmem_base, 2 * L::ACC_COLS);
 }
 
-template <int BN, int STAGES, bool W4>
+template <int BN, int STAGES, bool W4, bool ADD = false>
 int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int num_sms,
                       cudaStream_t stream)
 {
     using L = PersistSmem<BN, STAGES, W4>;
-    auto kernel = tma_gemm_persistent_kernel<BN, STAGES, W4>;
+    auto kernel = tma_gemm_persistent_kernel<BN, STAGES, W4, ADD>;
     static bool attr_set = false;
     if (!attr_set) {
         MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
@@ -1221,12 +1314,12 @@ int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const CUtens
     return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, ty, tp, n_tiles, total);
 }
 
-template <int BN, int STAGES, bool W4>
+template <int BN, int STAGES, bool W4, bool ADD = false>
 int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int splits,
                cudaStream_t stream)
 {
     using L = TmaSmem<BN, STAGES, W4>;
-    auto kernel = tma_gemm_kernel<BN, STAGES, W4>;
+    auto kernel = tma_gemm_kernel<BN, STAGES, W4, ADD>;
     static bool attr_set = false;
     if (!attr_set) {
         MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
@@ -1339,7 +1432,9 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     tp.small_acc = static_cast<long long>(p.K) * (p.act_zero ? 128 : 127) * (w4 ? 7 : 127) < (1ll << 22);
     // output tiles leave through TMA stores when Y's rows are 16-byte aligned and consecutive output
     // rows are consecutive rows of Y (not so for the cross-attention K/V layout, which skips row 0)
-    tp.tma_store = p.Y && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
+    tp.addend = p.addend;
+    tp.addend_scale = p.addend_scale;
+    tp.tma_store = p.Y && !p.addend && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
     if (conv) {
         int Wb, Hb, Bb;
         if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
@@ -1365,7 +1460,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     if (rc != MIXDQ_OK) return rc;
     // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
     // (W4 runs on 128-wide tiles only: its packed ring needs the room, and it measured no slower)
-    const bool wide = !w4 && (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
+    const bool wide = !w4 && !p.addend && (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
     const uint32_t bn = wide ? 256 : 128;
     if (w4)
         rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, bn, false);
@@ -1387,6 +1482,14 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
         rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
                                 static_cast<uint64_t>(p.ldy), persistent ? 32 : 64, 32, persistent);
         if (rc != MIXDQ_OK) return rc;
+    }
+    if (p.addend) {  // second branch of a shortcut-split layer: the instances with the two-scale epilogue
+        if (persistent)
+            return w4 ? launch_persistent<128, 6, true, true>(ta, tw, ty, tp, num_sms, stream)
+                      : launch_persistent<128, 6, false, true>(ta, tw, ty, tp, num_sms, stream);
+        const int sp = pick_splits(tiles, tp.k_blocks);
+        return w4 ? launch_tma<128, 6, true, true>(ta, tw, ty, tp, sp, stream)
+                  : launch_tma<128, 6, false, true>(ta, tw, ty, tp, sp, stream);
     }
     if (persistent) {
         if (wide) return launch_persistent<256, 4, false>(ta, tw, ty, tp, num_sms, stream);
@@ -1419,11 +1522,11 @@ int run_tma_prequantized(const Params& p, int amode, const void* packed, int w_b
     return run_tma_gemm(p, amode, packed, w_bits, const_cast<int8_t*>(aq), stream);
 }
 
-// Layout of the shortcut-split scratch: [int8 lo | int8 hi | int32 sums lo | int32 sums hi], each 256-byte aligned.
+// Layout of the shortcut-split scratch: [int8 lo | int8 hi | int32 sums of the lo branch], each 256-byte aligned.
 size_t split_layer_scratch_bytes(int64_t in_rows, int64_t row_len, int64_t split_at, int64_t out_rows, int64_t N)
 {
     return static_cast<size_t>(round_up(in_rows * split_at, 256) + round_up(in_rows * (row_len - split_at), 256) +
-                               2 * round_up(out_rows * N * 4, 256));
+                               round_up(out_rows * N * 4, 256));
 }
 
 bool split_path_ok(const Params& p, int amode, int split_at, int w_bits)
@@ -1446,9 +1549,10 @@ bool split_path_ok(const Params& p, int amode, int split_at, int w_bits)
     return tma_path_ok(lo, amode, w_bits) && tma_path_ok(hi, amode, w_bits);
 }
 
-// Shortcut-splitting (Sec. 4.1): one quantization pass with a scale per branch, one int8 GEMM (or implicit-GEMM
-// convolution) per branch into exact int32 sums, and the two-scale epilogue.  acc_lo_out / acc_hi_out: where
-// the sums go (nullptr: into the scratch); p.Y == nullptr: sums only.
+// Shortcut-splitting (Sec. 4.1): one quantization pass with a scale per branch, then one int8 GEMM (or
+// implicit-GEMM convolution) per branch.  The first writes its exact int32 sums; the second is the instance with
+// the two-scale epilogue, which reads those sums and stores y = fp16((s_lo * acc_lo + s_hi * acc_hi) * s_w[n] +
+// bias[n]).  acc_lo_out / acc_hi_out given (parity hook, p.Y == nullptr): both kernels write their sums there.
 int run_tma_split(const Params& p, int amode, int split_at, const void* packed_lo, const void* packed_hi, int w_bits,
                   const float* scale_lo, const float* scale_hi, int32_t* acc_lo_out, int32_t* acc_hi_out,
                   void* scratch, cudaStream_t stream)
@@ -1462,9 +1566,7 @@ int run_tma_split(const Params& p, int amode, int split_at, const void* packed_l
     base += round_up(in_rows * split_at, 256);
     int8_t* aq_hi = reinterpret_cast<int8_t*>(base);
     base += round_up(in_rows * (row_len - split_at), 256);
-    const long long acc_bytes = round_up(static_cast<long long>(p.M) * p.N * 4, 256);
-    int32_t* acc_lo = acc_lo_out ? acc_lo_out : reinterpret_cast<int32_t*>(base);
-    int32_t* acc_hi = acc_hi_out ? acc_hi_out : reinterpret_cast<int32_t*>(base + acc_bytes);
+    int32_t* acc_lo = p.Y ? reinterpret_cast<int32_t*>(base) : acc_lo_out;
 
     const long long tasks = in_rows * (row_len / 16);
     int rc = launch_pdl(quant_split_kernel, dim3(static_cast<unsigned>(ceil_div(tasks, 256))), dim3(256), 0, stream, 1,
@@ -1483,18 +1585,19 @@ int run_tma_split(const Params& p, int amode, int split_at, const void* packed_l
     q.K = conv ? 9 * split_at : split_at;
     rc = run_tma_gemm(q, amode, packed_lo, w_bits, aq_lo, stream);
     if (rc != MIXDQ_OK) return rc;
-    q.acc_out = acc_hi;
     q.act_scale = scale_hi;
     q.Cin = conv ? row_len - split_at : 0;
     q.K = conv ? 9 * (row_len - split_at) : row_len - split_at;
-    rc = run_tma_gemm(q, amode, packed_hi, w_bits, aq_hi, stream);
-    if (rc != MIXDQ_OK || !p.Y) return rc;
-
-    const bool vec = p.N % 4 == 0 && p.ldy % 4 == 0;
-    const long long work = static_cast<long long>(p.M) * (vec ? p.N / 4 : p.N);
-    const long long M = p.M;
-    return launch_pdl(combine_split_kernel, dim3(static_cast<unsigned>(ceil_div(work, 256))), dim3(256), 0, stream, 1,
-                      acc_lo, acc_hi, M, p.N, scale_lo, scale_hi, p.w_scale, p.bias, p.Y, p.ldy);
+    if (p.Y) {
+        q.acc_out = nullptr;
+        q.Y = p.Y;
+        q.bias = p.bias;
+        q.addend = acc_lo;
+        q.addend_scale = scale_lo;
+    } else {
+        q.acc_out = acc_hi_out;
+    }
+    return run_tma_gemm(q, amode, packed_hi, w_bits, aq_hi, stream);
 }
 
 }  // namespace i8

@@ -98,9 +98,9 @@ def test_split_and_q8_argument_errors_come_back_before_any_launch(lib):
     null = None
     fake = C.c_void_p(0x1000)       # never dereferenced: the checks below fail first
     odd = C.c_void_p(0x1008)
-    # scratch of a shortcut-split layer: two int8 copies + two int32 sums, each rounded up to 256 bytes
+    # scratch of a shortcut-split layer: two int8 copies + the first branch's int32 sums, each rounded up to 256 bytes
     assert lib.mixdq_split_workspace_bytes(64, 96, 32, 64, 48, C.byref(out)) == 0
-    assert out.value == 64 * 32 + 64 * 64 + 2 * 64 * 48 * 4
+    assert out.value == 64 * 32 + 64 * 64 + 64 * 48 * 4
     assert lib.mixdq_split_workspace_bytes(64, 96, 96, 64, 48, C.byref(out)) == -1    # nothing on the hi side
     assert lib.mixdq_split_workspace_bytes(64, 96, 0, 64, 48, C.byref(out)) == -1
     assert lib.mixdq_split_workspace_bytes(64, 96, 32, 64, 48, None) == -1
@@ -114,6 +114,7 @@ def test_split_and_q8_argument_errors_come_back_before_any_launch(lib):
     assert split(fake, 64, 96, 96, 32, fake, fake, 48, 3, fake, fake, fake, null, fake, fake, big, null, null) == -2
     assert split(fake, 64, 96, 96, 24, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -2
     assert split(fake, 64, 96, 96, 32, odd, fake, 48, 8, fake, fake, fake, null, fake, fake, big, null, null) == -3
+    assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, odd, big, null, null) == -3
     assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, null, big, null, null) == -4
     assert split(fake, 64, 96, 96, 32, fake, fake, 48, 8, fake, fake, fake, null, fake, fake, 100, null, null) == -4
     conv = lambda *a: lib.mixdq_conv3x3_a8_split(*a)
