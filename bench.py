@@ -476,6 +476,36 @@ def run_ours(args):
 
     ops_step = sweep.total_ops()
     peaks = measured_peaks()
+    # the largest layers one by one (the "large-M" int8 layers the 60 % tensor-roofline target is about): each as
+    # a graph of ten back-to-back launches on its own weights (warm L2), against the burst peak, because such a
+    # graph is over in a millisecond
+    per_layer = None
+    if args.table == "w4a8" and world == 1 and args.tokens == 0:
+        per_layer = []
+        burst = peaks["bf16_tflops"] * INT8_TO_BF16_NOMINAL
+        for name in ("up64_640#0", "res64_320_320#0", "res32_640_640#0", "up32_1280#0", "res16_1280_1280#0",
+                     "res16_2560_1280#0", "ffn1_1280#0", "ffn2_1280#0", "ffn1_640#0", "attn_1280#0"):
+            pl = next((q for q in sweep.layers if q.spec.name == name), None)
+            if pl is None:
+                continue
+            reps, rounds = 10, 3
+            with torch.cuda.stream(stream):
+                g1 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g1, stream=stream):
+                    for _ in range(reps):
+                        sweep.run_layer(pl)
+                g1.replay()
+                t0, t1 = ev(), ev()
+                t0.record()
+                for _ in range(rounds):
+                    g1.replay()
+                t1.record()
+                torch.cuda.synchronize()
+            us = t0.elapsed_time(t1) * 1e3 / (reps * rounds)
+            tops = pl.spec.ops(args.batch) / us / 1e6
+            per_layer.append({"layer": name, "kind": pl.spec.kind, "M": pl.spec.rows(args.batch), "N": pl.spec.N,
+                              "K": pl.spec.K, "w_bits": pl.spec.w_bits, "us": round(us, 2), "tops": round(tops, 1),
+                              "frac_of_burst_peak": round(tops / burst, 3)})
     if args.table == "w4a8":
         tc_ops = sweep.total_ops(tc_layers)
         achieved = tc_ops / (tc_ms * 1e-3) / 1e12
@@ -531,6 +561,7 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline,
             "breakdown_ms": {"tensor_int8_layers": tc_ms, "other_layers": other_ms},
+            "large_m_layers": per_layer,
             "device_status": status,
         }
         if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections and args.low_bits == 3:
