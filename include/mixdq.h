@@ -244,6 +244,14 @@ int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void* packed_W, 
                     const float* w_scale, const float* act_scale, const void* bias, void* Y, int32_t* status,
                     void* stream);
 
+/* The 3x3 convolution on a stored int8 NHWC image [B, H, W, Cin] (codes from mixdq_quantize_acts on the
+ * [B*H*W, Cin] pixel matrix); zero padding is code 0.  Geometry as for the two-kernel path of mixdq_conv3x3
+ * (Cin % 32 == 0; Wo a multiple of 128, or 128 / Wo a divisor or a multiple of Ho; stride 2 only on even H, W):
+ * MIXDQ_ERR_UNSUPPORTED otherwise.  Other arguments as in mixdq_linear_q8. */
+int mixdq_conv3x3_q8(const void* Xq, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                     int64_t Cout, int stride, int w_bits, const float* w_scale, const float* act_scale,
+                     const void* bias, void* Y, int32_t* status, void* stream);
+
 /* Parity hook: int32 accumulators [M, N] of mixdq_linear_q8. */
 int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
                             int32_t* acc_out, int32_t* status, void* stream);

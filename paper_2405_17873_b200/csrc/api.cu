@@ -336,6 +336,41 @@ extern "C" int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, con
     return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, nullptr, nullptr, nullptr, nullptr, acc_out, status, stream);
 }
 
+extern "C" int mixdq_conv3x3_q8(const void* Xq, int64_t B, int64_t H, int64_t W, int64_t Cin, const void* packed_W,
+                                int64_t Cout, int stride, int w_bits, const float* w_scale, const float* act_scale,
+                                const void* bias, void* Y, int32_t* status, void* stream)
+{
+    if (!Xq || !packed_W || !Y || !w_scale || !act_scale) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(B) || !fits_int(H) || !fits_int(W) || !fits_int(Cin) || !fits_int(Cout))
+        return MIXDQ_ERR_INVALID_ARG;
+    if (stride != 1 && stride != 2) return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    if (!fits_int(B * Ho * Wo) || !fits_int(9 * Cin) || !fits_int(B * H * W * Cin)) return MIXDQ_ERR_INVALID_ARG;
+    if (!aligned16(packed_W) || !aligned16(Xq)) return MIXDQ_ERR_ALIGNMENT;
+    i8::Params p;
+    p.ldx = 8;
+    p.M = static_cast<int>(B * Ho * Wo);
+    p.N = static_cast<int>(Cout);
+    p.K = static_cast<int>(9 * Cin);
+    p.H = static_cast<int>(H);
+    p.W = static_cast<int>(W);
+    p.Cin = static_cast<int>(Cin);
+    p.Ho = static_cast<int>(Ho);
+    p.Wo = static_cast<int>(Wo);
+    p.stride = stride;
+    p.batch = static_cast<int>(B);
+    p.act_scale = act_scale;
+    p.w_scale = w_scale;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = Cout;
+    p.status = status;
+    if (!i8::tma_path_ok(p, A_CONV3, w_bits)) return MIXDQ_ERR_UNSUPPORTED;
+    return i8::run_tma_prequantized(p, A_CONV3, packed_W, w_bits, static_cast<const int8_t*>(Xq),
+                                    static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------- shortcut-splitting (Sec. 4.1)
 
 namespace {

@@ -44,6 +44,7 @@ _SIGNATURES = {
                                              _vp, _vp, _sz, _vp, _vp]),
     "mixdq_quantize_acts": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "mixdq_linear_q8": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "mixdq_conv3x3_q8": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
     "mixdq_linear_q8_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp]),
     "mixdq_split_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, C.POINTER(_sz)]),
     "mixdq_linear_a8_split": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -319,6 +320,16 @@ def linear_q8(Xq, packed_W, N: int, w_bits: int, w_scale, act_scale, bias=None, 
     Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=Xq.device)
     _chk(lib().mixdq_linear_q8(_ptr(Xq), M, K, _ptr(packed_W), N, w_bits, _ptr(w_scale), _ptr(act_scale),
                                _ptr(bias), _ptr(Y), _ptr(status), _stream()), "mixdq_linear_q8")
+    return Y
+
+
+def conv3x3_q8(Xq, packed_W, Cout: int, w_bits: int, w_scale, act_scale, bias=None, stride: int = 1, status=None,
+               out=None):
+    B, H, W, Cin = Xq.shape
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    Y = out if out is not None else torch.empty((B, Ho, Wo, Cout), dtype=torch.float16, device=Xq.device)
+    _chk(lib().mixdq_conv3x3_q8(_ptr(Xq), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits, _ptr(w_scale),
+                                _ptr(act_scale), _ptr(bias), _ptr(Y), _ptr(status), _stream()), "mixdq_conv3x3_q8")
     return Y
 
 

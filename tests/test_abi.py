@@ -133,6 +133,13 @@ def test_split_and_q8_argument_errors_come_back_before_any_launch(lib):
     assert lib.mixdq_linear_q8(fake, 4, 40, fake, 16, 8, fake, fake, null, fake, null, null) == -2
     assert lib.mixdq_linear_q8(odd, 4, 32, fake, 16, 8, fake, fake, null, fake, null, null) == -3
     assert lib.mixdq_linear_q8_acc_i32(fake, 4, 32, fake, 16, 8, null, null, null) == -1
+    #                          Xq    B  H  W  Cin Wp    Co  s  b  ws    sx    bias  Y     st    stream
+    assert lib.mixdq_conv3x3_q8(null, 1, 8, 8, 32, fake, 16, 1, 8, fake, fake, null, fake, null, null) == -1
+    assert lib.mixdq_conv3x3_q8(fake, 1, 8, 8, 32, fake, 16, 3, 8, fake, fake, null, fake, null, null) == -1
+    assert lib.mixdq_conv3x3_q8(fake, 1, 8, 8, 32, fake, 16, 1, 3, fake, fake, null, fake, null, null) == -2
+    assert lib.mixdq_conv3x3_q8(fake, 1, 8, 8, 20, fake, 16, 1, 8, fake, fake, null, fake, null, null) == -2
+    assert lib.mixdq_conv3x3_q8(fake, 1, 6, 6, 32, fake, 16, 1, 8, fake, fake, null, fake, null, null) == -2
+    assert lib.mixdq_conv3x3_q8(odd, 1, 8, 8, 32, fake, 16, 1, 8, fake, fake, null, fake, null, null) == -3
 
 
 def test_census_helpers_for_split_and_shared_quantization():

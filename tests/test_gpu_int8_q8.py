@@ -83,3 +83,27 @@ def test_q8_argument_errors():
         mixdq.linear_q8(Xq, packed, 32, 8, s, sx)            # K % 16 != 0
     with pytest.raises(mixdq.MixdqError, match="unsupported"):
         mixdq.linear_q8(Xq[:, :32].contiguous(), packed, 32, 3, s, sx)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,C,N,stride", [(2, 8, 32, 48, 1), (1, 16, 160, 136, 1), (3, 16, 256, 320, 1),
+                                             (2, 16, 64, 40, 2), (1, 64, 32, 32, 1)])
+def test_conv3x3_on_a_stored_int8_image(bits, B, H, C, N, stride):
+    X = synth.normal_f16((B, H, H, C), 1.0, seed=H + C)
+    Wt = synth.normal_f16((N, 3, 3, C), 0.02, seed=N + C + 1)
+    b = synth.normal_f16((N,), 0.01, seed=N + 2)
+    s_ref, _, codes = oracle_weights(Wt.reshape(N, -1), bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    _, y_ref = orc.conv3x3_a8(X, codes.reshape(N, 3, 3, C), s_ref, sx_ref, b, stride)
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt.reshape(N, -1), bits, True)
+    sx = mixdq.act_scale(Xd)
+    Xq = mixdq.quantize_acts(Xd.reshape(-1, C), sx).reshape(B, H, H, C)
+    st = status_word()
+    y = mixdq.conv3x3_q8(Xq, packed, N, bits, s, sx, dev(b), stride, st)
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, H, C, N, stride, bits, 8))
+    y_one = mixdq.conv3x3(Xd, packed, N, bits, s, None, 8, sx, dev(b), stride, ws, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert_close(host(y), y_ref)
+    assert np.array_equal(host(y).view(np.uint16), host(y_one).view(np.uint16))
