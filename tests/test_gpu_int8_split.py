@@ -141,3 +141,36 @@ def test_split_argument_errors():
         mixdq.linear_a8_split(X, 24, p_lo, p_hi, 32, 8, s, sx, sx, workspace=ws)     # not a multiple of 16
     with pytest.raises(mixdq.MixdqError, match="invalid"):
         mixdq.linear_a8_split(X, 64, p_lo, p_hi, 32, 8, s, sx, sx, workspace=ws)     # nothing on the hi side
+
+
+@pytest.mark.parametrize("zero_side", ["lo", "hi"])
+def test_split_with_an_all_zero_branch(zero_side):
+    # a branch of zeros has the degenerate scale 1 and codes 0: its sum vanishes and the output is the other
+    # branch's layer alone
+    M, C_lo, C_hi, N = 200, 64, 96, 72
+    X = _concat(M, C_lo, C_hi, seed=31)
+    if zero_side == "lo":
+        X[:, :C_lo] = 0
+    else:
+        X[:, C_lo:] = 0
+    W = synth.normal_f16((N, C_lo + C_hi), 0.02, seed=32)
+    b = synth.normal_f16((N,), 0.01, seed=33)
+    ws_ref, _ = orc.weight_minmax_params(W, 8, True)
+    codes = orc.quantize_weights(W, 8, ws_ref, None)
+    s_lo_ref = orc.act_scale(orc.act_absmax(np.ascontiguousarray(X[:, :C_lo])), 8)
+    s_hi_ref = orc.act_scale(orc.act_absmax(np.ascontiguousarray(X[:, C_lo:])), 8)
+    assert (s_lo_ref if zero_side == "lo" else s_hi_ref) == np.float32(1.0)
+    a_lo_ref, a_hi_ref, y_ref = orc.linear_a8_split(X, codes, ws_ref, s_lo_ref, s_hi_ref, C_lo, b)
+    assert not (a_lo_ref if zero_side == "lo" else a_hi_ref).any()
+    Xd = dev(X)
+    s, p_lo, p_hi = _device_halves(W[:, :C_lo], W[:, C_lo:], W, 8)
+    s_lo, s_hi = mixdq.act_scale(Xd[:, :C_lo].contiguous()), mixdq.act_scale(Xd[:, C_lo:].contiguous())
+    assert host(s_lo)[0] == s_lo_ref and host(s_hi)[0] == s_hi_ref
+    ws = mixdq.new_workspace(mixdq.split_workspace_bytes(M, C_lo + C_hi, C_lo, M, N))
+    st = status_word()
+    a_lo, a_hi = mixdq.linear_a8_split_acc_i32(Xd, C_lo, p_lo, p_hi, N, 8, s_lo, s_hi, workspace=ws, status=st)
+    y = mixdq.linear_a8_split(Xd, C_lo, p_lo, p_hi, N, 8, s, s_lo, s_hi, dev(b), workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(a_lo), a_lo_ref) and np.array_equal(host(a_hi), a_hi_ref)
+    assert_close(host(y), y_ref)
