@@ -416,6 +416,31 @@ __device__ __forceinline__ void store_rows32_add_from_tmem(uint32_t acc, uint32_
 {
     const bool yvec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
     const bool avec = (p.N & 3) == 0;
+    // The first branch's sums of one group of 16 columns: lane -> (row it * 8 + lane / 4, columns 4 * (lane % 4)...),
+    // read through L2 (they are the previous kernel's output).  A group is fetched while the one before it is
+    // converted and stored, so that its L2 round trip is not exposed.
+    auto fetch = [&](int col, int4 (&pre)[4]) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int mm = m_first + it * 8 + (lane >> 2);
+            const int n = n0 + col + (lane & 3) * 4;
+            int4 a = make_int4(0, 0, 0, 0);
+            if (col < ncols && mm < p.M && n < p.N) {
+                const int32_t* ap = p.addend + static_cast<long long>(mm) * p.N + n;
+                if (avec) {  // N % 4 == 0 and n % 4 == 0: four existing, 16-byte aligned columns
+                    a = __ldcg(reinterpret_cast<const int4*>(ap));
+                } else {
+                    a.x = __ldcg(ap);
+                    if (n + 1 < p.N) a.y = __ldcg(ap + 1);
+                    if (n + 2 < p.N) a.z = __ldcg(ap + 2);
+                    if (n + 3 < p.N) a.w = __ldcg(ap + 3);
+                }
+            }
+            pre[it] = a;
+        }
+    };
+    int4 pre[4];
+    fetch(0, pre);
     for (int c0 = 0; c0 < ncols; c0 += 32) {
         if (n0 + c0 >= p.N) break;  // uniform across the warp
         uint32_t r[32];
@@ -433,25 +458,9 @@ __device__ __forceinline__ void store_rows32_add_from_tmem(uint32_t acc, uint32_
         for (int hh = 0; hh < 2; ++hh) {
             __syncwarp();  // the tile's previous contents have been read out
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const int rl = it * 8 + (lane >> 2), seg = lane & 3;
-                const int mm = m_first + rl;
-                const int n = n0 + c0 + 16 * hh + seg * 4;
-                int4 a = make_int4(0, 0, 0, 0);
-                if (mm < p.M && n < p.N) {
-                    const int32_t* ap = p.addend + static_cast<long long>(mm) * p.N + n;
-                    // (read through L2: the sums were written by the previous kernel of the stream)
-                    if (avec) {  // N % 4 == 0 and n % 4 == 0: four existing, 16-byte aligned columns
-                        a = __ldcg(reinterpret_cast<const int4*>(ap));
-                    } else {
-                        a.x = __ldcg(ap);
-                        if (n + 1 < p.N) a.y = __ldcg(ap + 1);
-                        if (n + 2 < p.N) a.z = __ldcg(ap + 2);
-                        if (n + 3 < p.N) a.w = __ldcg(ap + 3);
-                    }
-                }
-                *reinterpret_cast<int4*>(stage + rl * EPI32_ROW + seg * 16) = a;
-            }
+            for (int it = 0; it < 4; ++it)
+                *reinterpret_cast<int4*>(stage + (it * 8 + (lane >> 2)) * EPI32_ROW + (lane & 3) * 16) = pre[it];
+            fetch(c0 + 16 * hh + 16, pre);  // the next group (nothing past the last column)
             __syncwarp();
             uint4 out[2];
 #pragma unroll
