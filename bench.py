@@ -554,6 +554,7 @@ def run_ours(args):
             "config": {"workload": workload_name(args), "table": args.table, "batch": args.batch,
                        "layers": len(sweep.layers), "ops_per_step": ops_step,
                        "packed_weight_bytes": sweep.packed_weight_bytes(),
+                       "fp16_weight_bytes": 2 * sum(pl.spec.params for pl in sweep.layers),
                        "l2": "weights (distinct per layer) are larger than L2", "launch": "CUDA graph replay"},
             "clocks": clocks,
             "e2e": {"value": replicas.whole_job_rate(ops_step, e2e_ms) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
