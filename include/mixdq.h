@@ -149,6 +149,18 @@ int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t Cin, 
                                   int stride, int w_bits, int act_bits, size_t* out);
 
 /*
+ * Constants of a layer.  packed_W, w_scale, w_zero, bias, the weight code sums and a stored BOS row are
+ * constants of the layer (the paper quantizes weights offline, Sec. 4.1).  The layer kernels may load
+ * them BEFORE they wait for earlier work on the stream, so that their start overlaps the previous
+ * kernel's end; they must therefore be complete when a layer call that reads them is enqueued.  Buffers
+ * written by mixdq_pack_weights, mixdq_weight_minmax_params and mixdq_weight_code_sums on the SAME stream
+ * satisfy this by themselves (those calls end with a full stream dependency).  Constants produced any
+ * other way (a copy, a kernel of the caller's, another stream) need a stream synchronization or an event
+ * wait between their producer and the first layer call that uses them.  Everything else -- X, the
+ * activation scale and zero-point, the workspace, Y -- follows ordinary stream order.
+ */
+
+/*
  * Quantized linear layer  Y[M, N] = X[M, K] * dequant(W)^T + bias   (paper Sec. 4.1, 4.3).
  *   act_bits == 8 : W8A8 / W4A8.  X is quantized per tensor with *act_scale (device fp32)
  *                   inside the kernel, multiplied with the integer weight codes in int32
@@ -353,15 +365,17 @@ int mixdq_probe_mma_loop(int kind, int batches, double* ops_out, int32_t* status
  * mixdq_linear with act_bits = 8 for callers that have no device memory to give as a
  * workspace -- a process whose memory manager owns the whole GPU, code embedded in another
  * framework's allocator, or a loop that cannot afford the device-wide synchronization of
- * cudaMalloc.  The split-reduction scratch is a fixed array of
+ * cudaMalloc.  The layer's scratch -- the int8 copy of X that the quantization pass writes and
+ * the GEMM reads, placed behind the region a split reduction would use -- is a fixed array of
  * mixdq_static_scratch_bytes() bytes (8 MiB) inside the library image; every GPU that loads
  * the library holds it until the process exits.  The call allocates and frees nothing.
  *   - A problem whose scratch need (mixdq_workspace_bytes) exceeds the array is rejected with
  *     MIXDQ_ERR_WORKSPACE; nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device
  *     current).  Make that first call outside any stream capture.
- *   - All calls share the one array and each call clears the part it uses first, so two
- *     calls that can overlap on the GPU (different streams) race: serialize them.
+ *   - All calls share the one array, which keeps the previous call's contents; a call
+ *     overwrites what it reads (and clears what it needs zeroed) itself, so two calls that can
+ *     overlap on the GPU (different streams) race: serialize them.
  * Arguments as in mixdq_linear; weights symmetric, w_bits in {4, 8}.
  */
 size_t mixdq_static_scratch_bytes(void);

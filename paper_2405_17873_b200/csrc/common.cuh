@@ -69,6 +69,12 @@ int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4
 // tail and the next GEMM's set-up overlap.  Returns MIXDQ_OK or MIXDQ_ERR_CUDA.
 int prefer_max_shared_carveout(const void* kernel);
 
+// Once per (device, kernel): raise the kernel's dynamic shared-memory limit to `bytes`.
+int ensure_dynamic_smem(const void* kernel, int bytes);
+
+// Streaming multiprocessors of the current device (looked up once per device; 0 on error).
+int sm_count();
+
 #ifdef __CUDACC__
 
 // Launch with programmatic dependent launch enabled (and an optional cluster along z): the

@@ -37,7 +37,6 @@ struct Params {
     int32_t* status = nullptr;
     int32_t* ws_tickets = nullptr;  // split-K: one arrival counter per output tile
     int32_t* ws_acc = nullptr;      // split-K: int32 partial sums, padded to whole tiles
-    int force_splits = 0;           // > 0: use exactly this many reduction splits
     // two-kernel path, second branch of a shortcut-split layer: the first branch's int32 sums [M, N] and its
     // activation scale; the epilogue adds addend * (*addend_scale) * w_scale[n]
     const int32_t* addend = nullptr;

@@ -605,11 +605,7 @@ int launch_tc(const Params& p, const void* packed, int64_t pitch, int splits, cu
         rc = encode_tmap_2d_u8(&tmap, packed, static_cast<uint64_t>(p.K), p.N, pitch, BK, BN, true);
     if (rc != MIXDQ_OK) return rc;
     auto kernel = gemm_kernel<BN, STAGES, W4, AMODE>;
-    static bool attr_set = false;  // per template instance
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-        attr_set = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     dim3 grid(static_cast<unsigned>(ceil_div(p.N, BN)), static_cast<unsigned>(ceil_div(p.M, BM)),
               static_cast<unsigned>(splits));
     return launch_pdl(kernel, grid, dim3(kThreads), L::TOTAL, stream, 1, tmap, p);
@@ -630,20 +626,6 @@ size_t split_scratch_bytes(int64_t rows, int64_t N)
 size_t workspace_bytes(int64_t out_rows, int64_t N, int64_t in_rows, int64_t row_len)
 {
     return split_scratch_bytes(out_rows, N) + tma_scratch_bytes(in_rows, row_len);
-}
-
-// MIXDQ_I8_PATH=fused|tma overrides the choice between the fused single kernel and the
-// quantize-then-GEMM pair (diagnostics and tuning; unset = automatic).
-static int path_override()
-{
-    static int v = -1;
-    if (v < 0) {
-        const char* e = getenv("MIXDQ_I8_PATH");
-        v = 0;
-        if (e && !strcmp(e, "fused")) v = 1;
-        if (e && !strcmp(e, "tma")) v = 2;
-    }
-    return v;
 }
 
 int run(Params p, int amode, const void* packed, int w_bits, void* workspace, size_t ws_bytes,
@@ -667,7 +649,7 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
         if (amode == A_BOS || !p.w_code_sums || !tma_room || !tma_path_ok(p, amode, w_bits)) return MIXDQ_ERR_UNSUPPORTED;
         return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
     }
-    if (tma_room && tma_path_ok(p, amode, w_bits) && path_override() != 1)
+    if (tma_room && tma_path_ok(p, amode, w_bits))
         return run_tma(p, amode, packed, w_bits, static_cast<uint8_t*>(workspace) + split_bytes, stream);
 
     if (!tc_ok && !w4 && p.K <= 64) {
@@ -690,14 +672,12 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, 128);
     int splits = 1;
     const bool split_room = workspace && ws_bytes >= split_bytes;
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
     if (split_room && tiles < 96 && p.k_blocks >= 8) {
-        splits = static_cast<int>(148 / tiles);
+        splits = static_cast<int>(num_sms / tiles);
         if (splits > p.k_blocks / 4) splits = p.k_blocks / 4;
         if (splits < 1) splits = 1;
-    }
-    if (p.force_splits > 0) {
-        if (p.force_splits > 1 && !split_room) return MIXDQ_ERR_WORKSPACE;
-        splits = p.force_splits > p.k_blocks ? p.k_blocks : p.force_splits;
     }
     if (splits > 1) {
         // a workspace shared between layers may hold another layer's int8 activations here, so the

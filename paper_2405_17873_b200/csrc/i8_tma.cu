@@ -1312,11 +1312,7 @@ int launch_persistent(const CUtensorMap& ta, const CUtensorMap& tw, const CUtens
 {
     using L = PersistSmem<BN, STAGES, W4>;
     auto kernel = tma_gemm_persistent_kernel<BN, STAGES, W4, ADD>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-        attr_set = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     const int n_tiles = static_cast<int>(ceil_div(tp.N, BN));
     const int total = n_tiles * static_cast<int>(ceil_div(tp.M, BM));
     const dim3 grid(static_cast<unsigned>(total < num_sms ? total : num_sms));
@@ -1329,21 +1325,17 @@ int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& 
 {
     using L = TmaSmem<BN, STAGES, W4>;
     auto kernel = tma_gemm_kernel<BN, STAGES, W4, ADD>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-        attr_set = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     const dim3 grid(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
                     static_cast<unsigned>(splits));
     return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, static_cast<unsigned>(splits), ta, tw, ty, tp);
 }
 
 // Reduction splits (cluster size): enough CTAs to cover the SMs, at least 4 k-blocks each.
-int pick_splits(int64_t tiles, int k_blocks)
+int pick_splits(int64_t tiles, int k_blocks, int num_sms)
 {
     int s = 1;
-    while (s < 8 && tiles * (2 * s) <= 148 && k_blocks / (2 * s) >= 2) s *= 2;
+    while (s < 8 && tiles * (2 * s) <= num_sms && k_blocks / (2 * s) >= 2) s *= 2;
     return s;
 }
 
@@ -1478,13 +1470,9 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     if (rc != MIXDQ_OK) return rc;
 
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, bn);
-    static int num_sms = 0;
-    if (!num_sms) {
-        int dev = 0;
-        MIXDQ_CUDA_TRY(cudaGetDevice(&dev));
-        MIXDQ_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
-    }
-    const bool persistent = tiles >= num_sms && p.force_splits <= 0;
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
+    const bool persistent = tiles >= num_sms;
     if (tp.tma_store) {
         // store box: 64 x 32 (128-byte swizzle) in the one-tile kernel, 32 x 32 (64-byte swizzle) in the
         // persistent one, whose staging tiles are smaller
@@ -1496,7 +1484,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
         if (persistent)
             return w4 ? launch_persistent<128, 6, true, true>(ta, tw, ty, tp, num_sms, stream)
                       : launch_persistent<128, 6, false, true>(ta, tw, ty, tp, num_sms, stream);
-        const int sp = pick_splits(tiles, tp.k_blocks);
+        const int sp = pick_splits(tiles, tp.k_blocks, num_sms);
         return w4 ? launch_tma<128, 6, true, true>(ta, tw, ty, tp, sp, stream)
                   : launch_tma<128, 6, false, true>(ta, tw, ty, tp, sp, stream);
     }
@@ -1505,11 +1493,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
         return w4 ? launch_persistent<128, 6, true>(ta, tw, ty, tp, num_sms, stream)
                   : launch_persistent<128, 6, false>(ta, tw, ty, tp, num_sms, stream);
     }
-    int splits = pick_splits(tiles, tp.k_blocks);
-    if (p.force_splits > 0) {
-        splits = 1;
-        while (splits * 2 <= p.force_splits && splits * 2 <= 8 && splits * 2 <= tp.k_blocks) splits *= 2;
-    }
+    const int splits = pick_splits(tiles, tp.k_blocks, num_sms);
     if (wide) return launch_tma<256, 4, false>(ta, tw, ty, tp, splits, stream);
     return w4 ? launch_tma<128, 6, true>(ta, tw, ty, tp, splits, stream)
               : launch_tma<128, 6, false>(ta, tw, ty, tp, splits, stream);
@@ -1587,7 +1571,6 @@ int run_tma_split(const Params& p, int amode, int split_at, const void* packed_l
     q.bias = nullptr;
     q.act_zero = nullptr;
     q.w_code_sums = nullptr;
-    q.force_splits = 0;
     q.acc_out = acc_lo;
     q.act_scale = scale_lo;
     q.Cin = conv ? split_at : 0;

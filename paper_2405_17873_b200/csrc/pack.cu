@@ -330,6 +330,20 @@ bool width_ok(int bits) { return bits == 2 || bits == 3 || bits == 4 || bits == 
 
 using namespace mixdq;
 
+// The layer kernels load a layer's constants (packed weights, scales, zero-points, code sums) before they
+// wait for earlier kernels of the stream, so a kernel that WRITES such constants must be complete, not merely
+// finishing, when the next layer call is enqueued behind it.  The entry points below that produce constants
+// therefore end with this empty kernel: launched plainly, it starts only after everything before it on the
+// stream has completed and its writes are visible, and whatever follows it overlaps nothing but it.
+__global__ void constants_complete_kernel() {}
+
+static int finish_constants(cudaStream_t st)
+{
+    if (cudaGetLastError() != cudaSuccess) return MIXDQ_ERR_CUDA;
+    constants_complete_kernel<<<1, 32, 0, st>>>();
+    return check_launch();
+}
+
 extern "C" int mixdq_packed_bytes(int64_t N, int64_t K, int bits, int layout, size_t* out)
 {
     if (!out || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
@@ -352,7 +366,7 @@ extern "C" int mixdq_weight_minmax_params(const void* W, int64_t N, int64_t K, i
     if (!symmetric && !zero_out) return MIXDQ_ERR_INVALID_ARG;
     weight_minmax_kernel<<<static_cast<unsigned>(N), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __half*>(W), K, bits, symmetric, scale_out, zero_out);
-    return check_launch();
+    return finish_constants(static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits, const float* scale,
@@ -368,7 +382,7 @@ extern "C" int mixdq_pack_weights(const void* W, int64_t N, int64_t K, int bits,
     pack_kernel<<<static_cast<unsigned>(ceil_div(words, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __half*>(W), N, K, bits, scale, zero, layout, pitch,
         static_cast<uint8_t*>(packed_out));
-    return check_launch();
+    return finish_constants(static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int mixdq_unpack_weights(const void* packed, int64_t N, int64_t K, int bits, int is_signed,
@@ -439,5 +453,5 @@ extern "C" int mixdq_weight_code_sums(const void* packed_W, int64_t N, int64_t K
     const int64_t pitch = row_pitch_bytes(K, bits, MIXDQ_LAYOUT_DEVICE);
     code_sums_kernel<<<static_cast<unsigned>(N), 128, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(packed_W), K, bits, pitch, sums_out);
-    return check_launch();
+    return finish_constants(static_cast<cudaStream_t>(stream));
 }

@@ -4,8 +4,10 @@
 // memory manager has already claimed the whole GPU, a plug-in that runs inside another
 // framework's allocator and must not go around it, or a latency-critical loop where the
 // implicit device-wide synchronization of cudaMalloc / cudaFree is not acceptable.  For them
-// the split-reduction scratch of the int8 linear layer lives in a fixed array inside the
-// library image instead of a caller-provided workspace.
+// the scratch of the int8 linear layer -- above all the int8 copy of the activations that the
+// quantization pass writes and the GEMM kernel reads, behind the region reserved for a split
+// reduction -- lives in a fixed array inside the library image instead of a caller-provided
+// workspace.
 #include <mutex>
 
 #include "common.cuh"
@@ -60,9 +62,10 @@ extern "C" int mixdq_linear_a8_static_scratch(const void* X, int64_t M, int64_t 
     int rc = scratch_address(&scratch);
     if (rc != MIXDQ_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the array keeps whatever the previous call (possibly an aborted one) left behind, and the
-    // reduction needs its counters and partial sums to start at zero
-    MIXDQ_CUDA_TRY(cudaMemsetAsync(scratch, 0, need, st));
+    // The array keeps whatever the previous call left behind.  Nothing in it has to start at zero for
+    // the kernels reached from here: the quantization pass overwrites every byte of the int8 copy that
+    // the GEMM reads, and the one user of counters that start at zero (the split reduction of the
+    // single-kernel form) clears its region itself before it launches.
     i8::Params p;
     p.X = static_cast<const __half*>(X);
     p.ldx = ldx;

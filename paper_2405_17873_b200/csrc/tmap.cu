@@ -107,19 +107,72 @@ static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const voi
     return r == CUDA_SUCCESS ? MIXDQ_OK : MIXDQ_ERR_CUDA;
 }
 
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+// Function attributes and device properties belong to a device: everything cached here is keyed by it.
+int current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    return (dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+
+}  // namespace
+
 int prefer_max_shared_carveout(const void* kernel)
 {
     static std::mutex mu;
-    static std::unordered_set<const void*> done;
+    static std::unordered_set<const void*> done[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return MIXDQ_ERR_CUDA;
     std::lock_guard<std::mutex> lock(mu);
-    if (done.count(kernel)) return MIXDQ_OK;
+    if (done[dev].count(kernel)) return MIXDQ_OK;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
         cudaSuccess) {
         (void)cudaGetLastError();
         return MIXDQ_ERR_CUDA;
     }
-    done.insert(kernel);
+    done[dev].insert(kernel);
     return MIXDQ_OK;
+}
+
+int ensure_dynamic_smem(const void* kernel, int bytes)
+{
+    static std::mutex mu;
+    static std::unordered_set<const void*> done[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return MIXDQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[dev].count(kernel)) return MIXDQ_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MIXDQ_ERR_CUDA;
+    }
+    done[dev].insert(kernel);
+    return MIXDQ_OK;
+}
+
+int sm_count()
+{
+    static std::mutex mu;
+    static int count[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!count[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return 0;
+        }
+        count[dev] = n;
+    }
+    return count[dev];
 }
 
 }  // namespace mixdq

@@ -482,15 +482,10 @@ int launch_small_tiles(const Params& p, const void* packed, long long pitch, cud
     const int k_pad = static_cast<int>(round_up(p.K, kUnit));
     const size_t smem = static_cast<size_t>(MB) * (k_pad * 2 + 16) + 8 * 16 * MB * sizeof(float);
     auto kernel = wo_small_kernel<BITS, SIGNED, NT, TILES>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            16 * (kSmallKMax * 2 + 64) + 8 * 16 * 16 * 4));
-        attr_set = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), 16 * (kSmallKMax * 2 + 64) + 8 * 16 * 16 * 4) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     // groups of TILES channel tiles are dealt to CTAs in equal rounds of at most three CTAs per SM
     const int groups = static_cast<int>(ceil_div(p.N, 16 * TILES));
-    const int rounds = static_cast<int>(ceil_div(groups, 444));
+    const int rounds = static_cast<int>(ceil_div(groups, 3 * (sm_count() > 0 ? sm_count() : 1)));
     const dim3 grid(static_cast<unsigned>(ceil_div(groups, rounds)));
     return launch_pdl(kernel, grid, dim3(kThreads), smem, stream, 1, static_cast<const uint8_t*>(packed), pitch, p,
                       groups, k_pad);
@@ -500,7 +495,7 @@ template <int BITS, bool SIGNED, int NT>
 int launch_small(const Params& p, const void* packed, long long pitch, cudaStream_t stream)
 {
     // one channel tile per CTA (more reduction slices) when two per CTA would leave SMs idle
-    if (ceil_div(p.N, 32) < 148) return launch_small_tiles<BITS, SIGNED, NT, 1>(p, packed, pitch, stream);
+    if (ceil_div(p.N, 32) < sm_count()) return launch_small_tiles<BITS, SIGNED, NT, 1>(p, packed, pitch, stream);
     return launch_small_tiles<BITS, SIGNED, NT, 2>(p, packed, pitch, stream);
 }
 
@@ -511,12 +506,7 @@ int launch(const Params& p, int amode, const void* packed, long long pitch, cuda
     const int chunk_len = static_cast<int>(p.K > kChunkMax ? kChunkMax : round_up(p.K, kUnit));
     const size_t smem = static_cast<size_t>(MB) * (chunk_len * 2 + 64) + kSlices * kChanPerCta * MB * sizeof(float);
     auto kernel = wo_kernel<BITS, SIGNED, NT>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            32 * (kChunkMax * 2 + 64) + kSlices * kChanPerCta * 32 * 4));
-        attr_set = true;
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), 32 * (kChunkMax * 2 + 64) + kSlices * kChanPerCta * 32 * 4) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     dim3 grid(static_cast<unsigned>(ceil_div(p.N, kChanPerCta)), static_cast<unsigned>(ceil_div(p.M, MB)));
     return launch_pdl(kernel, grid, dim3(kThreads), smem, stream, 1, static_cast<const uint8_t*>(packed), pitch, p,
                       amode, chunk_len);

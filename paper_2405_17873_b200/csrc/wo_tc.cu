@@ -414,17 +414,9 @@ template <int BITS, bool SIGNED>
 int launch_tc(const CUtensorMap& tx, const TcParams& tp, cudaStream_t stream)
 {
     auto kernel = wo_tc_kernel<BITS, SIGNED>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MIXDQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL));
-        attr_set = true;
-    }
-    static int num_sms = 0;
-    if (!num_sms) {
-        int dev = 0;
-        MIXDQ_CUDA_TRY(cudaGetDevice(&dev));
-        MIXDQ_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
-    }
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), SMEM_TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
     const int n_tiles = static_cast<int>(ceil_div(tp.N, BN));
     const int total = n_tiles * static_cast<int>(ceil_div(tp.M, BM));
     const dim3 grid(static_cast<unsigned>(total < num_sms ? total : num_sms));

@@ -149,19 +149,21 @@ def new_workspace(nbytes: int, device="cuda") -> Optional[torch.Tensor]:
     return torch.zeros(nbytes, dtype=torch.uint8, device=device)
 
 
-def weight_minmax_params(W: torch.Tensor, bits: int, symmetric: bool):
+def weight_minmax_params(W: torch.Tensor, bits: int, symmetric: bool, scale_out: Optional[torch.Tensor] = None,
+                         zero_out: Optional[torch.Tensor] = None):
     N, K = W.shape
-    scale = torch.empty(N, dtype=torch.float32, device=W.device)
-    zero = torch.zeros(N, dtype=torch.int32, device=W.device)
+    scale = scale_out if scale_out is not None else torch.empty(N, dtype=torch.float32, device=W.device)
+    zero = zero_out if zero_out is not None else torch.zeros(N, dtype=torch.int32, device=W.device)
     _chk(lib().mixdq_weight_minmax_params(_ptr(W), N, K, bits, int(symmetric), _ptr(scale), _ptr(zero),
                                           _stream()), "mixdq_weight_minmax_params")
     return scale, zero
 
 
 def pack_weights(W: torch.Tensor, bits: int, scale: torch.Tensor, zero: Optional[torch.Tensor] = None,
-                 layout: int = LAYOUT_DEVICE) -> torch.Tensor:
+                 layout: int = LAYOUT_DEVICE, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     N, K = W.shape
-    out = torch.zeros(packed_bytes(N, K, bits, layout), dtype=torch.uint8, device=W.device)
+    if out is None:
+        out = torch.zeros(packed_bytes(N, K, bits, layout), dtype=torch.uint8, device=W.device)
     _chk(lib().mixdq_pack_weights(_ptr(W), N, K, bits, _ptr(scale), _ptr(zero), layout, _ptr(out), _stream()),
          "mixdq_pack_weights")
     return out

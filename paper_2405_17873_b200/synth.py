@@ -99,6 +99,13 @@ def text_embedding(B: int, seed: int = 4000, n_outlier_ch: int = 8, outlier_mag:
     return E.to(torch.float16).numpy()
 
 
+def bos_projection(e_bos: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+    """The stored BOS row of a K/V projection: the UNQUANTIZED fp16 layer applied to the BOS embedding,
+    accumulated in float64 and rounded once to fp16 (Sec. 3.1: this row is computed ahead of time in
+    floating point and never quantized).  Works on tensors of any device."""
+    return (W.to(torch.float64) @ e_bos.to(torch.float64)).to(torch.float16).contiguous()
+
+
 def kv_weight(N: int, seed: int) -> np.ndarray:
     return normal_f16((N, TEXT_DIM), 0.02, seed)
 

@@ -122,8 +122,7 @@ class UNetSweep:
             if l.kind == "bos_kv":
                 bias = None
                 if l.a_bits == 8:
-                    e0 = self.x[xk][0, 0].to(torch.float32)
-                    bos = (W.to(torch.float32) @ e0).to(torch.float16).contiguous()
+                    bos = synth.bos_projection(self.x[xk][0, 0], W)
             sums = None
             # convolutions whose geometry the two-kernel path does not take (conv_in: 4 channels) stay symmetric
             if self.act_asym and l.a_bits == 8 and (l.kind in ("linear", "conv1x1") or (l.kind == "conv3x3" and l.Cin % 32 == 0)):

@@ -1,8 +1,10 @@
-"""Parity at the full layer sizes of the SDXL-turbo-shaped UNet sweep (image batch 4), through
-the same entry points and with the same workspace the benchmark uses.  The oracle computes a
-sample of output rows one by one (a 3x3 conv output pixel is a dot product over its gathered
-window, which the CPU suite pins against the direct convolution); int32 accumulators of the
-sampled rows must match bit for bit, fp16 outputs within the path's tolerance."""
+"""Parity at full layer sizes of the SDXL-turbo-shaped UNet sweep (image batch 4) for the cases the census
+tests (test_gpu_census.py: every distinct shape, whole tensors on the int8 path) do not cover: the
+weight-bound regime of 16 tokens at full layer width, and the shortcut-split layers.  The oracle computes
+one output row in every 128-row tile, at a position that moves through the tile, plus the first and last
+rows (a 3x3 conv output pixel is a dot product over its gathered window, which the CPU suite pins against
+the direct convolution); int32 accumulators of those rows must match bit for bit, fp16 outputs within the
+path's tolerance."""
 import numpy as np
 import pytest
 import torch
@@ -17,9 +19,12 @@ B = 4
 _SPECS = {l.name: l for l in synth.unet_layers()}
 
 
-def _sample_rows(total, n=10, seed=0):
-    rng = np.random.default_rng(seed)
-    rows = set(rng.integers(0, total, size=n).tolist()) | {0, total - 1, min(127, total - 1), min(128, total - 1)}
+def _sample_rows(total, seed=0):
+    """One row of every 128-row tile, at an in-tile position that depends on the tile (and the layer), plus
+    the first and last rows and the rows either side of the first tile boundary."""
+    rows = {0, total - 1, min(127, total - 1), min(128, total - 1)}
+    for t in range((total + 127) // 128):
+        rows.add(min(total - 1, t * 128 + (37 * t + 5 + 11 * seed) % 128))
     return np.array(sorted(rows))
 
 
@@ -115,23 +120,6 @@ def _check_layer(name, w_bits, a_bits, rows_override=None):
         torch.cuda.synchronize()
         assert int(host(st)[0]) == 0
         _close(y[rows], y_ref)
-
-
-@pytest.mark.parametrize("name,w_bits", [
-    ("ffn1_1280#0", 4), ("ffn1_1280#1", 8), ("ffn2_1280#0", 4), ("attn_1280#0", 4), ("attn_640#0", 8),
-    ("ffn1_640#0", 4), ("kv_1280#0", 8), ("kv_640#0", 4), ("up64_640#0", 4), ("res64_320_320#0", 8),
-    ("res32_1920_640#0", 4), ("res16_2560_1280#0", 4), ("down64_320#0", 4), ("sc64_960#0", 4),
-    ("conv_in#0", 8), ("conv_out#0", 8), ("time_emb1#0", 4), ("add_emb1#0", 8)])
-def test_int8_layers_full_size(name, w_bits):
-    _check_layer(name, w_bits, 8)
-
-
-@pytest.mark.parametrize("name,w_bits", [
-    ("ffn1_1280#0", 3), ("ffn1_1280#1", 4), ("ffn2_1280#0", 8), ("attn_1280#0", 3), ("kv_1280#0", 4),
-    ("res64_320_320#0", 3), ("up32_1280#0", 4), ("res16_2560_1280#0", 8), ("down32_640#0", 3),
-    ("conv_in#0", 8), ("conv_out#0", 8), ("res_time_640#0", 4)])
-def test_weight_only_layers_full_size(name, w_bits):
-    _check_layer(name, w_bits, 16)
 
 
 @pytest.mark.parametrize("name,w_bits", [("ffn1_1280#0", 3), ("ffn1_1280#0", 4), ("ffn2_1280#0", 4),

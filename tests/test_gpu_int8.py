@@ -249,3 +249,33 @@ def test_conv1x1_equals_linear():
     s, _, packed = device_weights(Wt, 4, True)
     y = mixdq.conv1x1(Xd, packed, 48, 4, s, None, 8, mixdq.act_scale(Xd), None)
     assert_close(host(y).reshape(-1, 48), y_ref)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_pack_then_layer_on_one_stream_without_synchronization(bits):
+    """The layer kernels load their weights before they wait for earlier kernels of the stream; the pack entry
+    points end with a full stream dependency so that a layer call enqueued right behind them, with no
+    synchronization, still reads complete weights.  The same packed buffer is rewritten for every round."""
+    M, K, N = 256, 1280, 640
+    X = synth.normal_f16((M, K), 1.0, seed=77)
+    Xd = dev(X)
+    sx = mixdq.act_scale(Xd)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    st = status_word()
+    ws = workspace_for(M, N, K, bits)
+    packed = torch.zeros(mixdq.packed_bytes(N, K, bits), dtype=torch.uint8, device="cuda")
+    s = torch.zeros(N, dtype=torch.float32, device="cuda")
+    Ws = [synth.normal_f16((N, K), 0.02 * (1 + r), seed=780 + r) for r in range(6)]
+    Wd = [dev(W) for W in Ws]
+    outs = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in Ws]
+    torch.cuda.synchronize()
+    for r in range(len(Ws)):
+        mixdq.weight_minmax_params(Wd[r], bits, True, scale_out=s)
+        mixdq.pack_weights(Wd[r], bits, s, out=packed)
+        mixdq.linear(Xd, packed, N, bits, s, None, 8, sx, None, workspace=ws, status=st, out=outs[r])
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    for r, W in enumerate(Ws):
+        s_ref, _, codes = oracle_weights(W, bits, True)
+        _, y_ref = orc.linear_a8(X, codes, s_ref, sx_ref, None)
+        assert_close(host(outs[r]), y_ref)

@@ -52,18 +52,45 @@ def _exact_code(v: Fraction, inv: Fraction) -> int:
     return fl
 
 
+def _exact_codes_int64(X: np.ndarray, inv32: np.float32) -> np.ndarray:
+    """Nearest integer (ties to even) to x * inv for every fp16 x, in exact integer arithmetic: x = mx * 2^ex
+    and inv = mi * 2^ei with integer mantissas (11 and 24 bits), so the product is the 35-bit integer mx * mi
+    times a power of two, and the rounding is a shift with an explicit look at the bits shifted out."""
+    m, e = np.frexp(X.astype(np.float64))
+    mx = np.rint(m * 2048.0).astype(np.int64)            # exact: fp16 mantissas have at most 11 bits
+    assert np.array_equal(mx.astype(np.float64) * np.exp2(e - 11.0), X.astype(np.float64))
+    mi_f, ei = np.frexp(np.float64(inv32))
+    mi = int(round(mi_f * 2.0 ** 24))
+    assert mi * 2.0 ** (int(ei) - 24) == float(inv32)
+    n = np.abs(mx) * mi                                   # |product| = n * 2^sh
+    sh = (e.astype(np.int64) - 11) + (int(ei) - 24)
+    out = np.zeros(X.shape, np.int64)
+    up = sh >= 0
+    out[up] = n[up] << np.minimum(sh[up], 20)             # far beyond the clamp either way
+    dn = ~up
+    s = np.minimum(-sh[dn], 62)                           # n < 2^35: anything shifted further is 0 with a small remainder
+    fl = n[dn] >> s
+    rem = n[dn] - (fl << s)
+    half = np.int64(1) << (s - 1)
+    fl = fl + ((rem > half) | ((rem == half) & (fl % 2 == 1)))
+    out[dn] = fl
+    return np.where(mx < 0, -out, out)
+
+
 @pytest.mark.parametrize("scale", [0.03125, 0.0371, 1.0 / 127.0, 0.4321, 3.0e-4])
 def test_act_codes_all_fp16_patterns_vs_exact_rationals(scale):
     finite = np.isfinite(ALL_HALF)
     X = ALL_HALF[finite]
     got = orc.quantize_acts(X, np.float32(scale), 8)
     inv32 = np.float32(1.0) / np.float32(scale)          # numpy's IEEE fp32 divide
+    # every finite pattern, in exact integer arithmetic
+    want = np.clip(_exact_codes_int64(X, inv32), -127, 127)
+    assert np.array_equal(got.astype(np.int64), want)
+    # and the integer routine itself against Python rationals on a strided sample
     inv = Fraction(float(inv32))
-    # checking every pattern in Python rationals is slow; take a strided third plus all ties
-    idx = np.arange(0, X.size, 3)
-    for i in idx:
+    for i in range(0, X.size, 97):
         q = max(-127, min(127, _exact_code(Fraction(float(X[i])), inv)))
-        assert int(got[i]) == q, (float(X[i]), scale)
+        assert int(want[i]) == q, (float(X[i]), scale)
 
 
 def test_act_codes_ties_round_to_even():
