@@ -1,0 +1,575 @@
+// Pair form of the W8A8 / W4A8 GEMM for the large layers: two CTAs on neighbouring SMs (a cluster of two)
+// share one 256 x BN output tile and one stream of tensor-core instructions (tcgen05.mma.cta_group::2).
+//
+// Why: the single-CTA kernels in i8_tma.cu are bound by the bytes a CTA can keep in flight, not by the tensor
+// pipe.  A 128 x 128 x 128 k-block needs 32 KB of operands (24 KB with int4 weights) for 256 cycles of MMA
+// work, a ring slot is away for about 1900 cycles, and shared memory holds six such k-blocks: one k-block per
+// 330 cycles at best.  In the pair form each CTA still loads its own 128 rows of activations per k-block but
+// only HALF of the weight tile (BN / 2 rows), and one instruction covers 256 x BN x 32: at BN = 256 the same
+// 32 KB per CTA feed 512 cycles of MMA work, so the rings run ahead of the tensor pipe instead of behind it,
+// and the tensor pipe, not the operand delivery, sets the pace.
+//
+// Roles.  Both CTAs run the same program.  Activation and weight producers of BOTH CTAs load into their own
+// shared memory and signal the barriers of the pair's first CTA (the leader) -- plain TMA loads of this GPU's
+// memory with the cta_group::2 qualifier, which is what lets the barrier live in the peer CTA; nothing is
+// multicast.  Two threads of the leader issue the MMAs, which read both CTAs' shared memory and write both
+// CTAs' tensor memory (each CTA holds the 128 accumulator rows of its own activations), and hands slots back
+// with commits that arrive on the barriers of both CTAs.  int4 weights are expanded by each CTA's own warps
+// into its own half of the int8 weight tile; the peer's expansion warps arrive on the leader's barrier.  Each
+// CTA's epilogue warps dequantize and store its own 128 rows.  Tiles are walked persistently with two
+// accumulators of 256 columns each, so a tile's epilogue overlaps the next tile's main loop.
+//
+// BN is a run-time value (a multiple of 32 up to 256) chosen per layer so that the tiles fill whole rounds of
+// the SM pairs; shared-memory slots have the size of the widest tile.
+#include "i8_tiles.cuh"
+
+namespace mixdq {
+namespace i8 {
+
+namespace {
+
+// ---------------------------------------------------------------- PTX of the pair (cta_group::2) forms
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// Address of this CTA's shared-memory location `addr` as seen in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
+    return out;
+}
+
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem of both CTAs] (+)= A[both CTAs' smem, 128 rows each] * B[both CTAs' smem, N / 2 rows each]^T.
+__device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Once every MMA this thread issued so far has completed: arrive on the barrier at this shared-memory offset
+// in both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(both)
+                 : "memory");
+}
+
+// TMA tile loads into this CTA's shared memory whose completion is counted on a barrier of the leader CTA
+// (`bar` is an address in the cluster's shared window).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+
+// Arrive on a barrier that may belong to the other CTA of the cluster (address in the cluster's shared
+// window).  Default semantics, as for a local arrive: a release at cluster scope was measured to cost the
+// arriving thread some 2000 cycles per call (it turned a 550-cycle expansion turn into a 2600-cycle one).
+// What the arrival publishes are shared-memory tiles for the tensor core, and those are ordered by the
+// fence.proxy.async that every writer executes before its warp's arrival.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// ---------------------------------------------------------------- shared memory of one CTA of the pair
+
+constexpr int PAIR_BN_MAX = 256;
+constexpr int ACC_COLS = 256;  // tensor-memory columns of one accumulator (the widest tile)
+
+template <bool W4>
+struct PairSmem {
+    static constexpr int A_BYTES = BM * BK;                 // this CTA's 128 activation rows of a k-block
+    static constexpr int B_BYTES = (PAIR_BN_MAX / 2) * BK;  // this CTA's half of the int8 weight tile
+    static constexpr int P_BYTES = B_BYTES / 2;             // the same as packed int4
+    // Depths: everything that is in flight from L2 as deep as shared memory allows; the expanded int8 tiles of
+    // the W4 form are staging, one per expansion group.
+    // W4: the packed ring must be deeper than the number of expansion groups, or the request for a group's
+    // next tile goes out only when its last one has been expanded and the groups stall together once per lap.
+    static constexpr int AS = W4 ? 5 : 6;
+    static constexpr int ES = W4 ? 4 : 6;
+    static constexpr int PS = W4 ? 6 : 0;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_B = OFF_A + AS * A_BYTES;
+    static constexpr int OFF_P = OFF_B + ES * B_BYTES;
+    static constexpr int RINGS_END = OFF_P + PS * P_BYTES;
+    // barriers (8 bytes each).  FULL_A, READY_B, ACC_EMPTY are used in the leader only (both CTAs signal them);
+    // the others exist in both CTAs and are signalled by the leader's commits or by local producers.
+    static constexpr int FULL_A = 0;              // activation tiles of both CTAs have landed
+    static constexpr int EMPTY_A = FULL_A + AS;   // MMAs reading the k-block's activation tiles (W8: and weights) have finished
+    static constexpr int READY_B = EMPTY_A + AS;  // W8: weight halves of both CTAs have landed; W4: both expanded
+    static constexpr int EMPTY_B = READY_B + ES;  // W4: MMAs reading the int8 weight tiles have finished
+    static constexpr int FULL_P = EMPTY_B + ES;   // W4: this CTA's packed half has landed
+    static constexpr int EMPTY_P = FULL_P + PS;   // W4: this CTA's packed half has been read
+    static constexpr int ACC_FULL = EMPTY_P + PS;     // [2]
+    static constexpr int ACC_EMPTY = ACC_FULL + 2;    // [2]
+    static constexpr int TILE_GO = ACC_EMPTY + 2;     // leader: the first issuer has issued k-block 0 of a tile
+    static constexpr int NUM_BARS = TILE_GO + 1;
+    static constexpr int OFF_BARS = RINGS_END;
+    static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][PAIR_BN_MAX] floats
+    static constexpr int OFF_BIAS = OFF_COMB + 2 * PAIR_BN_MAX * 4;
+    static constexpr int OFF_MISC = OFF_BIAS + 2 * PAIR_BN_MAX * 4;
+    static constexpr int OFF_EPI = (OFF_MISC + 64 + 1023) & ~1023;  // staging tiles of the eight epilogue warps
+    static constexpr int TOTAL = OFF_EPI + 8 * EPI32_TILE + 1024;
+    static_assert(TOTAL <= 232448, "shared memory of one CTA");
+    // warps: 0 activation producer, 1 MMA issuer (leader) and tensor-memory allocation, 2-5 epilogue (first part
+    // of the columns), W4: 6-13 nibble expansion, then four epilogue helpers (the other columns), then the weight
+    // producer
+    static constexpr int HELPER0 = W4 ? 14 : 6;
+    static constexpr int B_WARP = HELPER0 + 4;
+    static constexpr int MMA2_WARP = B_WARP + 1;  // second MMA issuer (leader)
+    static constexpr int THREADS = (MMA2_WARP + 1) * 32;
+};
+
+struct PairArgs {
+    int bn;           // tile width (multiple of 32, <= 256); each CTA holds bn / 2 weight rows
+    int n_tiles;      // tiles along N
+    int total_tiles;  // pair tiles in all
+};
+
+template <bool W4>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairSmem<W4>::THREADS, 1)
+pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                 const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, const PairArgs g)
+{
+    using L = PairSmem<W4>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~static_cast<uintptr_t>(1023));
+    uint8_t* sB = smem + L::OFF_B;
+    const uint8_t* sP = smem + L::OFF_P;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
+    float* s_comb = reinterpret_cast<float*>(smem + L::OFF_COMB);
+    float* s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: leader
+    const bool leader = rank == 0;
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int nkb = p.k_blocks;
+    const int bn = g.bn, bh = g.bn >> 1;
+    const int my_tiles = (g.total_tiles - pair + npairs - 1) / npairs;
+
+    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t a0 = smem_u32(smem + L::OFF_A), b0 = smem_u32(sB), p0 = smem_u32(smem + L::OFF_P);
+    // the same barriers as seen in the leader CTA (for the leader: its own)
+    const uint32_t lead_bar0 = map_to_cta(bar0, 0);
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < L::AS; ++s) {
+            mbar_init(bar0 + 8 * (L::FULL_A + s), 1);   // the leader's producer arms it with the bytes of both CTAs
+            mbar_init(bar0 + 8 * (L::EMPTY_A + s), 1);  // one commit
+        }
+        for (int s = 0; s < L::ES; ++s) {
+            mbar_init(bar0 + 8 * (L::READY_B + s), W4 ? 4 : 1);  // W4: two expansion warps of each CTA
+            mbar_init(bar0 + 8 * (L::EMPTY_B + s), 1);
+        }
+        for (int s = 0; s < L::PS; ++s) {
+            mbar_init(bar0 + 8 * (L::FULL_P + s), 1);
+            mbar_init(bar0 + 8 * (L::EMPTY_P + s), 2);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar0 + 8 * (L::ACC_FULL + b), 2);    // one commit of each issuer
+            mbar_init(bar0 + 8 * (L::ACC_EMPTY + b), 16);  // eight epilogue warps of each CTA
+        }
+        mbar_init(bar0 + 8 * L::TILE_GO, 1);
+        *s_abort = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_w);
+        if (p.tma_store) tma_prefetch_desc(&tmap_y);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(s_tmem), 2 * ACC_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    // no CTA signals a barrier of its peer before that barrier exists
+    cluster_sync();
+    tc_fence_after_sync();
+    // everything above is independent of earlier kernels; global memory is not, except the packed weights
+    // (constants of the layer), whose producer runs ahead
+    if (warp != L::B_WARP) pdl_wait();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ activation-tile producer (own 128 rows)
+        if (lane == 0) {
+            uint32_t s = 0, par = 1;  // slots start out free: the first lap waits on the phase "before" phase 0
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = pair + t * npairs;
+                const int m0 = (tile / g.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM;
+                int img_b = 0, ho0 = 0, wo0 = 0, cb = 0, kh = 0, kw = 0, xa = 0;
+                if (p.conv) {
+                    img_b = m0 / p.HoWo;
+                    const int rem = m0 - img_b * p.HoWo;
+                    ho0 = rem / p.Wo;
+                    wo0 = rem - ho0 * p.Wo;
+                }
+                for (int i = 0; i < nkb; ++i) {
+                    if (!mbar_wait(bar0 + 8 * (L::EMPTY_A + s), par, s_abort)) {
+                        ok = false;
+                        break;
+                    }
+                    if (leader) mbar_arrive_expect_tx(bar0 + 8 * (L::FULL_A + s), 2 * L::A_BYTES);
+                    const uint32_t full = lead_bar0 + 8 * (L::FULL_A + s);
+                    if (p.conv) {
+                        tma_load_4d_pair(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1 + p.pad,
+                                         p.stride * ho0 + kh - 1 + p.pad, img_b, full);
+                        if (++cb == p.cblocks) {
+                            cb = 0;
+                            if (++kw == 3) {
+                                kw = 0;
+                                ++kh;
+                            }
+                        }
+                    } else {
+                        tma_load_2d_pair(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
+                        xa += BK;
+                    }
+                    if (++s == L::AS) {
+                        s = 0;
+                        par ^= 1;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == L::B_WARP) {
+        // ------------------------------------------------------------ weight-tile producer (own half of the rows)
+        if (lane == 0) {
+            constexpr int R = W4 ? L::PS : L::ES;
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            uint32_t s = 0, par = 1;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = pair + t * npairs;
+                const int n0 = (tile % g.n_tiles) * bn + static_cast<int>(rank) * bh;
+                int cb = 0, kx_tap = 0, xb = 0;
+                for (int i = 0; i < nkb; ++i) {
+                    // W8: the commit that frees the activation slot frees the weight slot (the rings move in lockstep)
+                    if (!mbar_wait(bar0 + 8 * ((W4 ? L::EMPTY_P : L::EMPTY_A) + s), par, s_abort)) {
+                        ok = false;
+                        break;
+                    }
+                    int x = xb;
+                    if (p.conv) {
+                        const int kx = kx_tap + cb * BK;
+                        x = W4 ? kx / 2 : kx;
+                        if (++cb == p.cblocks) {
+                            cb = 0;
+                            kx_tap += p.Cin;
+                        }
+                    }
+                    xb += ROW_BYTES;
+                    if (W4) {
+                        // packed rows are consumed inside this CTA: a barrier of its own
+                        const uint32_t full = bar0 + 8 * (L::FULL_P + s);
+                        mbar_arrive_expect_tx(full, static_cast<uint32_t>(bh * ROW_BYTES));
+                        tma_load_2d(p0 + s * L::P_BYTES, &tmap_w, x, n0, full);
+                    } else {
+                        if (leader) mbar_arrive_expect_tx(bar0 + 8 * (L::READY_B + s), static_cast<uint32_t>(bn * ROW_BYTES));
+                        tma_load_2d_pair(b0 + s * L::B_BYTES, &tmap_w, x, n0, lead_bar0 + 8 * (L::READY_B + s));
+                    }
+                    if (++s == R) {
+                        s = 0;
+                        par ^= 1;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1 || warp == L::MMA2_WARP) {
+        // ------------------------------------------------------------ MMA issuers (two threads of the leader)
+        // One thread needs some 650 cycles per k-block (four MMAs at about 62 cycles each, two waits, a commit
+        // whose cost to its thread is several times an MMA's, the loop) against 512 cycles of tensor-pipe work,
+        // and the pipe idles whenever its queue runs dry in between.  Two threads therefore alternate: warp 1
+        // takes the even k-blocks of a tile, the second issuer the odd ones, both into the SAME accumulator --
+        // the sums are integers, so the order in which the pipe adds the k-blocks does not matter, except that
+        // the MMA that overwrites the accumulator (the first of k-block 0) must come first: the second issuer
+        // starts a tile only after the first has issued k-block 0 (TILE_GO, with the tcgen05 fences that order
+        // the two threads' instructions).  A tile is complete when both threads' commits have arrived.
+        if (lane == 0 && leader) {
+            const int which = warp == 1 ? 0 : 1;
+            const uint32_t idesc = make_idesc(2, 1, 2 * BM, static_cast<uint32_t>(bn));
+            const uint64_t a_desc0 = smem_desc_sw128(a0), b_desc0 = smem_desc_sw128(b0);
+            const uint32_t tile_go = bar0 + 8 * L::TILE_GO;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int buf = t & 1;
+                const uint32_t use = static_cast<uint32_t>(t >> 1);  // how often this accumulator was used before
+                ok = mbar_wait(bar0 + 8 * (L::ACC_EMPTY + buf), (use & 1) ^ 1, s_abort);
+                if (!ok) break;
+                if (which == 1 && nkb > 1) {
+                    ok = mbar_wait(tile_go, t & 1, s_abort);
+                    if (!ok) break;
+                }
+                tc_fence_after_sync();
+                const uint32_t acc = tmem_base + buf * ACC_COLS;
+                // position of this thread's first k-block of the tile in the CTA's running sequence
+                uint32_t q = static_cast<uint32_t>(t) * static_cast<uint32_t>(nkb) + which;
+                uint32_t sa = q % L::AS, pa = (q / L::AS) & 1, se = q % L::ES, pe = (q / L::ES) & 1;
+                for (int i = which; i < nkb; i += 2) {
+                    if (!mbar_wait(bar0 + 8 * (L::FULL_A + sa), pa, s_abort) ||
+                        !mbar_wait(bar0 + 8 * (L::READY_B + se), pe, s_abort)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint64_t a_desc = a_desc0 + sa * (L::A_BYTES >> 4);
+                    const uint64_t b_desc = b_desc0 + se * (L::B_BYTES >> 4);
+                    mma_i8_pair(acc, a_desc, b_desc, idesc, i != 0);
+#pragma unroll
+                    for (int k = 1; k < BK / 32; ++k) mma_i8_pair(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
+                    if (i == 0 && nkb > 1) {
+                        // the overwriting MMA is in the pipe's queue: the other thread may add to the accumulator
+                        tc_fence_before_sync();
+                        mbar_arrive(tile_go);
+                    }
+                    tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa));
+                    if (W4) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se));
+                    sa += 2;
+                    if (sa >= static_cast<uint32_t>(L::AS)) {
+                        sa -= L::AS;
+                        pa ^= 1;
+                    }
+                    se += 2;
+                    if (se >= static_cast<uint32_t>(L::ES)) {
+                        se -= L::ES;
+                        pe ^= 1;
+                    }
+                }
+                // (a thread without a k-block in this tile still arrives: its commit has nothing to wait for)
+                if (ok) tc_commit_pair(bar0 + 8 * (L::ACC_FULL + buf));
+            }
+        }
+        __syncwarp();
+    } else if (warp < 6 || (warp >= L::HELPER0 && warp < L::HELPER0 + 4)) {
+        // ------------------------------------------------------------ epilogue warps and helpers (own 128 rows)
+        const int lg = warp & 3;
+        const int half = warp < 6 ? 0 : 1;
+        const int et = tid - 64;  // epilogue warps only: 0..127
+        const float sx = p.act_scale ? __ldg(p.act_scale) : 0.f;  // absent: accumulators only
+        const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
+        // the 32-column passes of a tile are dealt to the two halves of the warps
+        const int passes = bn >> 5;
+        const int c_begin = half == 0 ? 0 : ((passes + 1) >> 1) * 32;
+        const int c_count = half == 0 ? ((passes + 1) >> 1) * 32 : (passes >> 1) * 32;
+        uint8_t* stage = smem + L::OFF_EPI + (half * 4 + lg) * EPI32_TILE;
+        const uint32_t lead_acc_empty = lead_bar0 + 8 * L::ACC_EMPTY;
+        bool ok = true;
+        for (int t = 0; t < my_tiles; ++t) {
+            const int tile = pair + t * npairs;
+            const int m0 = (tile / g.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM, n0 = (tile % g.n_tiles) * bn;
+            const int buf = t & 1;
+            const uint32_t use = static_cast<uint32_t>(t >> 1);
+            float* comb = s_comb + buf * PAIR_BN_MAX;
+            float* bias = s_bias + buf * PAIR_BN_MAX;
+            // this tile's per-column factors (the buffer was last read two tiles ago)
+            for (int j = et; half == 0 && j < bn; j += 128) {
+                const int n = n0 + j;
+                float c = 0.f, b = 0.f;
+                if (n < p.N && p.w_scale) {
+                    c = sx * __ldg(p.w_scale + n);
+                    if (p.bias) b = __half2float(p.bias[n]);
+                    if (p.act_zero) b = fmaf(static_cast<float>(zshift * __ldg(p.w_code_sums + n)), c, b);
+                }
+                comb[j] = c;
+                bias[j] = b;
+            }
+            if (ok) ok = mbar_wait(bar0 + 8 * (L::ACC_FULL + buf), use & 1, s_abort);
+            tc_fence_after_sync();
+            // the factor tables are complete; the same barrier carries the vote on whether every warp's wait
+            // succeeded, so that all eight take the same path from here
+            uint32_t go;
+            asm volatile(
+                "{\n\t"
+                ".reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "barrier.cta.red.and.pred p, 1, 256, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t"
+                "}\n"
+                : "=r"(go)
+                : "r"((ok && !*s_abort) ? 1u : 0u)
+                : "memory");
+            if (!go) {
+                ok = false;
+                continue;
+            }
+            const uint32_t acc = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
+            if (p.acc_out) {
+                // raw int32 sums (parity hook): a lane owns a row, 32 columns of it at a time
+                const int m = m0 + lg * 32 + lane;
+                for (int c0 = c_begin; c0 < c_begin + c_count; c0 += 32) {
+                    if (n0 + c0 >= p.N) break;  // uniform across the warp
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc + c0, r);
+                    tmem_ld_wait();
+                    if (m < p.M) {
+                        int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (n0 + c0 + j < p.N) {
+                                int32_t v = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
+                                if (p.act_zero) v += zshift * __ldg(p.w_code_sums + n0 + c0 + j);
+                                dst[j] = v;
+                            }
+                        }
+                    }
+                }
+            }
+            if (p.Y && c_count > 0)
+                store_rows32_dispatch<W4>(acc + c_begin, 0, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
+                                          m0 + lg * 32, n0 + c_begin, lane);
+            // the accumulator may be overwritten once every epilogue warp of both CTAs has read it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(lead_acc_empty + 8 * buf);
+        }
+        if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
+    } else if (W4 && warp >= 6 && warp < L::HELPER0) {
+        // ------------------------------------------------------------ int4 -> int8 (x16) expansion, own half
+        // Four groups of two warps; group g takes the k-blocks g, g + 4, ... of the CTA's sequence and owns slot g
+        // of the packed ring and of the int8 ring.  Nibble -> high half of the byte (= 16 q): two ANDs and a
+        // shift per 8 codes; the factor 16 leaves in the epilogue by an exact shift.
+        const int group = (warp - 6) >> 1;
+        const int gt = tid - 192 - group * 64;  // 0..63 within the group
+        const int total_kb = my_tiles * nkb;
+        const int runs = bh * 4;  // 16-byte packed runs of this CTA's half tile
+        constexpr uint32_t PS = L::PS > 0 ? L::PS : 1;
+        const uint32_t lead_ready = lead_bar0 + 8 * (L::READY_B + group);
+        uint8_t* b_stage = sB + group * L::B_BYTES;
+        static_assert(!W4 || L::ES == 4, "one int8 slot per expansion group");
+        uint32_t n = 0;  // turns taken
+        for (int it = group; it < total_kb; it += 4, ++n) {
+            const uint32_t sp = static_cast<uint32_t>(it) % PS, rp = static_cast<uint32_t>(it) / PS;
+            const uint8_t* stg = sP + sp * L::P_BYTES;
+            bool ok = mbar_wait(bar0 + 8 * (L::FULL_P + sp), rp & 1, s_abort);
+            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * (L::EMPTY_B + group), (n & 1) ^ 1, s_abort);
+            if (!__all_sync(0xffffffffu, ok)) break;  // the warp leaves together
+            // all loads first: the compiler cannot move a load above a store to the other ring by itself
+            uint4 wv[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const int task = gt + t * 64;
+                wv[t] = task < runs ? *reinterpret_cast<const uint4*>(stg + task * 16) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const int task = gt + t * 64;
+                if (task < runs) {
+                    const int r = task >> 2, j = task & 3;
+                    const uint4 w = wv[t];
+                    uint4 c0, c1;
+                    c0.x = (w.x << 4) & 0xF0F0F0F0u;
+                    c0.y = w.x & 0xF0F0F0F0u;
+                    c0.z = (w.y << 4) & 0xF0F0F0F0u;
+                    c0.w = w.y & 0xF0F0F0F0u;
+                    c1.x = (w.z << 4) & 0xF0F0F0F0u;
+                    c1.y = w.z & 0xF0F0F0F0u;
+                    c1.z = (w.w << 4) & 0xF0F0F0F0u;
+                    c1.w = w.w & 0xF0F0F0F0u;
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j)) = c0;
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, 2 * j + 1)) = c1;
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster(lead_ready);
+                mbar_arrive(bar0 + 8 * (L::EMPTY_P + sp));
+            }
+        }
+    }
+
+    if (*s_abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (tid == 0 && p.status) atomicExch(p.status, MIXDQ_ERR_TIMEOUT);
+    }
+    // neither CTA leaves (or frees tensor memory) while its peer may still read its shared memory, signal its
+    // barriers or run instructions that write its tensor memory
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, 2 * ACC_COLS);
+}
+
+template <bool W4>
+int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+                  int num_sms, cudaStream_t stream)
+{
+    using L = PairSmem<W4>;
+    auto kernel = pair_gemm_kernel<W4>;
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
+    PairArgs g;
+    g.bn = bn;
+    g.n_tiles = static_cast<int>(ceil_div(tp.N, bn));
+    g.total_tiles = g.n_tiles * static_cast<int>(ceil_div(tp.M, 2 * BM));
+    const int pairs = g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2;
+    // (the cluster shape is part of the kernel: __cluster_dims__)
+    return launch_pdl(kernel, dim3(static_cast<unsigned>(2 * pairs)), dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, ty, tp,
+                      g);
+}
+
+}  // namespace
+
+int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
+                int num_sms, cudaStream_t stream)
+{
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2) return MIXDQ_ERR_INVALID_ARG;
+    return w4 ? launch_pair_t<true>(ta, tw, ty, tp, bn, num_sms, stream)
+              : launch_pair_t<false>(ta, tw, ty, tp, bn, num_sms, stream);
+}
+
+}  // namespace i8
+}  // namespace mixdq

@@ -9,16 +9,18 @@
 //      the A tile of filter tap (kh, kw) is a 4-D box of the int8 NHWC image shifted by
 //      (kh - 1, kw - 1), and the zero padding is TMA's out-of-bounds fill.
 // Output tile 128 x BN (BN = 128 or 256), 128-wide k-blocks, accumulators in tensor memory.
+#include <algorithm>
+#include <cmath>
+
 #include "common.cuh"
 #include "engines.h"
+#include "i8_tiles.cuh"
 
 namespace mixdq {
 namespace i8 {
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int BK = 128;
 constexpr float kMagic = 12582912.f;  // 1.5 * 2^23: fma(x, inv, magic) rounds x * inv to nearest even
 
 // Four codes as bytes.  Symmetric: clamp(rne(x * inv), -127, 127).  Asymmetric (zoff = zero - 128):
@@ -161,250 +163,6 @@ __device__ __forceinline__ int4 ld_cluster_v4(uint32_t addr, int cta_rank)
     return v;
 }
 
-struct TmaParams {
-    int M, N, k_blocks;
-    int conv;     // 0: A is a [M, K] int8 matrix; 1: A is an int8 NHWC image gathered per filter tap
-    int pad;      // conv: 1 when the int8 image carries its one-pixel border (asymmetric activations)
-    int cblocks;  // conv: k-blocks per filter tap = ceil(Cin / 128)
-    int Cin, HoWo, Wo;
-    int stride;   // conv: input pixels per output pixel along H and W (1 or 2)
-    int bos;      // output row m maps to row (m / 76) * 77 + m % 76 + 1 of Y
-    int batch;
-    const float* act_scale;
-    const int32_t* act_zero;     // asymmetric activations: zero-point (the int8 operand holds q - 128) ...
-    const int32_t* w_code_sums;  // ... and sum_k qw[n, k], so that sum_k (q - z) qw = acc + (128 - z) * sums[n]
-    const float* w_scale;
-    const __half* bias;
-    const __half* bos_out;
-    __half* Y;
-    long long ldy;
-    int32_t* acc_out;
-    int32_t* status;
-    // second branch of a shortcut-split layer: the first branch's int32 sums [M, N] and its activation scale;
-    // the epilogue adds addend * (*addend_scale) * w_scale[n] to every output (ADD instances of the kernels)
-    const int32_t* addend;
-    const float* addend_scale;
-    int small_acc;  // every |accumulator| (W4: after the >> 4) stays below 2^22
-    int tma_store;  // Y is written through its tensor map (row-contiguous output, 16-byte aligned rows)
-};
-
-// Staging tile of one epilogue warp, 32 rows x 64 fp16: dense 128-byte rows with the 128-byte swizzle
-// when a TMA store takes it from there, else rows 144 bytes apart (conflict-free both ways) for the
-// warp's own coalesced stores.  Tiles are 1024-byte aligned (the swizzle pattern follows the address).
-constexpr int EPI_ROW = 144;
-constexpr int EPI_WARP_BYTES = 5120;
-static_assert(32 * EPI_ROW <= EPI_WARP_BYTES && EPI_WARP_BYTES % 1024 == 0, "staging tile");
-
-// int32 accumulator -> float.  W4 accumulators carry the factor 16 of the nibble placement, removed
-// here by an exact shift.  SMALL: |v| < 2^22, so adding v to the bit pattern of 1.5 * 2^23 and
-// subtracting that constant is exact -- two full-rate instructions instead of a quarter-rate convert.
-template <bool W4, bool SMALL>
-__device__ __forceinline__ float acc_to_float(uint32_t r)
-{
-    const int32_t v = W4 ? (static_cast<int32_t>(r) >> 4) : static_cast<int32_t>(r);
-    if (SMALL) return __int_as_float(0x4B400000 + v) - 12582912.f;
-    return static_cast<float>(v);
-}
-
-// One warp's share of an output tile: 32 accumulator rows (one per lane, tensor-memory lanes of
-// `acc`) x `ncols` columns.  64 columns at a time: dequantize in registers, pass through the warp's
-// staging tile, and store with eight lanes along each row so that every store instruction writes
-// whole 128-byte lines.  comb / bias: per-column factors of the tile in shared memory.  acc2_off != 0:
-// a second accumulator that many columns further on holds the other half of the sum.
-template <bool W4, bool SMALL, bool TMA>
-__device__ __forceinline__ void store_rows_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
-                                                     const float* bias, uint8_t* stage, const TmaParams& p,
-                                                     const CUtensorMap* tmap_y, int m_first, int n0, int lane)
-{
-    const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
-    if (TMA && m_first >= p.M) return;  // uniform across the warp
-    for (int c0 = 0; c0 < ncols; c0 += 64) {
-        if (n0 + c0 >= p.N) break;  // uniform across the warp
-        if (TMA) {
-            // the previous bulk store must have read the staging tile before it is overwritten
-            if (lane == 0) tma_store_wait_read();
-            __syncwarp();
-        }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            uint32_t r[32];
-            tmem_ld_32x32(acc + c0 + 32 * h, r);
-            if (acc2_off) {
-                uint32_t r2[32];
-                tmem_ld_32x32(acc + acc2_off + c0 + 32 * h, r2);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] += r2[j];
-            } else {
-                tmem_ld_wait();
-            }
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-                const int c = c0 + 32 * h + j;
-                const float4 ca = *reinterpret_cast<const float4*>(comb + c);
-                const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
-                const float4 ba = *reinterpret_cast<const float4*>(bias + c);
-                const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
-                __half2 hv[4];
-                hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j]), ca.x, ba.x),
-                                          fmaf(acc_to_float<W4, SMALL>(r[j + 1]), ca.y, ba.y));
-                hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 2]), ca.z, ba.z),
-                                          fmaf(acc_to_float<W4, SMALL>(r[j + 3]), ca.w, ba.w));
-                hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 4]), cb.x, bb.x),
-                                          fmaf(acc_to_float<W4, SMALL>(r[j + 5]), cb.y, bb.y));
-                hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 6]), cb.z, bb.z),
-                                          fmaf(acc_to_float<W4, SMALL>(r[j + 7]), cb.w, bb.w));
-                const int chunk = (32 * h + j) >> 3;  // 16-byte chunk of the row
-                uint8_t* dst = TMA ? stage + lane * 128 + ((chunk ^ (lane & 7)) << 4) : stage + lane * EPI_ROW + chunk * 16;
-                *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(hv);
-            }
-        }
-        if (TMA) {
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                tma_store_2d(tmap_y, smem_u32(stage), n0 + c0, m_first);
-                tma_store_commit();
-            }
-            continue;
-        }
-        __syncwarp();
-#pragma unroll
-        for (int it8 = 0; it8 < 8; ++it8) {
-            const int rl = it8 * 4 + (lane >> 3), seg = lane & 7;
-            const int mm = m_first + rl;
-            const int n = n0 + c0 + seg * 8;
-            if (mm >= p.M || n >= p.N) continue;
-            long long orow = mm;
-            if (p.bos) {
-                const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
-                orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
-                       (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
-            }
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI_ROW + seg * 16);
-            __half* dst = p.Y + orow * p.ldy + n;
-            if (vec && n + 8 <= p.N) {
-                *reinterpret_cast<uint4*>(dst) = v;
-            } else {
-                const __half* hs = reinterpret_cast<const __half*>(&v);
-                for (int q = 0; q < 8; ++q)
-                    if (n + q < p.N) dst[q] = hs[q];
-            }
-        }
-        __syncwarp();
-    }
-}
-
-// Picks the instantiation for the launch's accumulator range and store route (both uniform).
-template <bool W4>
-__device__ __forceinline__ void store_rows_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
-                                                    const float* bias, uint8_t* stage, const TmaParams& p,
-                                                    const CUtensorMap* tmap_y, int m_first, int n0, int lane)
-{
-    if (p.tma_store) {
-        if (p.small_acc)
-            store_rows_from_tmem<W4, true, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-        else
-            store_rows_from_tmem<W4, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-    } else {
-        if (p.small_acc)
-            store_rows_from_tmem<W4, true, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-        else
-            store_rows_from_tmem<W4, false, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-    }
-}
-
-// The same in passes of 32 columns, for the persistent kernel, whose eight epilogue warps have to fit
-// their staging tiles beside a full pipeline: 32 rows x 32 fp16, as dense 64-byte rows with the
-// 64-byte swizzle when a TMA store (box 32 x 32) takes the tile, else rows 80 bytes apart.
-constexpr int EPI32_ROW = 80;
-constexpr int EPI32_TILE = 32 * EPI32_ROW;  // 2560: a multiple of 512, the period of the 64-byte swizzle
-
-template <bool W4, bool SMALL, bool TMA>
-__device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
-                                                       const float* bias, uint8_t* stage, const TmaParams& p,
-                                                       const CUtensorMap* tmap_y, int m_first, int n0, int lane)
-{
-    const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
-    if (TMA && m_first >= p.M) return;  // uniform across the warp
-    for (int c0 = 0; c0 < ncols; c0 += 32) {
-        if (n0 + c0 >= p.N) break;  // uniform across the warp
-        uint32_t r[32];
-        tmem_ld_32x32(acc + c0, r);
-        if (acc2_off) {
-            uint32_t r2[32];
-            tmem_ld_32x32(acc + acc2_off + c0, r2);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] += r2[j];
-        } else {
-            tmem_ld_wait();
-        }
-        uint4 out[4];  // this lane's row of the pass as fp16
-#pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-            const int c = c0 + j;
-            const float4 ca = *reinterpret_cast<const float4*>(comb + c);
-            const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
-            const float4 ba = *reinterpret_cast<const float4*>(bias + c);
-            const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
-            __half2 hv[4];
-            hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j]), ca.x, ba.x),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 1]), ca.y, ba.y));
-            hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 2]), ca.z, ba.z),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 3]), ca.w, ba.w));
-            hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 4]), cb.x, bb.x),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 5]), cb.y, bb.y));
-            hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 6]), cb.z, bb.z),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 7]), cb.w, bb.w));
-            out[j >> 3] = *reinterpret_cast<const uint4*>(hv);
-        }
-        if (TMA) {
-            // the previous bulk store must have read the staging tile; the conversion above hid that wait
-            if (lane == 0) tma_store_wait_read();
-            __syncwarp();
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint8_t* dst = TMA ? stage + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4) : stage + lane * EPI32_ROW + q * 16;
-            *reinterpret_cast<uint4*>(dst) = out[q];
-        }
-        if (TMA) {
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                tma_store_2d(tmap_y, smem_u32(stage), n0 + c0, m_first);
-                tma_store_commit();
-            }
-            continue;
-        }
-        __syncwarp();
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int rl = it * 8 + (lane >> 2), seg = lane & 3;
-            const int mm = m_first + rl;
-            const int n = n0 + c0 + seg * 8;
-            if (mm >= p.M || n >= p.N) continue;
-            long long orow = mm;
-            if (p.bos) {
-                const int prompt = mm / (MIXDQ_TOKENS_PER_PROMPT - 1);
-                orow = static_cast<long long>(prompt) * MIXDQ_TOKENS_PER_PROMPT +
-                       (mm - prompt * (MIXDQ_TOKENS_PER_PROMPT - 1) + 1);
-            }
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + rl * EPI32_ROW + seg * 16);
-            __half* dst = p.Y + orow * p.ldy + n;
-            if (vec && n + 8 <= p.N) {
-                *reinterpret_cast<uint4*>(dst) = v;
-            } else {
-                const __half* hs = reinterpret_cast<const __half*>(&v);
-                for (int q = 0; q < 8; ++q)
-                    if (n + q < p.N) dst[q] = hs[q];
-            }
-        }
-        __syncwarp();
-    }
-}
-
 // The 32-column passes for the second branch of a shortcut-split layer: y = acc * comb[c] + addend * ratio *
 // comb[c] + bias[c], where comb[c] = s_hi * s_w and ratio = s_lo / s_hi.  The first branch's sums come in through
 // the warp's staging tile, 16 columns at a time with four lanes along each row (coalesced), and the fp16 results
@@ -513,32 +271,19 @@ __device__ __forceinline__ void store_rows32_add_from_tmem(uint32_t acc, uint32_
     }
 }
 
-template <bool W4>
-__device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
-                                                      const float* bias, uint8_t* stage, const TmaParams& p,
-                                                      const CUtensorMap* tmap_y, int m_first, int n0, int lane)
-{
-    if (p.tma_store) {
-        if (p.small_acc)
-            store_rows32_from_tmem<W4, true, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-        else
-            store_rows32_from_tmem<W4, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-    } else {
-        if (p.small_acc)
-            store_rows32_from_tmem<W4, true, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-        else
-            store_rows32_from_tmem<W4, false, false>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
-    }
-}
-
-// Rings of the pipeline and their barriers.  W8: activation and weight tiles move in lockstep, STAGES
-// deep.  W4 (128-wide tiles only): the packed int4 rows have a ring of their own, deep enough to hide
-// the TMA round trip, and are expanded into a short ring of int8 weight tiles; the chain TMA ->
-// expansion -> MMA is longer than the activations' TMA -> MMA, and it is depth, not bandwidth, that
-// bounds it (measured: 4 instead of 6 common stages cost 20 % on long reductions).
+// Rings of the pipeline and their barriers.  What bounds the k-block cadence of these kernels is neither the
+// issue rate nor the tensor pipe but the bytes a CTA keeps in flight: a slot is away for about 1900 cycles
+// (TMA request, L2 round trip, MMAs, commit, the producer noticing), so a ring of D tiles delivers one tile
+// every 1900 / D cycles (measured with clock stamps: 6 stages of both operands -> 330 cycles per k-block,
+// 4 activation stages -> 460), against 256 cycles of MMA work per 128 x 128 x 128 k-block.  Shared memory
+// is the resource: everything not needed elsewhere goes into tiles that are in flight.
+// W8: activation and weight tiles move in lockstep, STAGES deep.  W4 (128-wide tiles only): the packed int4
+// rows have a ring of their own and are expanded into a short ring of int8 weight tiles, one slot per
+// expansion group -- staging, not data in flight, so it is kept as small as the four groups allow.
 template <int BN, int STAGES, bool W4, bool PERSIST>
 struct Rings {
     static_assert(!W4 || BN == 128, "W4 runs on 128-wide tiles");
+    static constexpr bool kW4 = W4;
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
     static constexpr int P_BYTES = BN * (BK / 2);
@@ -549,8 +294,8 @@ struct Rings {
     // barrier of the slot can then never be a whole pair of phases behind what the group's parity wait
     // assumes.  (All rings of the W8 kernels are even for the same reason: an issuer must meet every
     // phase of the barriers it waits on.)
-    static constexpr int AS = W4 ? 4 : STAGES;                  // activation tiles
-    static constexpr int ES = W4 ? 6 : STAGES;                  // int8 weight tiles (W4: expanded; four in the making)
+    static constexpr int AS = W4 ? 6 : STAGES;                  // activation tiles
+    static constexpr int ES = W4 ? 4 : STAGES;                  // int8 weight tiles (W4: expanded, one per expansion group)
     static_assert(AS % 2 == 0 && ES % 2 == 0, "slots must keep their MMA issuer");
     static constexpr int PS = W4 ? (PERSIST ? 4 : 6) : 0;       // packed int4 weight tiles
     static constexpr int OFF_A = 0;
@@ -729,25 +474,42 @@ __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int 
 }
 
 // The k-blocks first, first + step, ... of one output tile: wait for the tiles, issue the four MMAs
-// into `acc`, hand the slots back.  Runs in a single thread.  seq0 as above.
+// into `acc`, hand the slots back.  Runs in a single thread; ring slots, phase parities and descriptors
+// are carried along instead of recomputed.  seq0 as above; step <= 2.
 template <int BN, bool W4, class L>
 __device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t seq0, uint32_t a0,
                                                uint32_t b0, uint32_t bar0, volatile int* s_abort)
 {
     constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
+    static_assert(L::AS >= 2 && L::ES >= 2, "a step of two must stay inside one lap of a ring");
+    if (first >= nkb) return true;
+    const uint32_t q0 = seq0 + static_cast<uint32_t>(first);
+    uint32_t sa = q0 % L::AS, pa = (q0 / L::AS) & 1, se = q0 % L::ES, pe = (q0 / L::ES) & 1;
+    const uint64_t a_desc0 = smem_desc_sw128(a0), b_desc0 = smem_desc_sw128(b0);
+    uint32_t accumulate = 0;
     for (int i = first; i < nkb; i += step) {
-        const uint32_t q = seq0 + i;
-        const uint32_t sa = q % L::AS, ra = q / L::AS, se = q % L::ES, re = q / L::ES;
-        if (!mbar_wait(bar0 + 8 * (L::FULL_A + sa), ra & 1, s_abort)) return false;
-        if (!mbar_wait(bar0 + 8 * (L::READY_B + se), re & 1, s_abort)) return false;
+        if (!mbar_wait(bar0 + 8 * (L::FULL_A + sa), pa, s_abort)) return false;
+        if (!mbar_wait(bar0 + 8 * (L::READY_B + se), pe, s_abort)) return false;
         tc_fence_after_sync();
-        const uint64_t a_desc = smem_desc_sw128(a0 + sa * L::A_BYTES);
-        const uint64_t b_desc = smem_desc_sw128(b0 + se * L::B_BYTES);
+        // (the start-address field counts 16-byte units and every tile lies below 256 KB: no carry out of it)
+        const uint64_t a_desc = a_desc0 + sa * (L::A_BYTES >> 4);
+        const uint64_t b_desc = b_desc0 + se * (L::B_BYTES >> 4);
+        mma_i8_ss(acc, a_desc, b_desc, idesc, accumulate);
 #pragma unroll
-        for (int k = 0; k < BK / 32; ++k)
-            mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, (i != first) || k != 0);
+        for (int k = 1; k < BK / 32; ++k) mma_i8_ss(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
+        accumulate = 1;
         tc_commit(bar0 + 8 * (L::EMPTY_A + sa));
         if (W4) tc_commit(bar0 + 8 * (L::EMPTY_B + se));
+        sa += step;
+        if (sa >= static_cast<uint32_t>(L::AS)) {
+            sa -= L::AS;
+            pa ^= 1;
+        }
+        se += step;
+        if (se >= static_cast<uint32_t>(L::ES)) {
+            se -= L::ES;
+            pe ^= 1;
+        }
     }
     return true;
 }
@@ -762,8 +524,10 @@ struct TmaSmem : Rings<BN, STAGES, W4, false> {
     static constexpr int OFF_MISC = OFF_BIAS + BN * 4;
     static constexpr int TOTAL = OFF_MISC + 64 + 1024;
     static_assert(TOTAL <= 232448, "shared memory of one CTA");
-    // warps: 0 activation producer, 1 MMA issuer, 2-5 epilogue, 6-9 epilogue helpers (the other half
-    // of the tile's columns), W4: 6-13 nibble expansion during the main loop
+    // warps: 0 activation producer, 1 MMA issuer, 2-5 per-column factors during the main loop, W4: 6-13
+    // nibble expansion; then the weight producer and the second issuer.  An unsplit tile is dequantized and
+    // stored by all sixteen warps (EPI_WARPS), each taking 32 rows x BN / 4 columns; a split tile is moved
+    // to shared memory by warps 2-9.
     static constexpr int WORK_THREADS = W4 ? 448 : 320;
     static constexpr int B_WARP = WORK_THREADS / 32;      // TMA producer of the weight tiles
     // One thread issues a 128-wide MMA about every 68 cycles, the tensor core retires it in 64: a
@@ -772,7 +536,10 @@ struct TmaSmem : Rings<BN, STAGES, W4, false> {
     // into another, and the epilogue adds the two (integer adds: exact).
     static constexpr bool DUAL = BN == 128;
     static constexpr int MMA2_WARP = B_WARP + 1;
-    static constexpr int THREADS = WORK_THREADS + 32 + (DUAL ? 32 : 0);
+    static constexpr int EPI_WARPS = 16;
+    static constexpr int THREADS = EPI_WARPS * 32;
+    static_assert(WORK_THREADS + 32 + (DUAL ? 32 : 0) <= THREADS, "role warps");
+    static_assert(EPI_WARPS * EPI32_TILE <= R::RINGS_END, "staging tiles lie in the drained pipeline buffers");
     static constexpr int TMEM_COLS = DUAL ? 2 * BN : BN;
 };
 
@@ -880,10 +647,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
             expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, nkb, sB, sP, bar0, s_abort);
         }
-        if (warp < 10) {
-            // -------------------------------------------------------- epilogue, part 1
-            // warps 2-5 take the first half of the tile's columns, warps 6-9 the second half; both
-            // read the 32 tensor-memory lanes their rank within a warpgroup gives access to
+        if (warp < 10 && !direct) {
+            // -------------------------------------------------------- epilogue of a split tile, part 1
+            // (or accumulator dump): warps 2-5 take the first half of the tile's columns, warps 6-9 the second
+            // half; both read the 32 tensor-memory lanes their rank within a warpgroup gives access to
             asm volatile("bar.sync 1, 256;" ::: "memory");  // the factor tables above are complete
             bool ok = mbar_wait(bar_accum, 0, s_abort);
             tc_fence_after_sync();
@@ -892,16 +659,8 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             const int row = lg * 32 + lane;
             const int cbeg = warp < 6 ? 0 : BN / 2;
             const uint32_t acc = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + cbeg;
-            if (go && direct) {
-                // unsplit tile: dequantize and store straight from tensor memory; the staging tiles
-                // sit in the pipeline buffers, which are free once the last MMA has completed
-                uint8_t* stage = smem + (warp - 2) * EPI_WARP_BYTES;
-                store_rows_dispatch<W4>(acc, dual ? BN : 0, BN / 2, s_comb + cbeg, s_bias + cbeg, stage, p, &tmap_y,
-                                        m0 + lg * 32, n0 + cbeg, lane);
-                if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
-            } else if (go) {
-                // split tile (or accumulator dump): tensor memory -> registers -> shared memory,
-                // 16-byte chunks XOR-swizzled by row
+            if (go) {
+                // tensor memory -> registers -> shared memory, 16-byte chunks XOR-swizzled by row
                 uint8_t* prow = smem + row * (BN * 4);
                 for (int c0 = 0; c0 < BN / 2; c0 += 32) {
                     uint32_t r[32];
@@ -933,7 +692,28 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
     }
 
-    // ---------------------------------------------------------------- epilogue, part 2
+    if (direct) {
+        // ------------------------------------------------------------ epilogue of an unsplit tile
+        // Every warp of the CTA, its main-loop role over, takes 32 rows (the tensor-memory lanes its rank
+        // within a warpgroup gives access to) x BN / 4 columns: dequantize in registers, pass through a
+        // staging tile in the drained pipeline buffers, store (TMA box 32 x 32, or coalesced).  With eight
+        // warps the conversion, some six instructions per element, was issue-bound at about 2000 cycles.
+        asm volatile("bar.sync 1, %0;" ::"n"(L::THREADS) : "memory");  // the factor tables are complete
+        bool ok = mbar_wait(bar_accum, 0, s_abort);
+        tc_fence_after_sync();
+        if (__all_sync(0xffffffffu, ok && !*s_abort)) {
+            constexpr int COLS = BN / (L::EPI_WARPS / 4);
+            const int lg = warp & 3;
+            const int cbeg = (warp >> 2) * COLS;
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + cbeg;
+            uint8_t* stage = smem + warp * EPI32_TILE;
+            store_rows32_dispatch<W4>(acc, dual ? BN : 0, COLS, s_comb + cbeg, s_bias + cbeg, stage, p, &tmap_y,
+                                      m0 + lg * 32, n0 + cbeg, lane);
+            if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
+        }
+    }
+
+    // ---------------------------------------------------------------- epilogue of a split tile, part 2
     // Every CTA of the cluster holds partial sums of the same tile in its shared memory.  CTA
     // `rank` adds up rows [rank * 128 / splits, ...) over all of them (integer adds: exact,
     // order-free), dequantizes and stores; threads run along a row so stores coalesce.
@@ -1341,6 +1121,48 @@ int pick_splits(int64_t tiles, int k_blocks, int num_sms)
 
 }  // namespace
 
+// Which kernel form runs an int8 GEMM of M x N over k_blocks k-blocks: 0 = the single-CTA kernels of this file,
+// otherwise the tile width of the pair form.  Both are estimated in SM cycles from a model whose constants were
+// fitted to timings of every layer shape of the SDXL-turbo-shaped UNet at image batch 1 and 4 on a B200 (each
+// form at each width): rounds of tiles over the SMs (or SM pairs) times the cost of a tile -- the larger of its
+// main loop, a per-k-block cost that grows with the tile width, and its epilogue -- plus fixed costs.
+int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms)
+{
+    if (M < 2 * BM || num_sms < 2) return 0;
+    const double nkb = k_blocks;
+    // pair form: 256 x bn tiles, widths below 160 never paid off
+    double best = 0;
+    int best_bn = 0;
+    for (int bn = 160; bn <= 256; bn += 32) {
+        const double tiles = static_cast<double>(ceil_div(M, 2 * BM) * ceil_div(N, bn));
+        const double rounds = std::ceil(tiles / (num_sms / 2));
+        const double per_kb = w4 ? 350.0 + 1.4 * bn : 250.0 + 1.2 * bn;
+        const double t = rounds * (std::max(nkb * per_kb, 30.0 * bn) + 800.0) + 16.0 * bn + 5000.0;
+        if (best_bn == 0 || t < best) {
+            best = t;
+            best_bn = bn;
+        }
+    }
+    // single-CTA kernels: 128 x 128 tiles (128 x 256 for wide int8 layers), persistent once the tiles cover the
+    // SMs, else one tile per CTA with the reduction split over a cluster
+    double old;
+    const double c = w4 ? 580.0 : 420.0;
+    const bool wide = !w4 && (N >= 1024 || N % 256 == 0) && ceil_div(M, BM) * ceil_div(N, 256) >= 100;
+    if (wide) {
+        const double tiles = static_cast<double>(ceil_div(M, BM) * ceil_div(N, 256));
+        old = std::ceil(tiles / num_sms) * std::max(nkb * 620.0, 10000.0) + 3000.0;
+    } else {
+        const int64_t tiles = ceil_div(M, BM) * ceil_div(N, 128);
+        if (tiles >= num_sms) {
+            old = std::ceil(static_cast<double>(tiles) / num_sms) * std::max(nkb * c, 5000.0) + 3000.0;
+        } else {
+            const int s = pick_splits(tiles, k_blocks, num_sms);
+            old = std::ceil(nkb / s) * c + 3000.0 + 3000.0 + (s > 1 ? 2500.0 : 0.0);
+        }
+    }
+    return best < 1.05 * old ? best_bn : 0;
+}
+
 size_t tma_scratch_bytes(int64_t in_rows, int64_t K_row) { return static_cast<size_t>(round_up(in_rows * K_row, 256)); }
 
 // Box of 128 consecutive output pixels as (Wb, Hb, Bb) in image coordinates; false when the
@@ -1459,6 +1281,23 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
         tp.k_blocks = static_cast<int>(ceil_div(p.K, BK));
     }
     if (rc != MIXDQ_OK) return rc;
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
+    // the pair form (two-CTA tiles of 256 x bn, i8_pair.cu) where its estimate beats the single-CTA kernels
+    const int pair_bn = (!p.addend && amode != A_BOS) ? plan_pair_tile(p.M, p.N, tp.k_blocks, w4, num_sms) : 0;
+    if (pair_bn > 0) {
+        if (w4)
+            rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, pair_bn / 2, false);
+        else
+            rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(p.K), p.N, pitch, BK, pair_bn / 2, true);
+        if (rc != MIXDQ_OK) return rc;
+        if (tp.tma_store) {
+            rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
+                                    static_cast<uint64_t>(p.ldy), 32, 32, true);
+            if (rc != MIXDQ_OK) return rc;
+        }
+        return launch_pair(ta, tw, ty, tp, w4, pair_bn, num_sms, stream);
+    }
     // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
     // (W4 runs on 128-wide tiles only: its packed ring needs the room, and it measured no slower)
     const bool wide = !w4 && !p.addend && (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
@@ -1470,14 +1309,11 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     if (rc != MIXDQ_OK) return rc;
 
     const int64_t tiles = ceil_div(p.M, BM) * ceil_div(p.N, bn);
-    const int num_sms = sm_count();
-    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
     const bool persistent = tiles >= num_sms;
     if (tp.tma_store) {
-        // store box: 64 x 32 (128-byte swizzle) in the one-tile kernel, 32 x 32 (64-byte swizzle) in the
-        // persistent one, whose staging tiles are smaller
+        // store box: 32 columns x 32 rows (64-byte rows with the 64-byte swizzle), one per epilogue pass
         rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
-                                static_cast<uint64_t>(p.ldy), persistent ? 32 : 64, 32, persistent);
+                                static_cast<uint64_t>(p.ldy), 32, 32, true);
         if (rc != MIXDQ_OK) return rc;
     }
     if (p.addend) {  // second branch of a shortcut-split layer: the instances with the two-scale epilogue

@@ -1,0 +1,129 @@
+"""GPU parity of the two-CTA (tcgen05 cta_group::2) form of the W8A8 / W4A8 engine, which the planner
+chooses for the large layers: 256-row tiles of 160 to 256 columns, two MMA-issuing threads adding into one
+accumulator, each CTA loading its own activation rows and half of the weight tile.  Every case first
+checks that the planner really sends the shape to that form; int32 accumulators must match the oracle bit
+for bit (whole tensor), fp16 outputs within the path's tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mixdq_oracle as orc
+from paper_2405_17873_b200 import mixdq, synth
+from helpers import assert_close, dev, device_weights, host, oracle_weights, status_word, workspace_for
+
+pytestmark = pytest.mark.gpu
+
+
+def _kblocks(K):
+    return (K + 127) // 128
+
+
+# ragged rows / columns / reduction lengths, one and several tiles per CTA pair, all tile widths
+LINEAR_SHAPES = [(5567, 776, 784), (3274, 776, 432), (4458, 648, 1952), (6812, 328, 1936), (5968, 1304, 448),
+                 (4096, 640, 640), (1024, 10240, 1280), (16384, 320, 640)]
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,N,K", LINEAR_SHAPES)
+def test_linear_on_pair_tiles(bits, M, N, K):
+    rows, cols = mixdq.int8_tile_plan(M, N, _kblocks(K), bits)
+    assert rows == 256 and cols in (160, 192, 224, 256), (rows, cols)
+    X = synth.normal_f16((M, K), 1.0, seed=M + K)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 1)
+    b = synth.normal_f16((N,), 0.01, seed=N)
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.linear_a8(X, codes, s_ref, sx_ref, b)
+    Xd = dev(X)
+    s, _, packed = device_weights(W, bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    ws = workspace_for(M, N, K, bits)
+    acc = mixdq.linear_acc_i32(Xd, packed, N, bits, sx, workspace=ws, status=st)
+    y = mixdq.linear(Xd, packed, N, bits, s, None, 8, sx, dev(b), workspace=ws, status=st)
+    # the same layer on stored int8 activations: the same bits
+    xq = mixdq.quantize_acts(Xd, sx)
+    y_q8 = mixdq.linear_q8(xq, packed, N, bits, s, sx, dev(b), st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+    assert np.array_equal(host(y_q8).view(np.uint16), host(y).view(np.uint16))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,Cin,Cout,stride", [(4, 32, 320, 640, 1), (2, 64, 192, 328, 1), (8, 64, 160, 320, 2),
+                                                 (3, 64, 96, 640, 1)])
+def test_conv3x3_on_pair_tiles(bits, B, H, Cin, Cout, stride):
+    Ho = (H - 1) // stride + 1
+    rows, cols = mixdq.int8_tile_plan(B * Ho * Ho, Cout, 9 * _kblocks(Cin), bits)
+    assert rows == 256, (rows, cols)
+    X = synth.normal_f16((B, H, H, Cin), 1.0, seed=31 + Cin)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=32 + Cout)
+    b = synth.normal_f16((Cout,), 0.01, seed=33)
+    s_ref, _, codes = oracle_weights(Wt.reshape(Cout, -1), bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.conv3x3_a8(X, codes.reshape(Cout, 3, 3, Cin), s_ref, sx_ref, b, stride)
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt.reshape(Cout, -1), bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, H, Cin, Cout, stride, bits, 8))
+    acc = mixdq.conv3x3_acc_i32(Xd, packed, Cout, bits, sx, stride, ws, st)
+    y = mixdq.conv3x3(Xd, packed, Cout, bits, s, None, 8, sx, dev(b), stride, ws, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_asymmetric_activations_on_pair_tiles(bits):
+    """Asymmetric 8-bit activations (Sec. 4.1) through the same kernels: the zero-point term rides in the
+    per-column bias of the epilogue, the padded int8 image feeds the convolution."""
+    M, N, K = 4096, 640, 1280
+    assert mixdq.int8_tile_plan(M, N, _kblocks(K), bits)[0] == 256
+    X = synth.one_sided_f16((M, K), seed=5, shift=0.3)
+    W = synth.normal_f16((N, K), 0.02, seed=6)
+    b = synth.normal_f16((N,), 0.01, seed=7)
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    sa_ref, z_ref = orc.act_minmax_params(X)
+    acc_ref, y_ref = orc.linear_a8_asym(X, codes, s_ref, sa_ref, z_ref, b)
+    Xd = dev(X)
+    s, _, packed = device_weights(W, bits, True)
+    sums = mixdq.weight_code_sums(packed, N, K, bits)
+    sa, za = mixdq.act_asym_params(Xd)
+    st = status_word()
+    ws = workspace_for(M, N, K, bits)
+    acc = mixdq.linear_a8_asym_acc_i32(Xd, packed, N, bits, sums, sa, za, ws, st)
+    y = mixdq.linear_a8_asym(Xd, packed, N, bits, s, sums, sa, za, dev(b), ws, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert host(sa)[0] == sa_ref and int(host(za)[0]) == z_ref
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+    # 3x3 convolution on the image kept with its border of zero-point codes
+    B, H, Cin, Cout = 4, 32, 320, 640
+    assert mixdq.int8_tile_plan(B * H * H, Cout, 9 * _kblocks(Cin), bits)[0] == 256
+    Xc = synth.one_sided_f16((B, H, H, Cin), seed=8, shift=0.2)
+    Wc = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=9)
+    sc_ref, _, cc = oracle_weights(Wc.reshape(Cout, -1), bits, True)
+    sca_ref, zc_ref = orc.act_minmax_params(Xc)
+    accc_ref, yc_ref = orc.conv3x3_a8_asym(Xc, cc.reshape(Cout, 3, 3, Cin), sc_ref, sca_ref, zc_ref, None, 1)
+    Xcd = dev(Xc)
+    sc, _, pc = device_weights(Wc.reshape(Cout, -1), bits, True)
+    csums = mixdq.weight_code_sums(pc, Cout, 9 * Cin, bits)
+    sca, zca = mixdq.act_asym_params(Xcd)
+    wsc = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, H, Cin, Cout, 1, bits, 8))
+    accc = mixdq.conv3x3_a8_asym_acc_i32(Xcd, pc, Cout, bits, csums, sca, zca, 1, wsc, st)
+    yc = mixdq.conv3x3_a8_asym(Xcd, pc, Cout, bits, sc, csums, sca, zca, None, 1, wsc, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(accc), accc_ref)
+    assert_close(host(yc), yc_ref)
+
+
+def test_planner_keeps_small_layers_on_single_cta_tiles():
+    assert mixdq.int8_tile_plan(1024, 1280, 10, 4) == (128, 128)     # attention projection, image batch 4
+    assert mixdq.int8_tile_plan(256, 1280, 40, 4)[0] == 128          # FFN-2 at image batch 1
+    assert mixdq.int8_tile_plan(100, 64, 2, 8)[0] == 128
