@@ -61,6 +61,9 @@ def parse():
                          "the default run")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the per-configuration records, the weight-bound layers and the two weight-only sweeps "
+                         "that the default run appends to its line")
     return ap.parse_args()
 
 
@@ -324,6 +327,194 @@ def run_fp16_library(args):
                                  " (cuBLAS / cuDNN), fp16 weights distinct per layer"}}))
 
 
+# ----------------------------------------------------------------------------- per-configuration records
+
+NOMINAL = {"int8_tops": 4500.0, "f16_tflops": 2250.0, "hbm_gbs": 8000.0}  # dense peaks of the part, for context
+
+
+def _time_graph(torch, stream, fn, reps=10, rounds=3):
+    """Average microseconds of one call of fn, from a CUDA graph of `reps` back-to-back calls replayed `rounds`
+    times (events on the launching stream; one untimed replay first)."""
+    with torch.cuda.stream(stream):
+        fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                fn()
+        g.replay()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(rounds):
+            g.replay()
+        t1.record()
+        torch.cuda.synchronize()
+    return t0.elapsed_time(t1) * 1e3 / (reps * rounds)
+
+
+def _fracs(rate, measured, nominal, probe=None):
+    d = {"of_measured": round(rate / measured, 4), "of_nominal": round(rate / nominal, 4)}
+    if probe:
+        d["of_int8_mma_probe"] = round(rate / probe, 4)
+    return d
+
+
+def config_records(torch, mixdq, synth, stream, peaks, probe_int8):
+    """One record per stated configuration besides the layer sweep: the single W8A8 linear layer, the weight-only
+    trio at 4096 and 16 tokens, the FFN pair in W4A8 / W8A8 at image batch 1 and 4, the BOS-aware K / V
+    projections at prompt batch 1 and 8.  Quantization pass + GEMM per call; a graph of ten calls on one set of
+    weights (warm L2) unless stated; activation scales computed at set-up."""
+    dev = lambda a: torch.from_numpy(a).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    int8_peak = peaks["bf16_tflops"] * INT8_TO_BF16_NOMINAL
+    out = []
+
+    def a8_linear(tag, X, W, b, bits):
+        M, K = X.shape
+        N = W.shape[0]
+        Xd, Wd = dev(X), dev(W)
+        s, _ = mixdq.weight_minmax_params(Wd, bits, True)
+        pk = mixdq.pack_weights(Wd, bits, s)
+        sx = mixdq.act_scale(Xd)
+        ws = mixdq.new_workspace(mixdq.workspace_bytes(M, N, K, bits, 8))
+        Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        bd = None if b is None else dev(b)
+        us = _time_graph(torch, stream, lambda: mixdq.linear(Xd, pk, N, bits, s, None, 8, sx, bd, ws, status, out=Y))
+        tops = 2.0 * M * N * K / us / 1e6
+        rows, cols = mixdq.int8_tile_plan(M, N, (K + 127) // 128, bits)
+        out.append({"config": tag, "M": M, "N": N, "K": K, "w_bits": bits, "a_bits": 8, "us": round(us, 2),
+                    "tops": round(tops, 1), "bound": "tensor", "l2": "warm", "tile": f"{rows}x{cols}",
+                    "frac": _fracs(tops, int8_peak, NOMINAL["int8_tops"], probe_int8)})
+
+    # 1. single linear layer, W8A8
+    X, W, b = synth.single_linear(seed=0)
+    a8_linear("1: single linear W8A8", X, W, b, 8)
+    # 3. FFN pair (GEGLU projection, then 5120 -> 1280) with 1 % outlier channels, image batch 1 and 4
+    for B in (1, 4):
+        for bits in (4, 8):
+            Xf = synth.ffn_input(B, seed=3000 + B)
+            a8_linear(f"3: FFN-1 1280->10240 B={B}", Xf, synth.normal_f16((10240, 1280), 0.02, 3100), None, bits)
+            Xg = synth.normal_f16((B * 256, 5120), 0.3, 3104)   # the size and rough range of a GEGLU output
+            a8_linear(f"3: FFN-2 5120->1280 B={B}", Xg, synth.normal_f16((1280, 5120), 0.02, 3102), None, bits)
+    # 4. BOS-aware K / V projections, W8A8
+    for B in (1, 8):
+        for N in (640, 1280):
+            E = synth.text_embedding(B)
+            Wk = synth.kv_weight(N, seed=4200 + N)
+            Ed, Wd = dev(E), dev(Wk)
+            s, _ = mixdq.weight_minmax_params(Wd, 8, True)
+            pk = mixdq.pack_weights(Wd, 8, s)
+            sx = mixdq.act_scale(Ed.reshape(-1, E.shape[-1]), 77)
+            bos = synth.bos_projection(Ed[0, 0], Wd)
+            ws = mixdq.new_workspace(mixdq.workspace_bytes(B * 76, N, 2048, 8, 8))
+            Y = torch.empty((B, 77, N), dtype=torch.float16, device="cuda")
+            us = _time_graph(torch, stream, lambda: mixdq.crossattn_kv(Ed, pk, N, 8, s, sx, bos, ws, status, out=Y))
+            tops = 2.0 * B * 76 * N * 2048 / us / 1e6
+            out.append({"config": f"4: BOS-aware K/V 2048->{N} B={B}", "M": B * 76, "N": N, "K": 2048, "w_bits": 8,
+                        "a_bits": 8, "us": round(us, 2), "tops": round(tops, 1), "bound": "latency (a few tiles)",
+                        "l2": "warm", "frac": _fracs(tops, int8_peak, NOMINAL["int8_tops"], probe_int8)})
+    # 2. weight-only trio (W3 / W4 / W8, fp16 activations) at 4096 tokens (tensor-bound) and 16 (weight stream)
+    for M in (4096, 16):
+        for idx in range(3):
+            X, W, b, bits = synth.weight_only_layer(idx, M)
+            N, K = W.shape
+            Xd, Wd = dev(X), dev(W)
+            s, z = mixdq.weight_minmax_params(Wd, bits, False)
+            pk = mixdq.pack_weights(Wd, bits, s, z)
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            bd = dev(b)
+            us = _time_graph(torch, stream, lambda: mixdq.linear(Xd, pk, N, bits, s, z, 16, None, bd, None, status, out=Y))
+            rec = {"config": f"2: weight-only {K}->{N} at {M} tokens", "M": M, "N": N, "K": K, "w_bits": bits,
+                   "a_bits": 16, "us": round(us, 2), "l2": "warm"}
+            if M >= 64:
+                tf = 2.0 * M * N * K / us / 1e6
+                rec.update({"tflops": round(tf, 1), "bound": "tensor",
+                            "frac": _fracs(tf, peaks["bf16_tflops"], NOMINAL["f16_tflops"])})
+            else:
+                gbs = (pk.numel() + 8 * N + 2 * M * (K + N)) / us / 1e3
+                rec.update({"gb_per_s": round(gbs, 1), "bound": "launch latency (under 0.5 MB of weights)",
+                            "frac": _fracs(gbs, peaks["hbm_gbs"], NOMINAL["hbm_gbs"])})
+            out.append(rec)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return out
+
+
+def weight_bound_records(torch, mixdq, synth, stream, peaks):
+    """The weight-only engine where it is bound by the weight stream: the transformer FFN layers on 16 tokens,
+    with as many distinct copies of the packed weights as it takes to exceed L2 several times over, walked
+    inside one graph, so that every launch streams its weights from HBM."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(11)
+    out = []
+    for (K, N, bits) in ((1280, 10240, 8), (1280, 10240, 4), (1280, 10240, 3), (5120, 1280, 4), (1280, 1280, 4)):
+        W = (torch.randn((N, K), generator=g, device="cuda") * 0.02).half()
+        s, z = mixdq.weight_minmax_params(W, bits, False)
+        pk0 = mixdq.pack_weights(W, bits, s, z)
+        copies = max(4, int(512e6 // pk0.numel()) + 1)
+        pks = [pk0.clone() for _ in range(copies)]
+        X = torch.randn((16, K), generator=g, device="cuda").half()
+        Y = torch.empty((16, N), dtype=torch.float16, device="cuda")
+        with torch.cuda.stream(stream):
+            mixdq.linear(X, pks[0], N, bits, s, z, 16, None, None, None, status, out=Y)
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream):
+                for pk in pks:
+                    mixdq.linear(X, pk, N, bits, s, z, 16, None, None, None, status, out=Y)
+            gr.replay()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record()
+            gr.replay()
+            gr.replay()
+            t1.record()
+            torch.cuda.synchronize()
+        us = t0.elapsed_time(t1) * 1e3 / (2 * copies)
+        alg = pk0.numel() + 8 * N + 2 * 16 * (K + N)
+        gbs = alg / us / 1e3
+        out.append({"layer": f"{K}->{N} at 16 tokens", "w_bits": bits, "us": round(us, 2), "gb_per_s": round(gbs, 1),
+                    "algorithmic_bytes": alg, "l2": f"cold: {copies} copies of the weights walked in one graph",
+                    "frac": _fracs(gbs, peaks["hbm_gbs"], NOMINAL["hbm_gbs"])})
+        del pks
+    return out
+
+
+def sub_sweep_record(torch, UNetSweep, stream, peaks, batch, tokens, steps=10):
+    """The 3.66-bit weight-only table over the whole network (tokens = 0: image batch `batch`; tokens > 0: every
+    linear layer on that many rows), one step as a CUDA graph, `steps` timed replays."""
+    sw = UNetSweep(batch, "a16", seed=5, tokens=tokens)
+    with torch.cuda.stream(stream):
+        sw.step()
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=stream):
+            sw.step()
+        for _ in range(3):
+            gr.replay()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(steps):
+            gr.replay()
+        t1.record()
+        torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    rec = {"workload": f"unet_linear_sweep_a16_{tokens}tokens" if tokens else f"unet_sweep_sdxl512_a16_b{batch}",
+           "layers": len(sw.layers), "ms_per_step": round(ms, 3), "steps": steps, "device_status": int(sw.status.item()),
+           "l2": "weights (distinct per layer) are larger than L2"}
+    if tokens:
+        alg = sum(sw.algorithmic_bytes(pl) for pl in sw.layers)
+        gbs = alg / (ms * 1e-3) / 1e9
+        rec.update({"bound": "hbm", "gb_per_s": round(gbs, 1), "algorithmic_bytes_per_step": alg,
+                    "frac": _fracs(gbs, peaks["hbm_gbs"], NOMINAL["hbm_gbs"])})
+    else:
+        tf = sw.total_ops() / (ms * 1e-3) / 1e12
+        rec.update({"bound": "tensor", "tflops": round(tf, 1),
+                    "frac": _fracs(tf, peaks["bf16_tflops_sustained"], NOMINAL["f16_tflops"])})
+    del sw
+    torch.cuda.empty_cache()
+    return rec
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def run_ours(args):
@@ -480,7 +671,11 @@ def run_ours(args):
     # a graph of ten back-to-back launches on its own weights (warm L2), against the burst peak, because such a
     # graph is over in a millisecond
     per_layer = None
+    probe_int8 = None
     if args.table == "w4a8" and world == 1 and args.tokens == 0:
+        # second denominator: back-to-back int8 MMAs on operands resident in shared memory, all SMs
+        with torch.cuda.stream(stream):
+            probe_int8 = mixdq.probe_mma_loop(1, 64)
         per_layer = []
         burst = peaks["bf16_tflops"] * INT8_TO_BF16_NOMINAL
         for name in ("up64_640#0", "res64_320_320#0", "res32_640_640#0", "up32_1280#0", "res16_1280_1280#0",
@@ -503,22 +698,32 @@ def run_ours(args):
                 torch.cuda.synchronize()
             us = t0.elapsed_time(t1) * 1e3 / (reps * rounds)
             tops = pl.spec.ops(args.batch) / us / 1e6
+            kb = 9 * ((pl.spec.Cin + 127) // 128) if pl.spec.kind == "conv3x3" else (pl.spec.K + 127) // 128
+            rows, cols = mixdq.int8_tile_plan(pl.spec.rows(args.batch), pl.spec.N, kb, pl.spec.w_bits)
             per_layer.append({"layer": name, "kind": pl.spec.kind, "M": pl.spec.rows(args.batch), "N": pl.spec.N,
-                              "K": pl.spec.K, "w_bits": pl.spec.w_bits, "us": round(us, 2), "tops": round(tops, 1),
-                              "frac_of_burst_peak": round(tops / burst, 3)})
+                              "K": pl.spec.K, "w_bits": pl.spec.w_bits, "tile": f"{rows}x{cols}", "us": round(us, 2),
+                              "tops": round(tops, 1), "frac_of_burst_peak": round(tops / burst, 3),
+                              "frac_of_sustained_peak": round(tops / (peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL), 3),
+                              "frac_of_int8_mma_probe": round(tops / probe_int8, 3),
+                              "frac_of_nominal": round(tops / NOMINAL["int8_tops"], 3)})
     if args.table == "w4a8":
         tc_ops = sweep.total_ops(tc_layers)
         achieved = tc_ops / (tc_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL
-        # DRAM bytes per step of these kernels from one ncu capture of this command at batch 4 (caches flushed
-        # before every launch; see profiles/dram_bench_unet_sweep_w4a8_b4.txt): 3.01 GB read by the quantization
-        # passes (every layer's input once) + 3.00 GB by the GEMMs (weights and int8 activations once)
-        traffic = 6.01e9 if (args.batch == 4 and world == 1 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections) else None
+        # (no DRAM counter figure here: the kernels have changed since the last capture of a whole step; the
+        # algorithmic bytes of the step stand beside it, and per-layer captures are summarised under profiles/)
+        traffic = None
+        alg_bytes = sum(sweep.algorithmic_bytes(pl) for pl in tc_layers)
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s", "frac": achieved / peak,
                     "traffic": traffic,
-                    "kernel": "i8 tcgen05 kind::i8 GEMM kernels (tma_gemm_kernel, tma_gemm_persistent_kernel) with "
-                              "their quant_kernel pre-pass, all tensor-core int8 layers of the step",
+                    "kernel": "i8 tcgen05 kind::i8 GEMM kernels (pair_gemm_kernel on two-CTA tiles, tma_gemm_kernel, "
+                              "tma_gemm_persistent_kernel) with their quant_kernel pre-pass, all tensor-core int8 layers of "
+                              "the step",
                     "peak_source": f"{peaks['source']} bf16 sustained x {INT8_TO_BF16_NOMINAL:g} (nominal int8:bf16)",
+                    "frac_of_nominal": achieved / NOMINAL["int8_tops"],
+                    "frac_of_int8_mma_probe": (achieved / probe_int8) if probe_int8 else None,
+                    "algorithmic_bytes_per_step": alg_bytes,
+                    "algorithmic_gb_per_s": alg_bytes / (tc_ms * 1e-3) / 1e9,
                     "launches_per_step": group_launches[0], "layers": len(tc_layers), "ms_per_step": tc_ms}
     elif args.tokens > 0:
         # a few tokens per layer: one stream over the packed weights, bound by HBM
@@ -565,6 +770,22 @@ def run_ours(args):
             "large_m_layers": per_layer,
             "device_status": status,
         }
+        default_run = (world == 1 and args.table == "w4a8" and args.tokens == 0 and not args.act_asym and
+                       not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections and
+                       args.batch == 4 and not args.no_extras)
+        if default_run:
+            from paper_2405_17873_b200 import synth
+            out["peaks"] = {"measured": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_burst": peaks["bf16_tflops"],
+                                         "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                                         "int8_mma_loop_probe_tops": round(probe_int8, 1), "source": peaks["source"]},
+                            "nominal": NOMINAL}
+            del sweep.workspace
+            out["configs"] = config_records(torch, mixdq, synth, stream, peaks, probe_int8)
+            out["weight_bound_layers"] = weight_bound_records(torch, mixdq, synth, stream, peaks)
+            sweep = None
+            torch.cuda.empty_cache()
+            out["other_sweeps"] = [sub_sweep_record(torch, UNetSweep, stream, peaks, args.batch, 0),
+                                   sub_sweep_record(torch, UNetSweep, stream, peaks, args.batch, 16)]
         if world == 1 and not args.no_cpu_baseline and args.tokens == 0 and not args.act_asym and not args.shortcut_split and not args.share_qkv_quant and not args.fuse_projections and args.low_bits == 3:
             out["cpu_baseline"] = cpu_baseline(args.table, args.batch, 15.0)
         print(json.dumps(out))

@@ -238,7 +238,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     tc_fence_after_sync();
     // everything above is independent of earlier kernels; global memory is not, except the packed weights
     // (constants of the layer), whose producer runs ahead
-    if (warp != L::B_WARP) pdl_wait();
+    // (and the warps that expand them, which touch shared memory only)
+    if (warp != L::B_WARP && !(W4 && warp >= 6 && warp < L::HELPER0)) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {

@@ -595,7 +595,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     tc_fence_after_sync();
     // everything above is independent of earlier kernels; global memory is not, except the packed
     // weights: no kernel that launches dependents early writes them, so their producer runs ahead
-    if (warp != L::B_WARP) pdl_wait();
+    // (nor do the warps that expand them, which touch shared memory only: the first weight tiles are expanded
+    // while the previous kernel drains, and those warps wait before they turn to anything else)
+    const bool expander = W4 && warp >= 6 && warp < L::B_WARP;
+    if (warp != L::B_WARP && !expander) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
@@ -646,6 +649,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             // -------------------------------------------------------- int4 -> int8 (x16) expansion
             const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
             expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, nkb, sB, sP, bar0, s_abort);
+            pdl_wait();  // before these warps help with the epilogue
         }
         if (warp < 10 && !direct) {
             // -------------------------------------------------------- epilogue of a split tile, part 1
@@ -899,7 +903,8 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp != L::B_WARP) pdl_wait();  // the weight producer runs ahead of earlier kernels
+    // the weight producer runs ahead of earlier kernels, and so do the warps that expand int4 weight tiles
+    if (warp != L::B_WARP && !(W4 && warp >= 6 && warp < L::HELPER0)) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
@@ -1075,6 +1080,7 @@ tma_gemm_persistent_kernel(const __grid_constant__ CUtensorMap tmap_a, const __g
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion
         const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
         expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, my_tiles * nkb, sB, sP, bar0, s_abort);
+        pdl_wait();
     }
 
     if (*s_abort) {
