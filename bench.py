@@ -744,8 +744,8 @@ def run_ours(args):
         alg = sum(sweep.algorithmic_bytes(pl) for pl in sweep.layers)
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "traffic": None,
-                    "kernel": "wo::wo_tc_kernel (tcgen05 kind::f16, weights expanded to fp16 in shared memory), "
-                              "all layers of the step",
+                    "kernel": "weight expansion to fp16 (once per layer call, into the workspace) + pair_gemm_kernel in its "
+                              "tcgen05 kind::f16 mode; layers under 256 rows on wo_tc_kernel / wo_kernel; all layers of the step",
                     "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
                     "launches_per_step": group_launches[1], "ms_per_step": other_ms,
                     "algorithmic_gb_per_s": alg / (other_ms * 1e-3) / 1e9}

@@ -147,7 +147,11 @@ int mixdq_weight_code_sums(const void* packed_W, int64_t N, int64_t K, int bits,
  * A result of 0 means the call runs without scratch.  The workspace is optional for every
  * call (NULL / 0 bytes): without it the int8 layers run as one fused kernel that quantizes
  * the activations while it feeds the tensor cores; with it, the activations are first
- * quantized once into the workspace and the GEMM is then fed entirely by TMA.
+ * quantized once into the workspace and the GEMM is then fed entirely by TMA.  Weight-only
+ * layers (act_bits = 16) on 256 rows or more use a workspace too: the layer's weights are
+ * expanded once per call to fp16 integers (q - zero) there and the GEMM runs on fp16 tensor
+ * cores with both operands fed by TMA (the paper's weight-only mode saves memory, not time:
+ * Table 1 caption); without it, or on fewer rows, weight tiles are expanded inside the GEMM.
  */
 int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_bits, int act_bits,
                           size_t* out);

@@ -70,6 +70,8 @@ int linear_impl(const void* X, int64_t M, int64_t K, int64_t ldx, const void* pa
     p.Y = static_cast<__half*>(Y);
     p.ldy = N;
     p.status = status;
+    p.workspace = workspace;
+    p.ws_bytes = ws_bytes;
     return wo::run(p, A_LINEAR, packed_W, w_bits, st);
 }
 
@@ -136,6 +138,8 @@ int conv3_impl(const void* X, int64_t B, int64_t H, int64_t W, int64_t Cin, cons
     p.Y = static_cast<__half*>(Y);
     p.ldy = Cout;
     p.status = status;
+    p.workspace = workspace;
+    p.ws_bytes = ws_bytes;
     return wo::run(p, A_CONV3, packed_W, w_bits, st);
 }
 
@@ -214,7 +218,8 @@ extern "C" int mixdq_workspace_bytes(int64_t rows, int64_t N, int64_t K, int w_b
     if (!out || rows <= 0 || N <= 0 || K <= 0) return MIXDQ_ERR_INVALID_ARG;
     if (act_bits != 8 && act_bits != 16) return MIXDQ_ERR_UNSUPPORTED;
     if (w_bits != 2 && w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
-    *out = (act_bits == 8) ? i8::workspace_bytes(rows, N, rows, K) : 0;
+    // weight-only layers: room for the weights expanded to fp16, used on 256 rows or more
+    *out = (act_bits == 8) ? i8::workspace_bytes(rows, N, rows, K) : (rows >= 256 ? wo::expanded_weight_bytes(N, K) : 0);
     return MIXDQ_OK;
 }
 
@@ -227,7 +232,8 @@ extern "C" int mixdq_conv3x3_workspace_bytes(int64_t B, int64_t H, int64_t W, in
     if (w_bits != 2 && w_bits != 3 && w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     const int64_t Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
     // room for the int8 image with a one-pixel border, which the asymmetric-activation call keeps
-    *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * (H + 2) * (W + 2), Cin) : 0;
+    *out = (act_bits == 8) ? i8::workspace_bytes(B * Ho * Wo, Cout, B * (H + 2) * (W + 2), Cin)
+                           : (B * Ho * Wo >= 256 ? wo::expanded_weight_bytes(Cout, 9 * Cin) : 0);
     return MIXDQ_OK;
 }
 

@@ -61,7 +61,7 @@ int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4]
                       const uint32_t box[4], uint32_t hw_step = 1);
 // The same for an fp16 NHWC image (box extents in elements, strides in bytes).
 int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                       const uint32_t box[4]);
+                       const uint32_t box[4], uint32_t hw_step = 1);
 
 // Once per kernel: ask for the largest shared-memory carve-out.  An SM changes its L1 / shared
 // split only when idle, so kernels with different preferences cannot share an SM and the change

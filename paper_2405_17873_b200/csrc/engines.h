@@ -88,9 +88,17 @@ struct Params {
     __half* Y = nullptr;
     long long ldy = 0;
     int32_t* status = nullptr;
+    // optional scratch for the layer's weights expanded to fp16 (many-token path); no initial content needed
+    void* workspace = nullptr;
+    size_t ws_bytes = 0;
 };
 
 int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream);
+// Many-token path with a workspace: the packed weights are expanded ONCE per call to fp16 (q - zero), then both
+// operands reach a two-CTA tcgen05 kind::f16 GEMM by TMA; see wo_pair.cu.
+size_t expanded_weight_bytes(int64_t N, int64_t K);
+bool pair_path_ok(const Params& p, int amode, int w_bits);
+int run_pair(const Params& p, int amode, const void* packed, int w_bits, cudaStream_t stream);
 // Many-token path on tcgen05 (fp16 MMA, weights expanded into shared memory); see wo_tc.cu.
 bool tc_path_ok(const Params& p, int amode, int w_bits);
 int run_tc(const Params& p, int amode, const void* packed, int w_bits, int batch, cudaStream_t stream);

@@ -79,6 +79,29 @@ __device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, ui
         : "memory");
 }
 
+// The same with fp16 operands and fp32 accumulation.
+__device__ __forceinline__ void mma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <bool F16>
+__device__ __forceinline__ void mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate)
+{
+    if (F16)
+        mma_f16_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+    else
+        mma_i8_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+}
+
 // Once every MMA this thread issued so far has completed: arrive on the barrier at this shared-memory offset
 // in both CTAs of the pair.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)
@@ -122,8 +145,12 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar)
 constexpr int PAIR_BN_MAX = 256;
 constexpr int ACC_COLS = 256;  // tensor-memory columns of one accumulator (the widest tile)
 
-template <bool W4>
+// MODE: 0 = int8 weights, 1 = int4 weights (expanded in shared memory), 2 = fp16 operands (kind::f16)
+template <int MODE>
 struct PairSmem {
+    static constexpr bool W4 = MODE == 1;
+    static constexpr bool F16 = MODE == 2;
+    static constexpr int BKE = F16 ? BK / 2 : BK;           // elements of a k-block (its rows are 128 bytes either way)
     static constexpr int A_BYTES = BM * BK;                 // this CTA's 128 activation rows of a k-block
     static constexpr int B_BYTES = (PAIR_BN_MAX / 2) * BK;  // this CTA's half of the int8 weight tile
     static constexpr int P_BYTES = B_BYTES / 2;             // the same as packed int4
@@ -172,12 +199,15 @@ struct PairArgs {
     int total_tiles;  // pair tiles in all
 };
 
-template <bool W4>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairSmem<W4>::THREADS, 1)
+template <int MODE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairSmem<MODE>::THREADS, 1)
 pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, const PairArgs g)
 {
-    using L = PairSmem<W4>;
+    using L = PairSmem<MODE>;
+    constexpr bool W4 = L::W4;
+    constexpr bool F16 = L::F16;
+    constexpr int BKE = L::BKE;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
@@ -239,7 +269,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     // everything above is independent of earlier kernels; global memory is not, except the packed weights
     // (constants of the layer), whose producer runs ahead
     // (and the warps that expand them, which touch shared memory only)
-    if (warp != L::B_WARP && !(W4 && warp >= 6 && warp < L::HELPER0)) pdl_wait();
+    // (fp16 mode: the weight operand is the output of the expansion kernel launched just before: everyone waits)
+    if ((F16 || warp != L::B_WARP) && !(W4 && warp >= 6 && warp < L::HELPER0)) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
@@ -265,7 +296,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (leader) mbar_arrive_expect_tx(bar0 + 8 * (L::FULL_A + s), 2 * L::A_BYTES);
                     const uint32_t full = lead_bar0 + 8 * (L::FULL_A + s);
                     if (p.conv) {
-                        tma_load_4d_pair(a0 + s * L::A_BYTES, &tmap_a, cb * BK, p.stride * wo0 + kw - 1 + p.pad,
+                        tma_load_4d_pair(a0 + s * L::A_BYTES, &tmap_a, cb * BKE, p.stride * wo0 + kw - 1 + p.pad,
                                          p.stride * ho0 + kh - 1 + p.pad, img_b, full);
                         if (++cb == p.cblocks) {
                             cb = 0;
@@ -276,7 +307,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         }
                     } else {
                         tma_load_2d_pair(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
-                        xa += BK;
+                        xa += BKE;
                     }
                     if (++s == L::AS) {
                         s = 0;
@@ -290,7 +321,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // ------------------------------------------------------------ weight-tile producer (own half of the rows)
         if (lane == 0) {
             constexpr int R = W4 ? L::PS : L::ES;
-            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
+            constexpr int ROW_BYTES = W4 ? BK / 2 : BK;   // bytes of a k-block of one weight row
+            constexpr int ROW_STEP = F16 ? BKE : ROW_BYTES;  // the same in units of the weight map's element
             uint32_t s = 0, par = 1;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
@@ -305,14 +337,14 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                     int x = xb;
                     if (p.conv) {
-                        const int kx = kx_tap + cb * BK;
+                        const int kx = kx_tap + cb * BKE;
                         x = W4 ? kx / 2 : kx;
                         if (++cb == p.cblocks) {
                             cb = 0;
                             kx_tap += p.Cin;
                         }
                     }
-                    xb += ROW_BYTES;
+                    xb += ROW_STEP;
                     if (W4) {
                         // packed rows are consumed inside this CTA: a barrier of its own
                         const uint32_t full = bar0 + 8 * (L::FULL_P + s);
@@ -342,7 +374,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // the two threads' instructions).  A tile is complete when both threads' commits have arrived.
         if (lane == 0 && leader) {
             const int which = warp == 1 ? 0 : 1;
-            const uint32_t idesc = make_idesc(2, 1, 2 * BM, static_cast<uint32_t>(bn));
+            const uint32_t idesc = F16 ? make_idesc(1, 0, 2 * BM, static_cast<uint32_t>(bn))
+                                       : make_idesc(2, 1, 2 * BM, static_cast<uint32_t>(bn));
             const uint64_t a_desc0 = smem_desc_sw128(a0), b_desc0 = smem_desc_sw128(b0);
             const uint32_t tile_go = bar0 + 8 * L::TILE_GO;
             bool ok = true;
@@ -369,9 +402,10 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     tc_fence_after_sync();
                     const uint64_t a_desc = a_desc0 + sa * (L::A_BYTES >> 4);
                     const uint64_t b_desc = b_desc0 + se * (L::B_BYTES >> 4);
-                    mma_i8_pair(acc, a_desc, b_desc, idesc, i != 0);
+                    // four instructions of 32 bytes along the reduction: 32 int8 or 16 fp16 elements each
+                    mma_pair<F16>(acc, a_desc, b_desc, idesc, i != 0);
 #pragma unroll
-                    for (int k = 1; k < BK / 32; ++k) mma_i8_pair(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
+                    for (int k = 1; k < BK / 32; ++k) mma_pair<F16>(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
                     if (i == 0 && nkb > 1) {
                         // the overwriting MMA is in the pipe's queue: the other thread may add to the accumulator
                         tc_fence_before_sync();
@@ -400,7 +434,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int lg = warp & 3;
         const int half = warp < 6 ? 0 : 1;
         const int et = tid - 64;  // epilogue warps only: 0..127
-        const float sx = p.act_scale ? __ldg(p.act_scale) : 0.f;  // absent: accumulators only
+        // (fp16 mode: the activations are not quantized, the factor of a column is its weight scale)
+        const float sx = F16 ? 1.f : (p.act_scale ? __ldg(p.act_scale) : 0.f);  // absent: accumulators only
         const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
         // the 32-column passes of a tile are dealt to the two halves of the warps
         const int passes = bn >> 5;
@@ -448,7 +483,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 continue;
             }
             const uint32_t acc = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
-            if (p.acc_out) {
+            if (!F16 && p.acc_out) {
                 // raw int32 sums (parity hook): a lane owns a row, 32 columns of it at a time
                 const int m = m0 + lg * 32 + lane;
                 for (int c0 = c_begin; c0 < c_begin + c_count; c0 += 32) {
@@ -469,9 +504,14 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 }
             }
-            if (p.Y && c_count > 0)
-                store_rows32_dispatch<W4>(acc + c_begin, 0, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
-                                          m0 + lg * 32, n0 + c_begin, lane);
+            if (p.Y && c_count > 0) {
+                if (F16)
+                    store_rows32_f32(acc + c_begin, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
+                                     m0 + lg * 32, n0 + c_begin, lane);
+                else
+                    store_rows32_dispatch<W4>(acc + c_begin, 0, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
+                                              m0 + lg * 32, n0 + c_begin, lane);
+            }
             // the accumulator may be overwritten once every epilogue warp of both CTAs has read it
             tc_fence_before_sync();
             __syncwarp();
@@ -545,12 +585,12 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (warp == 1) tmem_dealloc_pair(tmem_base, 2 * ACC_COLS);
 }
 
-template <bool W4>
+template <int MODE>
 int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
                   int num_sms, cudaStream_t stream)
 {
-    using L = PairSmem<W4>;
-    auto kernel = pair_gemm_kernel<W4>;
+    using L = PairSmem<MODE>;
+    auto kernel = pair_gemm_kernel<MODE>;
     if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     PairArgs g;
     g.bn = bn;
@@ -568,8 +608,15 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap&
                 int num_sms, cudaStream_t stream)
 {
     if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2) return MIXDQ_ERR_INVALID_ARG;
-    return w4 ? launch_pair_t<true>(ta, tw, ty, tp, bn, num_sms, stream)
-              : launch_pair_t<false>(ta, tw, ty, tp, bn, num_sms, stream);
+    return w4 ? launch_pair_t<1>(ta, tw, ty, tp, bn, num_sms, stream)
+              : launch_pair_t<0>(ta, tw, ty, tp, bn, num_sms, stream);
+}
+
+int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+                    int num_sms, cudaStream_t stream)
+{
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || tp.acc_out) return MIXDQ_ERR_INVALID_ARG;
+    return launch_pair_t<2>(ta, tw, ty, tp, bn, num_sms, stream);
 }
 
 }  // namespace i8

@@ -41,9 +41,10 @@ struct TmaParams {
 // int32 accumulator -> float.  W4 accumulators carry the factor 16 of the nibble placement, removed
 // here by an exact shift.  SMALL: |v| < 2^22, so adding v to the bit pattern of 1.5 * 2^23 and
 // subtracting that constant is exact -- two full-rate instructions instead of a quarter-rate convert.
-template <bool W4, bool SMALL>
+template <bool W4, bool SMALL, bool F32 = false>
 __device__ __forceinline__ float acc_to_float(uint32_t r)
 {
+    if (F32) return __uint_as_float(r);  // fp16 MMAs accumulate in fp32: the register already holds the sum
     const int32_t v = W4 ? (static_cast<int32_t>(r) >> 4) : static_cast<int32_t>(r);
     if (SMALL) return __int_as_float(0x4B400000 + v) - 12582912.f;
     return static_cast<float>(v);
@@ -57,7 +58,7 @@ __device__ __forceinline__ float acc_to_float(uint32_t r)
 constexpr int EPI32_ROW = 80;
 constexpr int EPI32_TILE = 32 * EPI32_ROW;  // 2560: a multiple of 512, the period of the 64-byte swizzle
 
-template <bool W4, bool SMALL, bool TMA>
+template <bool W4, bool SMALL, bool TMA, bool F32 = false>
 __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
                                                        const float* bias, uint8_t* stage, const TmaParams& p,
                                                        const CUtensorMap* tmap_y, int m_first, int n0, int lane)
@@ -86,14 +87,14 @@ __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t ac
             const float4 ba = *reinterpret_cast<const float4*>(bias + c);
             const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
             __half2 hv[4];
-            hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j]), ca.x, ba.x),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 1]), ca.y, ba.y));
-            hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 2]), ca.z, ba.z),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 3]), ca.w, ba.w));
-            hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 4]), cb.x, bb.x),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 5]), cb.y, bb.y));
-            hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL>(r[j + 6]), cb.z, bb.z),
-                                      fmaf(acc_to_float<W4, SMALL>(r[j + 7]), cb.w, bb.w));
+            hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r[j]), ca.x, ba.x),
+                                      fmaf(acc_to_float<W4, SMALL, F32>(r[j + 1]), ca.y, ba.y));
+            hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r[j + 2]), ca.z, ba.z),
+                                      fmaf(acc_to_float<W4, SMALL, F32>(r[j + 3]), ca.w, ba.w));
+            hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r[j + 4]), cb.x, bb.x),
+                                      fmaf(acc_to_float<W4, SMALL, F32>(r[j + 5]), cb.y, bb.y));
+            hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r[j + 6]), cb.z, bb.z),
+                                      fmaf(acc_to_float<W4, SMALL, F32>(r[j + 7]), cb.w, bb.w));
             out[j >> 3] = *reinterpret_cast<const uint4*>(hv);
         }
         if (TMA) {
@@ -142,6 +143,11 @@ __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t ac
     }
 }
 
+// fp32 accumulators (weight-only layers on fp16 MMAs)
+__device__ __forceinline__ void store_rows32_f32(uint32_t acc, int ncols, const float* comb, const float* bias,
+                                                 uint8_t* stage, const TmaParams& p, const CUtensorMap* tmap_y,
+                                                 int m_first, int n0, int lane);
+
 template <bool W4>
 __device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
                                                       const float* bias, uint8_t* stage, const TmaParams& p,
@@ -160,10 +166,25 @@ __device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc
     }
 }
 
+__device__ __forceinline__ void store_rows32_f32(uint32_t acc, int ncols, const float* comb, const float* bias,
+                                                 uint8_t* stage, const TmaParams& p, const CUtensorMap* tmap_y,
+                                                 int m_first, int n0, int lane)
+{
+    if (p.tma_store)
+        store_rows32_from_tmem<false, false, true, true>(acc, 0, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+    else
+        store_rows32_from_tmem<false, false, false, true>(acc, 0, ncols, comb, bias, stage, p, tmap_y, m_first, n0, lane);
+}
+
 // Pair form (i8_pair.cu): persistent kernel of two-CTA clusters on 256 x bn tiles.  ta: activation map with a
 // box of 128 rows (or pixels), tw: weight map with a box of bn / 2 rows, ty: output map with a 32 x 32 box.
 int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
                 int num_sms, cudaStream_t stream);
+// The same kernel on fp16 operands (kind::f16, fp32 accumulators) for the weight-only layers: ta an fp16 map with a
+// box of 128 rows x 64 elements, tw the map of the layer's weights expanded to fp16 (q - zero) with a box of
+// bn / 2 rows x 64 elements; tp.k_blocks counts blocks of 64 elements and tp.act_scale is unused.
+int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+                    int num_sms, cudaStream_t stream);
 
 }  // namespace i8
 }  // namespace mixdq

@@ -77,9 +77,9 @@ int encode_tmap_4d_u8(CUtensorMap* map, const void* base, const uint64_t dims[4]
 }
 
 int encode_tmap_4d_f16(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                       const uint32_t box[4])
+                       const uint32_t box[4], uint32_t hw_step)
 {
-    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, base, dims, strides_bytes, box, 1);
+    return encode_tmap_4d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, base, dims, strides_bytes, box, hw_step);
 }
 
 static int encode_tmap_4d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, const uint64_t dims[4],

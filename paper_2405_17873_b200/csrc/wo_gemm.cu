@@ -531,6 +531,7 @@ int run(Params p, int amode, const void* packed, int w_bits, cudaStream_t stream
         return MIXDQ_ERR_ALIGNMENT;
     const long long pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
     const bool is_signed = p.w_zero == nullptr;
+    if (pair_path_ok(p, amode, w_bits)) return run_pair(p, amode, packed, w_bits, stream);
     if (tc_path_ok(p, amode, w_bits) && !(w_bits <= 3 && is_signed)) return run_tc(p, amode, packed, w_bits, p.batch, stream);
     if (w_bits == 3) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_nt<3, false>(p, amode, packed, pitch, stream);
     if (w_bits == 2) return is_signed ? MIXDQ_ERR_UNSUPPORTED : launch_nt<2, false>(p, amode, packed, pitch, stream);

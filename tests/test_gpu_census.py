@@ -138,14 +138,17 @@ def test_weight_only_layer_one_row_per_tile(name, w_bits, B):
     s, z = mixdq.weight_minmax_params(Wd, w_bits, False)
     packed = mixdq.pack_weights(Wd, w_bits, s, z)
     st = status_word()
+    # with the workspace the layer sweep passes (256 rows or more: weights expanded once to fp16, two-CTA fp16 GEMM)
     if l.kind == "conv3x3":
-        y = host(mixdq.conv3x3(Xd, packed, l.N, w_bits, s, z, 16, None, dev(b), l.stride, None, st)).reshape(-1, l.N)
+        ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, l.H, l.H, l.Cin, l.N, l.stride, w_bits, 16))
+        y = host(mixdq.conv3x3(Xd, packed, l.N, w_bits, s, z, 16, None, dev(b), l.stride, ws, st)).reshape(-1, l.N)
         rows = rows_one_per_tile(y.shape[0])
         a_rows = window_rows(X, rows, l.stride)
     else:
         # the weight-only table keeps the text projections in fp16 activations too: a plain linear layer on all rows
         X2 = np.ascontiguousarray(X.reshape(-1, l.K))
-        y = host(mixdq.linear(Xd.reshape(-1, l.K), packed, l.N, w_bits, s, z, 16, None, dev(b), None, st))
+        ws = mixdq.new_workspace(mixdq.workspace_bytes(X2.shape[0], l.N, l.K, w_bits, 16))
+        y = host(mixdq.linear(Xd.reshape(-1, l.K), packed, l.N, w_bits, s, z, 16, None, dev(b), ws, st))
         rows = rows_one_per_tile(X2.shape[0])
         a_rows = X2[rows]
     y_ref = orc.linear_a16(np.ascontiguousarray(a_rows), codes, s_ref, z_ref, b)

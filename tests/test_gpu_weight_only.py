@@ -10,12 +10,14 @@ from helpers import assert_close, dev, device_weights, host, oracle_weights
 pytestmark = pytest.mark.gpu
 
 
-def _run(X, W, b, bits, symmetric=False):
+def _run(X, W, b, bits, symmetric=False, use_ws=False):
+    M, K = X.shape
     N = W.shape[0]
     s_ref, z_ref, codes = oracle_weights(W, bits, symmetric)
     y_ref = orc.linear_a16(X, codes, s_ref, z_ref, b)
     s, z, packed = device_weights(W, bits, symmetric)
-    y = mixdq.linear(dev(X), packed, N, bits, s, z, 16, None, None if b is None else dev(b))
+    ws = mixdq.new_workspace(mixdq.workspace_bytes(M, N, K, bits, 16)) if use_ws else None
+    y = mixdq.linear(dev(X), packed, N, bits, s, z, 16, None, None if b is None else dev(b), ws)
     torch.cuda.synchronize()
     assert_close(host(y), y_ref)
 
@@ -52,6 +54,38 @@ def test_symmetric_codes_many_tokens(bits):
     X = synth.normal_f16((256, 640), 1.0, seed=3)
     W = synth.normal_f16((72, 640), 0.02, seed=4)
     _run(X, W, None, bits, symmetric=True)
+    _run(X, W, None, bits, symmetric=True, use_ws=True)
+
+
+# 256 tokens or more and a workspace: the weights are expanded once to fp16 integers in the workspace and a
+# two-CTA tcgen05 kind::f16 GEMM reads both operands by TMA (ragged rows, columns and reduction lengths, one
+# and several tiles per CTA pair)
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("M,K,N", [(256, 64, 32), (300, 2888, 136), (2100, 328, 1300), (1000, 1288, 1290), (4096, 320, 1280),
+                                   (5000, 200, 264)])
+def test_many_token_shapes_with_workspace(bits, M, K, N):
+    X = synth.normal_f16((M, K), 1.0, seed=M * 7 + K)
+    W = synth.normal_f16((N, K), 0.02, seed=N * 11 + K)
+    b = synth.normal_f16((N,), 0.01, seed=N + 2)
+    _run(X, W, b, bits, use_ws=True)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("geom", [(2, 16, 16, 64, 40, 1), (1, 32, 32, 200, 136, 1), (3, 32, 32, 192, 136, 1),
+                                  (2, 32, 32, 72, 264, 2), (1, 64, 64, 96, 48, 2)])
+def test_weight_only_conv3x3_with_workspace(bits, geom):
+    B, H, Wd, Cin, Cout, stride = geom
+    X = synth.normal_f16((B, H, Wd, Cin), 1.0, seed=17)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=18)
+    b = synth.normal_f16((Cout,), 0.01, seed=19)
+    s_ref, z_ref, codes = oracle_weights(Wt.reshape(Cout, -1), bits, False)
+    y_ref = orc.conv3x3_a16(X, codes.reshape(Cout, 3, 3, Cin), s_ref, z_ref, b, stride)
+    s, z, packed = device_weights(Wt.reshape(Cout, -1), bits, False)
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, Wd, Cin, Cout, stride, bits, 16))
+    assert ws is not None
+    y = mixdq.conv3x3(dev(X), packed, Cout, bits, s, z, 16, None, dev(b), stride, ws)
+    torch.cuda.synchronize()
+    assert_close(host(y), y_ref)
 
 
 @pytest.mark.parametrize("bits", [4, 8])
