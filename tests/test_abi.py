@@ -67,7 +67,9 @@ def test_packed_bytes_size_laws(lib):
 def test_argument_errors_come_back_before_any_launch(lib):
     out = C.c_size_t(0)
     assert lib.mixdq_workspace_bytes(256, 320, 320, 8, 8, C.byref(out)) == 0 and out.value > 0
-    assert lib.mixdq_workspace_bytes(256, 320, 320, 4, 16, C.byref(out)) == 0 and out.value == 0
+    # weight-only layers: room for the fp16 expansion of the weights from 256 rows on, none below
+    assert lib.mixdq_workspace_bytes(256, 320, 320, 4, 16, C.byref(out)) == 0 and out.value == 320 * 320 * 2
+    assert lib.mixdq_workspace_bytes(16, 320, 320, 4, 16, C.byref(out)) == 0 and out.value == 0
     assert lib.mixdq_workspace_bytes(256, 320, 320, 5, 8, C.byref(out)) == -2
     assert lib.mixdq_workspace_bytes(0, 320, 320, 8, 8, C.byref(out)) == -1
     null = None
