@@ -276,6 +276,19 @@ int mixdq_conv3x3_q8(const void* Xq, int64_t B, int64_t H, int64_t W, int64_t Ci
                      int64_t Cout, int stride, int w_bits, const float* w_scale, const float* act_scale,
                      const void* bias, void* Y, int32_t* status, void* stream);
 
+/*
+ * Self-test of the kernels' bounded waits (the paper has no counterpart).  Runs mixdq_linear_q8 on the given
+ * operands, except that the weight tile of reduction block drop_k_block (1-based, blocks of 128) is announced
+ * to its barrier and then never requested.  The warps that wait for it give up when their cycle budget (a few
+ * hundred milliseconds) runs out: the kernel raises its abort flag, lets its copies in flight land, writes
+ * MIXDQ_ERR_TIMEOUT to *status (required), releases its tensor memory and returns; nothing traps and the
+ * context stays usable.  Y is written with unspecified values.  The call itself returns MIXDQ_OK (the launch
+ * succeeded).  For tests: it shows that a lost transfer ends in a status word, not in a hung GPU.
+ */
+int mixdq_selftest_abandoned_wait(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
+                                  const float* w_scale, const float* act_scale, void* Y, int drop_k_block,
+                                  int32_t* status, void* stream);
+
 /* Parity hook: int32 accumulators [M, N] of mixdq_linear_q8. */
 int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
                             int32_t* acc_out, int32_t* status, void* stream);

@@ -321,7 +321,7 @@ namespace {
 
 int linear_q8_impl(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N, int w_bits,
                    const float* w_scale, const float* act_scale, const void* bias, void* Y, int32_t* acc_out,
-                   int32_t* status, void* stream)
+                   int32_t* status, void* stream, int test_drop_b_kblock = 0)
 {
     if (!Xq || !packed_W || (!Y && !acc_out)) return MIXDQ_ERR_INVALID_ARG;
     if (!fits_int(M) || !fits_int(K) || !fits_int(N)) return MIXDQ_ERR_INVALID_ARG;
@@ -341,6 +341,7 @@ int linear_q8_impl(const void* Xq, int64_t M, int64_t K, const void* packed_W, i
     p.ldy = N;
     p.acc_out = acc_out;
     p.status = status;
+    p.test_drop_b_kblock = test_drop_b_kblock;
     return i8::run_tma_prequantized(p, A_LINEAR, packed_W, w_bits, static_cast<const int8_t*>(Xq),
                                     static_cast<cudaStream_t>(stream));
 }
@@ -353,6 +354,16 @@ extern "C" int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void*
 {
     if (!Y) return MIXDQ_ERR_INVALID_ARG;
     return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, w_scale, act_scale, bias, Y, nullptr, status, stream);
+}
+
+extern "C" int mixdq_selftest_abandoned_wait(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N,
+                                             int w_bits, const float* w_scale, const float* act_scale, void* Y,
+                                             int drop_k_block, int32_t* status, void* stream)
+{
+    if (!Y || !status) return MIXDQ_ERR_INVALID_ARG;
+    if (drop_k_block < 1 || drop_k_block > (K + 127) / 128) return MIXDQ_ERR_INVALID_ARG;
+    return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, w_scale, act_scale, nullptr, Y, nullptr, status, stream,
+                          drop_k_block);
 }
 
 extern "C" int mixdq_linear_q8_acc_i32(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N,

@@ -41,6 +41,9 @@ struct Params {
     // activation scale; the epilogue adds addend * (*addend_scale) * w_scale[n]
     const int32_t* addend = nullptr;
     const float* addend_scale = nullptr;
+    // self-test of the bounded waits (mixdq_selftest_abandoned_wait): > 0 = the weight tile of that k-block
+    // (1-based) is announced to its barrier but never requested, so the waits on it run out
+    int test_drop_b_kblock = 0;
 };
 
 // Scratch of the fused kernel's split reduction (tickets + int32 partial sums).

@@ -400,15 +400,17 @@ __device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const 
         if (round > 0 && !mbar_wait(bar0 + 8 * (EMPTY + s), (round & 1) ^ 1, s_abort)) return false;
         const uint32_t full = bar0 + 8 * (FULL + s);
         mbar_arrive_expect_tx(full, BN * ROW_BYTES);
+        // (self-test of the bounded waits: one announced tile is never requested)
+        const bool drop = p.test_drop_b_kblock != 0 && kb_begin + i + 1 == p.test_drop_b_kblock;
         if (p.conv) {
             const int kx = kx_tap + cb * BK;
-            tma_load_2d(ring0 + s * SLOT, tmap_w, W4 ? kx / 2 : kx, n0, full);
+            if (!drop) tma_load_2d(ring0 + s * SLOT, tmap_w, W4 ? kx / 2 : kx, n0, full);
             if (++cb == p.cblocks) {
                 cb = 0;
                 kx_tap += p.Cin;
             }
         } else {
-            tma_load_2d(ring0 + s * SLOT, tmap_w, xb, n0, full);
+            if (!drop) tma_load_2d(ring0 + s * SLOT, tmap_w, xb, n0, full);
             xb += ROW_BYTES;
         }
         if (++s == R) {
@@ -1263,6 +1265,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     // rows are consecutive rows of Y (not so for the cross-attention K/V layout, which skips row 0)
     tp.addend = p.addend;
     tp.addend_scale = p.addend_scale;
+    tp.test_drop_b_kblock = p.test_drop_b_kblock;
     tp.tma_store = p.Y && !p.addend && amode != A_BOS && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
     if (conv) {
         int Wb, Hb, Bb;
@@ -1290,7 +1293,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     const int num_sms = sm_count();
     if (num_sms <= 0) return MIXDQ_ERR_CUDA;
     // the pair form (two-CTA tiles of 256 x bn, i8_pair.cu) where its estimate beats the single-CTA kernels
-    const int pair_bn = (!p.addend && amode != A_BOS) ? plan_pair_tile(p.M, p.N, tp.k_blocks, w4, num_sms) : 0;
+    const int pair_bn = (!p.addend && amode != A_BOS && !p.test_drop_b_kblock) ? plan_pair_tile(p.M, p.N, tp.k_blocks, w4, num_sms) : 0;
     if (pair_bn > 0) {
         if (w4)
             rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, pair_bn / 2, false);

@@ -46,6 +46,7 @@ _SIGNATURES = {
     "mixdq_quantize_acts": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "mixdq_linear_q8": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
     "mixdq_conv3x3_q8": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "mixdq_selftest_abandoned_wait": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _int, _vp, _vp]),
     "mixdq_linear_q8_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp]),
     "mixdq_split_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, C.POINTER(_sz)]),
     "mixdq_linear_a8_split": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -340,6 +341,16 @@ def conv3x3_q8(Xq, packed_W, Cout: int, w_bits: int, w_scale, act_scale, bias=No
     Y = out if out is not None else torch.empty((B, Ho, Wo, Cout), dtype=torch.float16, device=Xq.device)
     _chk(lib().mixdq_conv3x3_q8(_ptr(Xq), B, H, W, Cin, _ptr(packed_W), Cout, stride, w_bits, _ptr(w_scale),
                                 _ptr(act_scale), _ptr(bias), _ptr(Y), _ptr(status), _stream()), "mixdq_conv3x3_q8")
+    return Y
+
+
+def selftest_abandoned_wait(Xq, packed_W, N: int, w_bits: int, w_scale, act_scale, drop_k_block: int, status):
+    """mixdq_linear_q8 with one weight tile never requested: *status becomes MIXDQ_ERR_TIMEOUT (-6)."""
+    M, K = Xq.shape
+    Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib().mixdq_selftest_abandoned_wait(_ptr(Xq), M, K, _ptr(packed_W), N, w_bits, _ptr(w_scale), _ptr(act_scale),
+                                             _ptr(Y), drop_k_block, _ptr(status), _stream()),
+         "mixdq_selftest_abandoned_wait")
     return Y
 
 
