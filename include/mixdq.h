@@ -60,7 +60,7 @@ unsigned long long mixdq_kernel_launches(void);
  * current device and with a workspace, for a layer of M output rows, N output channels and k_blocks
  * reduction blocks of 128 (linear layer: ceil(K / 128); 3x3 convolution: 9 * ceil(Cin / 128)).
  * *tile_rows x *tile_cols (HOST pointers) is 256 x {160, 192, 224, 256} when two CTAs on neighbouring SMs
- * share a tile (tcgen05 cta_group::2), else 128 x {128, 256}.  The BOS-aware projection and the second branch
+ * share a tile (tcgen05 cta_group::2), else 128 x {64, 96, 128, 256}.  The BOS-aware projection and the second branch
  * of a shortcut-split layer always run on 128-row tiles.  For tests and benchmarks: nothing is launched. */
 int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols);
 

@@ -194,7 +194,7 @@ extern "C" int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int 
     } else {
         const bool wide = w_bits == 8 && (N >= 1024 || N % 256 == 0) && ceil_div(M, 128) * ceil_div(N, 256) >= 100;
         *tile_rows = 128;
-        *tile_cols = wide ? 256 : 128;
+        *tile_cols = wide ? 256 : i8::plan_narrow_tile(static_cast<int>(M), static_cast<int>(N), static_cast<int>(k_blocks), sms);
     }
     return MIXDQ_OK;
 }

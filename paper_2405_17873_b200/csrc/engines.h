@@ -60,6 +60,8 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
 // Tile width of the pair form (two-CTA tiles of 256 x width) when the planner prefers it for an int8 GEMM of
 // M x N over k_blocks k-blocks of 128, else 0 (the single-CTA kernels run).
 int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms);
+// Tile width (128, 96 or 64) of the one-tile kernel on 128-wide slots.
+int plan_narrow_tile(int M, int N, int k_blocks, int num_sms);
 // The two steps as calls of their own, for activations that are stored as int8 between layers: the codes of
 // X [rows, K] into a dense int8 matrix, and the GEMM / implicit-GEMM convolution on such codes (p.X unused).
 int run_quant(const __half* X, long long ldx, long long rows, int K, const float* act_scale, int8_t* out,

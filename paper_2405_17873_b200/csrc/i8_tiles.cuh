@@ -34,6 +34,7 @@ struct TmaParams {
     // the epilogue adds addend * (*addend_scale) * w_scale[n] to every output (ADD instances of the kernels)
     const int32_t* addend;
     const float* addend_scale;
+    int tile_n;              // one-tile kernel with 128-wide slots: width of the tiles actually computed (0: 128)
     int test_drop_b_kblock;  // self-test: never request the weight tile of this k-block (1-based; 0: none)
     int small_acc;  // every |accumulator| (W4: after the >> 4) stays below 2^22
     int tma_store;  // Y is written through its tensor map (row-contiguous output, 16-byte aligned rows)

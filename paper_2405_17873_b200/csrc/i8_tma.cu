@@ -381,7 +381,8 @@ __device__ __forceinline__ bool produce_a_tile(const CUtensorMap* tmap_a, const 
 // thread, and with both operands on one thread the issue rate sets the k-block cadence.
 template <int BN, bool W4, class L>
 __device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const TmaParams& p, uint32_t seq0, int kb_begin,
-                                               int nkb, int n0, uint32_t ring0, uint32_t bar0, volatile int* s_abort)
+                                               int nkb, int n0, uint32_t ring0, uint32_t bar0, volatile int* s_abort,
+                                               int b_rows = BN)
 {
     constexpr int ROW_BYTES = W4 ? BK / 2 : BK;
     constexpr int R = W4 ? L::PS : L::ES;
@@ -399,7 +400,7 @@ __device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const 
     for (int i = 0; i < nkb; ++i) {
         if (round > 0 && !mbar_wait(bar0 + 8 * (EMPTY + s), (round & 1) ^ 1, s_abort)) return false;
         const uint32_t full = bar0 + 8 * (FULL + s);
-        mbar_arrive_expect_tx(full, BN * ROW_BYTES);
+        mbar_arrive_expect_tx(full, static_cast<uint32_t>(b_rows * ROW_BYTES));  // the rows of the weight map's box
         // (self-test of the bounded waits: one announced tile is never requested)
         const bool drop = p.test_drop_b_kblock != 0 && kb_begin + i + 1 == p.test_drop_b_kblock;
         if (p.conv) {
@@ -430,8 +431,9 @@ __device__ __forceinline__ bool produce_b_tile(const CUtensorMap* tmap_w, const 
 // swizzled int8 tile: nibble -> high half of the byte (= 16 q), two ANDs and a shift per 8 codes.
 template <int BN, class L>
 __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int total_kb, uint8_t* sB, const uint8_t* sP,
-                                               uint32_t bar0, volatile int* s_abort)
+                                               uint32_t bar0, volatile int* s_abort, int b_rows = BN)
 {
+    const int runs = b_rows * 4;  // 16-byte packed runs of a tile
     constexpr int RUNS = (BN * 4) / 64;           // 16-byte packed runs per thread
     constexpr uint32_t PS = L::PS > 0 ? L::PS : 1;  // (instantiated, never run, for W8)
     for (int it = group; it < total_kb; it += 4) {
@@ -447,11 +449,13 @@ __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int 
 #pragma unroll
         for (int t = 0; t < RUNS; ++t) {
             const int task = gt + t * 64;
-            wv[t] = *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16);
+            wv[t] = task < runs ? *reinterpret_cast<const uint4*>(stg + (task >> 2) * (BK / 2) + (task & 3) * 16)
+                                : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int t = 0; t < RUNS; ++t) {
             const int task = gt + t * 64;
+            if (task >= runs) continue;
             const int r = task >> 2, j = task & 3;
             const uint4 w = wv[t];
             uint4 c0, c1;
@@ -480,9 +484,9 @@ __device__ __forceinline__ void expand_nibbles(int group, int gt, int lane, int 
 // are carried along instead of recomputed.  seq0 as above; step <= 2.
 template <int BN, bool W4, class L>
 __device__ __forceinline__ bool issue_k_blocks(int first, int step, int nkb, uint32_t acc, uint32_t seq0, uint32_t a0,
-                                               uint32_t b0, uint32_t bar0, volatile int* s_abort)
+                                               uint32_t b0, uint32_t bar0, volatile int* s_abort, int n_cols = BN)
 {
-    constexpr uint32_t idesc = make_idesc(2, 1, BM, BN);
+    const uint32_t idesc = make_idesc(2, 1, BM, static_cast<uint32_t>(n_cols));
     static_assert(L::AS >= 2 && L::ES >= 2, "a step of two must stay inside one lap of a ring");
     if (first >= nkb) return true;
     const uint32_t q0 = seq0 + static_cast<uint32_t>(first);
@@ -564,7 +568,10 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM;
+    // width of this launch's tiles: narrower than the template's 128 (96, 64 or 32) when that puts more CTAs on
+    // the SMs in one wave; shared-memory slots and the accumulator keep the template's size
+    const int bn = (BN == 128 && p.tile_n > 0) ? p.tile_n : BN;
+    const int n0 = blockIdx.x * bn, m0 = blockIdx.y * BM;
     // the CTAs of a cluster (gridDim.z of them) share one output tile and split the reduction
     const int splits = gridDim.z, rank = blockIdx.z;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * rank) / splits);
@@ -610,13 +617,13 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     } else if (warp == L::B_WARP) {
         // ------------------------------------------------------------ weight-tile producer
         if (lane == 0)
-            produce_b_tile<BN, W4, L>(&tmap_w, p, 0, kb_begin, nkb, n0, smem_u32(W4 ? sP : sB), bar0, s_abort);
+            produce_b_tile<BN, W4, L>(&tmap_w, p, 0, kb_begin, nkb, n0, smem_u32(W4 ? sP : sB), bar0, s_abort, bn);
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const bool ok = issue_k_blocks<BN, W4, L>(0, dual ? 2 : 1, nkb, tmem_base, 0, smem_u32(sA), smem_u32(sB), bar0,
-                                                      s_abort);
+                                                      s_abort, bn);
             if (ok) tc_commit(bar_accum);
         }
         __syncwarp();
@@ -627,7 +634,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             // stored BOS rows
             const float sx = p.act_scale ? __ldg(p.act_scale) : 0.f;  // absent: accumulators only
             const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
-            for (int j = tid - 64; j < BN; j += 128) {
+            for (int j = tid - 64; j < bn; j += 128) {
                 const int n = n0 + j;
                 float comb = 0.f, b = 0.f;
                 if (n < p.N && p.w_scale) {
@@ -643,14 +650,14 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 // row 0 of every prompt: the stored floating-point BOS projection, copied as is
                 for (int idx = tid - 64; idx < p.batch * BN; idx += 128) {
                     const int b = idx / BN, j = idx - b * BN;
-                    if (n0 + j < p.N)
+                    if (j < bn && n0 + j < p.N)
                         p.Y[static_cast<long long>(b) * MIXDQ_TOKENS_PER_PROMPT * p.ldy + n0 + j] = p.bos_out[n0 + j];
                 }
             }
         } else if (W4) {
             // -------------------------------------------------------- int4 -> int8 (x16) expansion
             const int group = (warp - 6) >> 1;  // warps 6-7, 8-9, 10-11, 12-13
-            expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, nkb, sB, sP, bar0, s_abort);
+            expand_nibbles<BN, L>(group, tid - 192 - group * 64, lane, nkb, sB, sP, bar0, s_abort, bn);
             pdl_wait();  // before these warps help with the epilogue
         }
         if (warp < 10 && !direct) {
@@ -693,7 +700,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         // ------------------------------------------------------------ second MMA issuer: odd k-blocks
         if (lane == 0 && dual) {
             const bool ok = issue_k_blocks<BN, W4, L>(1, 2, nkb, tmem_base + BN, 0, smem_u32(sA), smem_u32(sB), bar0,
-                                                      s_abort);
+                                                      s_abort, bn);
             if (ok) tc_commit(bar_accum);
         }
     }
@@ -707,8 +714,9 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         asm volatile("bar.sync 1, %0;" ::"n"(L::THREADS) : "memory");  // the factor tables are complete
         bool ok = mbar_wait(bar_accum, 0, s_abort);
         tc_fence_after_sync();
-        if (__all_sync(0xffffffffu, ok && !*s_abort)) {
-            constexpr int COLS = BN / (L::EPI_WARPS / 4);
+        constexpr int COLS = BN / (L::EPI_WARPS / 4);
+        // (a column group past the tile's width has nothing to store)
+        if (__all_sync(0xffffffffu, ok && !*s_abort) && (warp >> 2) * COLS < bn) {
             const int lg = warp & 3;
             const int cbeg = (warp >> 2) * COLS;
             const uint32_t acc = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + cbeg;
@@ -745,7 +753,7 @@ tma_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (n + 2 < p.N) cl.z = sl * __ldg(p.w_scale + n + 2);
             if (n + 3 < p.N) cl.w = sl * __ldg(p.w_scale + n + 3);
         }
-        if (n < p.N && tid < L::WORK_THREADS) {
+        if (n < p.N && chunk * 4 < bn && tid < L::WORK_THREADS) {
 #pragma unroll 2
             for (int rl = tid / CHUNKS; rl < rows_per; rl += RSTEP) {
                 const int row = rank * rows_per + rl;
@@ -1114,7 +1122,8 @@ int launch_tma(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& 
     using L = TmaSmem<BN, STAGES, W4>;
     auto kernel = tma_gemm_kernel<BN, STAGES, W4, ADD>;
     if (ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), L::TOTAL) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
-    const dim3 grid(static_cast<unsigned>(ceil_div(tp.N, BN)), static_cast<unsigned>(ceil_div(tp.M, BM)),
+    const int bn = (BN == 128 && tp.tile_n > 0) ? tp.tile_n : BN;
+    const dim3 grid(static_cast<unsigned>(ceil_div(tp.N, bn)), static_cast<unsigned>(ceil_div(tp.M, BM)),
                     static_cast<unsigned>(splits));
     return launch_pdl(kernel, grid, dim3(L::THREADS), L::TOTAL, stream, static_cast<unsigned>(splits), ta, tw, ty, tp);
 }
@@ -1169,6 +1178,20 @@ int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms)
         }
     }
     return best < 1.05 * old ? best_bn : 0;
+}
+
+// Width of the one-tile kernel's tiles for a layer the single-CTA kernels run on 128-wide slots: 128, or 96 / 64
+// when that raises the number of CTAs while they still fit the SMs in one wave and the reduction is not split.
+int plan_narrow_tile(int M, int N, int k_blocks, int num_sms)
+{
+    const int64_t row_tiles = ceil_div(M, BM);
+    const int64_t t128 = row_tiles * ceil_div(N, 128);
+    if (t128 >= num_sms || pick_splits(t128, k_blocks, num_sms) != 1) return 128;
+    for (int cand : {64, 96}) {
+        const int64_t t = row_tiles * ceil_div(N, cand);
+        if (t < num_sms && t > t128) return cand;
+    }
+    return 128;
 }
 
 size_t tma_scratch_bytes(int64_t in_rows, int64_t K_row) { return static_cast<size_t>(round_up(in_rows * K_row, 256)); }
@@ -1310,7 +1333,15 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
     // (W4 runs on 128-wide tiles only: its packed ring needs the room, and it measured no slower)
     const bool wide = !w4 && !p.addend && (p.N >= 1024 || p.N % 256 == 0) && ceil_div(p.M, BM) * ceil_div(p.N, 256) >= 100;
-    const uint32_t bn = wide ? 256 : 128;
+    uint32_t bn = wide ? 256 : 128;
+    // Tile-count quantization of the one-tile kernel: a layer whose 128-wide tiles number between half the SMs
+    // and all of them (1024 x 1280 outputs: 80 tiles on 148 SMs) leaves SMs idle and cannot split its reduction
+    // either.  Narrower tiles (96 or 64 columns, multiples of the 32-column epilogue pass) in the same 128-wide
+    // slots put more CTAs on the machine in one wave, each with proportionally less MMA, expansion and epilogue work.
+    if (!wide && !p.addend) {
+        bn = static_cast<uint32_t>(plan_narrow_tile(p.M, p.N, tp.k_blocks, num_sms));
+        if (bn != 128) tp.tile_n = static_cast<int>(bn);
+    }
     if (w4)
         rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, bn, false);
     else
