@@ -381,9 +381,10 @@ def config_records(torch, mixdq, synth, stream, peaks, probe_int8):
         bd = None if b is None else dev(b)
         us = _time_graph(torch, stream, lambda: mixdq.linear(Xd, pk, N, bits, s, None, 8, sx, bd, ws, status, out=Y))
         tops = 2.0 * M * N * K / us / 1e6
-        rows, cols = mixdq.int8_tile_plan(M, N, (K + 127) // 128, bits)
+        rows, cols, sp = mixdq.int8_tile_plan(M, N, (K + 127) // 128, bits, with_splits=True)
         out.append({"config": tag, "M": M, "N": N, "K": K, "w_bits": bits, "a_bits": 8, "us": round(us, 2),
-                    "tops": round(tops, 1), "bound": "tensor", "l2": "warm", "tile": f"{rows}x{cols}",
+                    "tops": round(tops, 1), "bound": "tensor", "l2": "warm",
+                    "tile": f"{rows}x{cols}" + (f", reduction over {sp} CTA pairs" if sp > 1 else ""),
                     "frac": _fracs(tops, int8_peak, NOMINAL["int8_tops"], probe_int8)})
 
     # 1. single linear layer, W8A8
@@ -699,9 +700,11 @@ def run_ours(args):
             us = t0.elapsed_time(t1) * 1e3 / (reps * rounds)
             tops = pl.spec.ops(args.batch) / us / 1e6
             kb = 9 * ((pl.spec.Cin + 127) // 128) if pl.spec.kind == "conv3x3" else (pl.spec.K + 127) // 128
-            rows, cols = mixdq.int8_tile_plan(pl.spec.rows(args.batch), pl.spec.N, kb, pl.spec.w_bits)
+            rows, cols, sp = mixdq.int8_tile_plan(pl.spec.rows(args.batch), pl.spec.N, kb, pl.spec.w_bits, with_splits=True)
             per_layer.append({"layer": name, "kind": pl.spec.kind, "M": pl.spec.rows(args.batch), "N": pl.spec.N,
-                              "K": pl.spec.K, "w_bits": pl.spec.w_bits, "tile": f"{rows}x{cols}", "us": round(us, 2),
+                              "K": pl.spec.K, "w_bits": pl.spec.w_bits,
+                              "tile": f"{rows}x{cols}" + (f", reduction over {sp} CTA pairs" if sp > 1 else ""),
+                              "us": round(us, 2),
                               "tops": round(tops, 1), "frac_of_burst_peak": round(tops / burst, 3),
                               "frac_of_sustained_peak": round(tops / (peaks["bf16_tflops_sustained"] * INT8_TO_BF16_NOMINAL), 3),
                               "frac_of_int8_mma_probe": round(tops / probe_int8, 3),

@@ -61,8 +61,12 @@ unsigned long long mixdq_kernel_launches(void);
  * reduction blocks of 128 (linear layer: ceil(K / 128); 3x3 convolution: 9 * ceil(Cin / 128)).
  * *tile_rows x *tile_cols (HOST pointers) is 256 x {160, 192, 224, 256} when two CTAs on neighbouring SMs
  * share a tile (tcgen05 cta_group::2), else 128 x {64, 96, 128, 256}.  The BOS-aware projection and the second branch
- * of a shortcut-split layer always run on 128-row tiles.  For tests and benchmarks: nothing is launched. */
-int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols);
+ * of a shortcut-split layer always run on 128-row tiles.  *reduction_splits (HOST): for 256-row tiles the number
+ * of CTA pairs that share one tile's reduction (1: each pair walks whole tiles; 2 to 4: layers with few tiles and
+ * a long reduction, partial sums added through distributed shared memory); 0 for 128-row tiles.  For tests and
+ * benchmarks: nothing is launched. */
+int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols,
+                         int* reduction_splits);
 
 /* Static, NUL-terminated description of an error code (host pointer, never NULL). */
 const char* mixdq_strerror(int code);

@@ -179,19 +179,24 @@ extern "C" unsigned long long mixdq_kernel_launches(void)
     return g_layer_kernel_launches.load(std::memory_order_relaxed);
 }
 
-extern "C" int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols)
+extern "C" int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols,
+                                    int* reduction_splits)
 {
-    if (!tile_rows || !tile_cols || M <= 0 || N <= 0 || k_blocks <= 0 || M > 0x7fffffff || N > 0x7fffffff ||
+    if (!tile_rows || !tile_cols || !reduction_splits || M <= 0 || N <= 0 || k_blocks <= 0 || M > 0x7fffffff || N > 0x7fffffff ||
         k_blocks > 0x7fffffff)
         return MIXDQ_ERR_INVALID_ARG;
     if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
     const int sms = sm_count();
     if (sms <= 0) return MIXDQ_ERR_CUDA;
-    const int bn = i8::plan_pair_tile(static_cast<int>(M), static_cast<int>(N), static_cast<int>(k_blocks), w_bits == 4, sms);
+    int splits = 1;
+    const int bn = i8::plan_pair_tile(static_cast<int>(M), static_cast<int>(N), static_cast<int>(k_blocks), w_bits == 4, sms,
+                                      &splits);
     if (bn > 0) {
         *tile_rows = 256;
         *tile_cols = bn;
+        *reduction_splits = splits;
     } else {
+        *reduction_splits = 0;  // (decided at launch: a cluster of up to eight CTAs when the tiles are few)
         const bool wide = w_bits == 8 && (N >= 1024 || N % 256 == 0) && ceil_div(M, 128) * ceil_div(N, 256) >= 100;
         *tile_rows = 128;
         *tile_cols = wide ? 256 : i8::plan_narrow_tile(static_cast<int>(M), static_cast<int>(N), static_cast<int>(k_blocks), sms);

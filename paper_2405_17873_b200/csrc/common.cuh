@@ -82,8 +82,21 @@ int sm_count();
 // (barrier init, tensor-memory allocation, descriptor prefetch) overlaps that tail.  Every
 // kernel launched this way calls pdl_wait() before it touches global memory.
 template <typename... KArgs, typename... Args>
+inline int launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              unsigned cluster_x, unsigned cluster_z, Args&&... args);
+
+template <typename... KArgs, typename... Args>
 inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                       unsigned cluster_z, Args&&... args)
+{
+    return launch_pdl_cluster(kernel, grid, block, smem, stream, 1u, cluster_z, static_cast<Args&&>(args)...);
+}
+
+// The same with a cluster of cluster_x x 1 x cluster_z CTAs (kernels whose CTA pairs share tensor-core
+// instructions need their pairs adjacent along x).
+template <typename... KArgs, typename... Args>
+inline int launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              unsigned cluster_x, unsigned cluster_z, Args&&... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -94,11 +107,11 @@ inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.x = cluster_x;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = cluster_z;
     cfg.attrs = attr;
-    cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    cfg.numAttrs = (cluster_z > 1 || cluster_x > 1) ? 2 : 1;
     if (prefer_max_shared_carveout(reinterpret_cast<const void*>(kernel)) != MIXDQ_OK) return MIXDQ_ERR_CUDA;
     g_layer_kernel_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);

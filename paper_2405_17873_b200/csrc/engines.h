@@ -58,8 +58,9 @@ int run(Params p, int amode, const void* packed, int w_bits, void* workspace, si
 bool tma_path_ok(const Params& p, int amode, int w_bits);
 int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream);
 // Tile width of the pair form (two-CTA tiles of 256 x width) when the planner prefers it for an int8 GEMM of
-// M x N over k_blocks k-blocks of 128, else 0 (the single-CTA kernels run).
-int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms);
+// M x N over k_blocks k-blocks of 128, else 0 (the single-CTA kernels run).  *splits (optional): how many CTA
+// pairs share one tile's reduction (1: persistent pairs; without the pointer only that form is considered).
+int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits = nullptr);
 // Tile width (128, 96 or 64) of the one-tile kernel on 128-wide slots.
 int plan_narrow_tile(int M, int N, int k_blocks, int num_sms);
 // The two steps as calls of their own, for activations that are stored as int8 between layers: the codes of

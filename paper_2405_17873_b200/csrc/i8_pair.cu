@@ -21,6 +21,8 @@
 //
 // BN is a run-time value (a multiple of 32 up to 256) chosen per layer so that the tiles fill whole rounds of
 // the SM pairs; shared-memory slots have the size of the widest tile.
+#include <mutex>
+
 #include "i8_tiles.cuh"
 
 namespace mixdq {
@@ -103,10 +105,9 @@ __device__ __forceinline__ void mma_pair(uint32_t d_tmem, uint64_t a_desc, uint6
 }
 
 // Once every MMA this thread issued so far has completed: arrive on the barrier at this shared-memory offset
-// in both CTAs of the pair.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+// in both CTAs of the pair (`both`: their bits in the cluster's CTA mask).
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t both)
 {
-    const uint16_t both = 3;
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
                  "h"(both)
                  : "memory");
@@ -197,10 +198,16 @@ struct PairArgs {
     int bn;           // tile width (multiple of 32, <= 256); each CTA holds bn / 2 weight rows
     int n_tiles;      // tiles along N
     int total_tiles;  // pair tiles in all
+    int splits;       // > 1: one tile per cluster of 2 * splits CTAs, the reduction split over its CTA pairs
 };
 
+// Grid (2 * splits * (pairs or tiles), 1, 1) with clusters of 2 * splits CTAs along x: CTAs 2 i and 2 i + 1 of a
+// cluster are an MMA pair (a cluster of this kernel must be even along x: the launch is refused otherwise).  splits == 1: the pairs walk the tiles persistently.  splits > 1 (layers with too few tiles to fill
+// the machine): one tile per cluster, pair i takes the i-th share of the reduction, every CTA leaves its 128 x bn
+// partial sums in shared memory, and after a cluster barrier each CTA adds up its share of the rows over the
+// pairs through distributed shared memory (integer adds: exact and order-free), dequantizes and stores.
 template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairSmem<MODE>::THREADS, 1)
+__global__ void __launch_bounds__(PairSmem<MODE>::THREADS, 1)
 pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, const PairArgs g)
 {
@@ -220,17 +227,24 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t rank = cluster_ctarank();  // 0: leader
+    const uint32_t crank = cluster_ctarank();  // rank in the cluster: pair crank / 2, CTA crank % 2 of the pair
+    const uint32_t rank = crank & 1u;          // 0: the pair's leader
+    const uint32_t leader_rank = crank & ~1u;
     const bool leader = rank == 0;
-    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int nkb = p.k_blocks;
+    const int splits = g.splits, slice = static_cast<int>(crank >> 1);
+    // (non-split: index of this pair and number of pairs; split: index of this cluster's tile)
+    const int pair = static_cast<int>(blockIdx.x) / (2 * splits), npairs = static_cast<int>(gridDim.x) / (2 * splits);
+    // this pair's share of the reduction (all of it unless the tile is split over the cluster)
+    const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * slice) / splits);
+    const int nkb = static_cast<int>((static_cast<long long>(p.k_blocks) * (slice + 1)) / splits) - kb_begin;
     const int bn = g.bn, bh = g.bn >> 1;
-    const int my_tiles = (g.total_tiles - pair + npairs - 1) / npairs;
+    const int my_tiles = splits > 1 ? 1 : (g.total_tiles - pair + npairs - 1) / npairs;
+    const uint16_t pair_mask = static_cast<uint16_t>(3u << leader_rank);  // the two CTAs of this pair
 
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t a0 = smem_u32(smem + L::OFF_A), b0 = smem_u32(sB), p0 = smem_u32(smem + L::OFF_P);
     // the same barriers as seen in the leader CTA (for the leader: its own)
-    const uint32_t lead_bar0 = map_to_cta(bar0, 0);
+    const uint32_t lead_bar0 = map_to_cta(bar0, leader_rank);
 
     pdl_launch_dependents();
     if (tid == 0) {
@@ -281,12 +295,16 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = pair + t * npairs;
                 const int m0 = (tile / g.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM;
-                int img_b = 0, ho0 = 0, wo0 = 0, cb = 0, kh = 0, kw = 0, xa = 0;
+                int img_b = 0, ho0 = 0, wo0 = 0, cb = 0, kh = 0, kw = 0, xa = kb_begin * BKE;
                 if (p.conv) {
                     img_b = m0 / p.HoWo;
                     const int rem = m0 - img_b * p.HoWo;
                     ho0 = rem / p.Wo;
                     wo0 = rem - ho0 * p.Wo;
+                    const int tap = kb_begin / p.cblocks;
+                    cb = kb_begin - tap * p.cblocks;
+                    kh = tap / 3;
+                    kw = tap - 3 * kh;
                 }
                 for (int i = 0; i < nkb; ++i) {
                     if (!mbar_wait(bar0 + 8 * (L::EMPTY_A + s), par, s_abort)) {
@@ -328,7 +346,12 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int tile = pair + t * npairs;
                 const int n0 = (tile % g.n_tiles) * bn + static_cast<int>(rank) * bh;
-                int cb = 0, kx_tap = 0, xb = 0;
+                int cb = 0, kx_tap = 0, xb = kb_begin * ROW_STEP;
+                if (p.conv) {
+                    const int tap = kb_begin / p.cblocks;
+                    cb = kb_begin - tap * p.cblocks;
+                    kx_tap = tap * p.Cin;  // first reduction index of the filter tap
+                }
                 for (int i = 0; i < nkb; ++i) {
                     // W8: the commit that frees the activation slot frees the weight slot (the rings move in lockstep)
                     if (!mbar_wait(bar0 + 8 * ((W4 ? L::EMPTY_P : L::EMPTY_A) + s), par, s_abort)) {
@@ -411,8 +434,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         tc_fence_before_sync();
                         mbar_arrive(tile_go);
                     }
-                    tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa));
-                    if (W4) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se));
+                    tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa), pair_mask);
+                    if (W4) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
                     sa += 2;
                     if (sa >= static_cast<uint32_t>(L::AS)) {
                         sa -= L::AS;
@@ -425,7 +448,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 }
                 // (a thread without a k-block in this tile still arrives: its commit has nothing to wait for)
-                if (ok) tc_commit_pair(bar0 + 8 * (L::ACC_FULL + buf));
+                if (ok) tc_commit_pair(bar0 + 8 * (L::ACC_FULL + buf), pair_mask);
             }
         }
         __syncwarp();
@@ -483,7 +506,23 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 continue;
             }
             const uint32_t acc = tmem_base + buf * ACC_COLS + (static_cast<uint32_t>(lg * 32) << 16);
-            if (!F16 && p.acc_out) {
+            if (splits > 1) {
+                // this pair's share of the sums: tensor memory -> registers -> shared memory (the drained pipeline
+                // buffers), rows bn * 4 bytes apart, 16-byte chunks XOR-swizzled by row; reduced below
+                const int row = lg * 32 + lane;
+                uint8_t* prow = smem + row * (bn * 4);
+                for (int c0 = c_begin; c0 < c_begin + c_count; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc + c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int chunk = (c0 >> 2) + j;
+                        *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) =
+                            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    }
+                }
+            } else if (!F16 && p.acc_out) {
                 // raw int32 sums (parity hook): a lane owns a row, 32 columns of it at a time
                 const int m = m0 + lg * 32 + lane;
                 for (int c0 = c_begin; c0 < c_begin + c_count; c0 += 32) {
@@ -504,7 +543,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                 }
             }
-            if (p.Y && c_count > 0) {
+            if (splits == 1 && p.Y && c_count > 0) {
                 if (F16)
                     store_rows32_f32(acc + c_begin, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
                                      m0 + lg * 32, n0 + c_begin, lane);
@@ -573,6 +612,76 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     }
 
+    if (splits > 1) {
+        // ------------------------------------------------------------ reduction over the pairs of the cluster
+        // CTA (pair `slice`, rank r) adds up rows [slice * ceil(128 / splits), ...) of the rank-r halves of all
+        // pairs; consecutive threads take consecutive groups of four columns, so stores coalesce.
+        __syncthreads();
+        cluster_sync();
+        if (!*s_abort) {
+            const int tile = pair;
+            const int m_base = (tile / g.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM, n0 = (tile % g.n_tiles) * bn;
+            const int rows_per = (BM + splits - 1) / splits;
+            const int r0 = slice * rows_per;
+            const int r1 = r0 + rows_per < BM ? r0 + rows_per : BM;
+            const int chunks = bn >> 2;
+            const float* comb = s_comb;  // accumulator 0's tables
+            const float* bias = s_bias;
+            const int zshift = p.act_zero ? 128 - __ldg(p.act_zero) : 0;
+            const uint32_t base = smem_u32(smem);
+            for (int idx = tid; idx < (r1 - r0) * chunks; idx += L::THREADS) {
+                const int row = r0 + idx / chunks, chunk = idx % chunks;
+                const int m = m_base + row, n = n0 + chunk * 4;
+                if (m >= p.M || n >= p.N) continue;
+                const uint32_t off = base + row * (bn * 4) + ((chunk ^ (row & 7)) << 4);
+                int4 acc = make_int4(0, 0, 0, 0);
+                float4 facc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int q = 0; q < splits; ++q) {
+                    uint32_t remote;
+                    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(off), "r"(2 * q + static_cast<int>(rank)));
+                    int4 v;
+                    asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                 : "r"(remote));
+                    if (F16) {
+                        facc.x += __int_as_float(v.x);
+                        facc.y += __int_as_float(v.y);
+                        facc.z += __int_as_float(v.z);
+                        facc.w += __int_as_float(v.w);
+                    } else {
+                        acc.x += v.x;
+                        acc.y += v.y;
+                        acc.z += v.z;
+                        acc.w += v.w;
+                    }
+                }
+                const int a[4] = {acc.x, acc.y, acc.z, acc.w};
+                const float f[4] = {facc.x, facc.y, facc.z, facc.w};
+                if (!F16 && p.acc_out) {
+                    int32_t* dst = p.acc_out + static_cast<long long>(m) * p.N + n;
+                    for (int j = 0; j < 4; ++j)
+                        if (n + j < p.N)
+                            dst[j] = (W4 ? (a[j] >> 4) : a[j]) + (p.act_zero ? zshift * __ldg(p.w_code_sums + n + j) : 0);
+                }
+                if (p.Y) {
+                    __half h[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float v = F16 ? f[j] : acc_to_float<W4, false>(static_cast<uint32_t>(a[j]));
+                        h[j] = __float2half_rn(fmaf(v, comb[chunk * 4 + j], bias[chunk * 4 + j]));
+                    }
+                    __half* dst = p.Y + static_cast<long long>(m) * p.ldy + n;
+                    if ((p.ldy & 3) == 0 && n + 4 <= p.N) {
+                        *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h);
+                    } else {
+                        for (int j = 0; j < 4; ++j)
+                            if (n + j < p.N) dst[j] = h[j];
+                    }
+                }
+            }
+        }
+    }
+
     if (*s_abort) {
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
         if (tid == 0 && p.status) atomicExch(p.status, MIXDQ_ERR_TIMEOUT);
@@ -586,7 +695,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 }
 
 template <int MODE>
-int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn, int splits,
                   int num_sms, cudaStream_t stream)
 {
     using L = PairSmem<MODE>;
@@ -596,27 +705,66 @@ int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMa
     g.bn = bn;
     g.n_tiles = static_cast<int>(ceil_div(tp.N, bn));
     g.total_tiles = g.n_tiles * static_cast<int>(ceil_div(tp.M, 2 * BM));
-    const int pairs = g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2;
-    // (the cluster shape is part of the kernel: __cluster_dims__)
-    return launch_pdl(kernel, dim3(static_cast<unsigned>(2 * pairs)), dim3(L::THREADS), L::TOTAL, stream, 1, ta, tw, ty, tp,
-                      g);
+    g.splits = splits;
+    // persistent pairs, or one cluster of `splits` pairs per tile
+    const int pairs = splits > 1 ? g.total_tiles : (g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2);
+    return launch_pdl_cluster(kernel, dim3(static_cast<unsigned>(2 * splits * pairs)), dim3(L::THREADS), L::TOTAL, stream,
+                              static_cast<unsigned>(2 * splits), 1u, ta, tw, ty, tp, g);
 }
 
 }  // namespace
 
-int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
-                int num_sms, cudaStream_t stream)
+// How many clusters of `cluster_ctas` CTAs of the pair kernel the device holds at once (a cluster lives inside one
+// GPC, so this is well below SMs / cluster_ctas for the larger clusters); asked of the occupancy calculator once per
+// device, width and cluster size.  0 on error.
+int pair_cluster_capacity(bool w4, int cluster_ctas)
 {
-    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2) return MIXDQ_ERR_INVALID_ARG;
-    return w4 ? launch_pair_t<1>(ta, tw, ty, tp, bn, num_sms, stream)
-              : launch_pair_t<0>(ta, tw, ty, tp, bn, num_sms, stream);
+    static std::mutex mu;
+    static int cache[64][2][9] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || cluster_ctas < 2 || cluster_ctas > 8) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    int& slot = cache[dev][w4 ? 1 : 0][cluster_ctas];
+    if (slot == 0) {
+        const void* kernel = w4 ? reinterpret_cast<const void*>(pair_gemm_kernel<1>) : reinterpret_cast<const void*>(pair_gemm_kernel<0>);
+        const int smem = w4 ? PairSmem<1>::TOTAL : PairSmem<0>::TOTAL;
+        const int threads = w4 ? PairSmem<1>::THREADS : PairSmem<0>::THREADS;
+        if (ensure_dynamic_smem(kernel, smem) != MIXDQ_OK) return 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(cluster_ctas) * 64);
+        cfg.blockDim = dim3(static_cast<unsigned>(threads));
+        cfg.dynamicSmemBytes = static_cast<size_t>(smem);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = static_cast<unsigned>(cluster_ctas);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return 0;
+        }
+        slot = n > 0 ? n : -1;
+    }
+    return slot > 0 ? slot : 0;
+}
+
+int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
+                int splits, int num_sms, cudaStream_t stream)
+{
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || splits < 1 || splits > 4 || splits > tp.k_blocks)
+        return MIXDQ_ERR_INVALID_ARG;
+    return w4 ? launch_pair_t<1>(ta, tw, ty, tp, bn, splits, num_sms, stream)
+              : launch_pair_t<0>(ta, tw, ty, tp, bn, splits, num_sms, stream);
 }
 
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
                     int num_sms, cudaStream_t stream)
 {
     if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || tp.acc_out) return MIXDQ_ERR_INVALID_ARG;
-    return launch_pair_t<2>(ta, tw, ty, tp, bn, num_sms, stream);
+    return launch_pair_t<2>(ta, tw, ty, tp, bn, 1, num_sms, stream);
 }
 
 }  // namespace i8

@@ -180,8 +180,11 @@ __device__ __forceinline__ void store_rows32_f32(uint32_t acc, int ncols, const 
 
 // Pair form (i8_pair.cu): persistent kernel of two-CTA clusters on 256 x bn tiles.  ta: activation map with a
 // box of 128 rows (or pixels), tw: weight map with a box of bn / 2 rows, ty: output map with a 32 x 32 box.
+// splits > 1: one tile per cluster of `splits` CTA pairs, each pair taking a share of the reduction (<= 4).
 int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
-                int num_sms, cudaStream_t stream);
+                int splits, int num_sms, cudaStream_t stream);
+// Clusters of `cluster_ctas` CTAs of that kernel the current device can hold at once (0 on error).
+int pair_cluster_capacity(bool w4, int cluster_ctas);
 // The same kernel on fp16 operands (kind::f16, fp32 accumulators) for the weight-only layers: ta an fp16 map with a
 // box of 128 rows x 64 elements, tw the map of the layer's weights expanded to fp16 (q - zero) with a box of
 // bn / 2 rows x 64 elements; tp.k_blocks counts blocks of 64 elements and tp.act_scale is unused.

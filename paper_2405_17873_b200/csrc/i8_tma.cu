@@ -1143,21 +1143,36 @@ int pick_splits(int64_t tiles, int k_blocks, int num_sms)
 // fitted to timings of every layer shape of the SDXL-turbo-shaped UNet at image batch 1 and 4 on a B200 (each
 // form at each width): rounds of tiles over the SMs (or SM pairs) times the cost of a tile -- the larger of its
 // main loop, a per-k-block cost that grows with the tile width, and its epilogue -- plus fixed costs.
-int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms)
+int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits)
 {
+    if (splits) *splits = 1;
     if (M < 2 * BM || num_sms < 2) return 0;
     const double nkb = k_blocks;
+    const int pairs = num_sms / 2;
     // pair form: 256 x bn tiles, widths below 160 never paid off
     double best = 0;
-    int best_bn = 0;
+    int best_bn = 0, best_splits = 1;
     for (int bn = 160; bn <= 256; bn += 32) {
-        const double tiles = static_cast<double>(ceil_div(M, 2 * BM) * ceil_div(N, bn));
-        const double rounds = std::ceil(tiles / (num_sms / 2));
+        const int64_t tiles = ceil_div(M, 2 * BM) * ceil_div(N, bn);
         const double per_kb = w4 ? 350.0 + 1.4 * bn : 250.0 + 1.2 * bn;
+        const double rounds = std::ceil(static_cast<double>(tiles) / pairs);
         const double t = rounds * (std::max(nkb * per_kb, 30.0 * bn) + 800.0) + 16.0 * bn + 5000.0;
         if (best_bn == 0 || t < best) {
             best = t;
             best_bn = bn;
+            best_splits = 1;
+        }
+        // few tiles, long reduction: one tile per cluster, the reduction split over up to four pairs; the
+        // partial tiles meet through distributed shared memory at a fixed cost of some 14 000 cycles
+        // (a cluster sits inside one GPC: the device holds fewer clusters of 4, 6 or 8 CTAs than SMs / size)
+        for (int sp = 2; sp <= 4 && splits && tiles * sp <= pairs && k_blocks / sp >= 8; ++sp) {
+            if (tiles > pair_cluster_capacity(w4, 2 * sp)) continue;
+            const double ts = std::ceil(nkb / sp) * per_kb + 16.0 * bn + 14000.0 + 5000.0;
+            if (ts < best) {
+                best = ts;
+                best_bn = bn;
+                best_splits = sp;
+            }
         }
     }
     // single-CTA kernels: 128 x 128 tiles (128 x 256 for wide int8 layers), persistent once the tiles cover the
@@ -1177,7 +1192,9 @@ int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms)
             old = std::ceil(nkb / s) * c + 3000.0 + 3000.0 + (s > 1 ? 2500.0 : 0.0);
         }
     }
-    return best < 1.05 * old ? best_bn : 0;
+    if (best >= 1.05 * old) return 0;
+    if (splits) *splits = best_splits;
+    return best_bn;
 }
 
 // Width of the one-tile kernel's tiles for a layer the single-CTA kernels run on 128-wide slots: 128, or 96 / 64
@@ -1316,7 +1333,9 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
     const int num_sms = sm_count();
     if (num_sms <= 0) return MIXDQ_ERR_CUDA;
     // the pair form (two-CTA tiles of 256 x bn, i8_pair.cu) where its estimate beats the single-CTA kernels
-    const int pair_bn = (!p.addend && amode != A_BOS && !p.test_drop_b_kblock) ? plan_pair_tile(p.M, p.N, tp.k_blocks, w4, num_sms) : 0;
+    int pair_splits = 1;
+    const int pair_bn = (!p.addend && amode != A_BOS && !p.test_drop_b_kblock)
+                            ? plan_pair_tile(p.M, p.N, tp.k_blocks, w4, num_sms, &pair_splits) : 0;
     if (pair_bn > 0) {
         if (w4)
             rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, pair_bn / 2, false);
@@ -1328,7 +1347,7 @@ static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bi
                                     static_cast<uint64_t>(p.ldy), 32, 32, true);
             if (rc != MIXDQ_OK) return rc;
         }
-        return launch_pair(ta, tw, ty, tp, w4, pair_bn, num_sms, stream);
+        return launch_pair(ta, tw, ty, tp, w4, pair_bn, pair_splits, num_sms, stream);
     }
     // 256-wide tiles halve the A traffic per output but need enough tiles to cover the SMs
     // (W4 runs on 128-wide tiles only: its packed ring needs the room, and it measured no slower)

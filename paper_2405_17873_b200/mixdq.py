@@ -25,7 +25,7 @@ _SIGNATURES = {
     "mixdq_version": (C.c_int, []),
     "mixdq_strerror": (C.c_char_p, [_int]),
     "mixdq_kernel_launches": (C.c_ulonglong, []),
-    "mixdq_int8_tile_plan": (_int, [_i64, _i64, _i64, _int, C.POINTER(_int), C.POINTER(_int)]),
+    "mixdq_int8_tile_plan": (_int, [_i64, _i64, _i64, _int, C.POINTER(_int), C.POINTER(_int), C.POINTER(_int)]),
     "mixdq_packed_bytes": (_int, [_i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_weight_minmax_params": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp, _vp]),
     "mixdq_pack_weights": (_int, [_vp, _i64, _i64, _int, _vp, _vp, _int, _vp, _vp]),
@@ -124,11 +124,11 @@ def kernel_launches() -> int:
     return int(lib().mixdq_kernel_launches())
 
 
-def int8_tile_plan(M: int, N: int, k_blocks: int, w_bits: int):
-    """(tile_rows, tile_cols) of the int8 tensor-core GEMM for this shape on the current device."""
-    r, c = _int(0), _int(0)
-    _chk(lib().mixdq_int8_tile_plan(M, N, k_blocks, w_bits, C.byref(r), C.byref(c)), "mixdq_int8_tile_plan")
-    return r.value, c.value
+def int8_tile_plan(M: int, N: int, k_blocks: int, w_bits: int, with_splits: bool = False):
+    """(tile_rows, tile_cols[, reduction_splits]) of the int8 tensor-core GEMM for this shape on the current device."""
+    r, c, sp = _int(0), _int(0), _int(0)
+    _chk(lib().mixdq_int8_tile_plan(M, N, k_blocks, w_bits, C.byref(r), C.byref(c), C.byref(sp)), "mixdq_int8_tile_plan")
+    return (r.value, c.value, sp.value) if with_splits else (r.value, c.value)
 
 
 def packed_bytes(N: int, K: int, bits: int, layout: int = LAYOUT_DEVICE) -> int:

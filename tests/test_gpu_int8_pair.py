@@ -123,6 +123,66 @@ def test_asymmetric_activations_on_pair_tiles(bits):
     assert_close(host(yc), yc_ref)
 
 
+# few tiles, long reduction: one tile per cluster of two to four CTA pairs, partial sums added through distributed
+# shared memory (ragged rows, columns and reduction; linear and convolution, stride 1 and 2)
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,N,K", [(1000, 1184, 6160), (1024, 1280, 11520), (1000, 1270, 11536), (1024, 640, 17280)])
+def test_linear_on_split_pair_tiles(bits, M, N, K):
+    rows, cols, splits = mixdq.int8_tile_plan(M, N, _kblocks(K), bits, with_splits=True)
+    if not (rows == 256 and splits >= 2):
+        # (the choice depends on the width and on how many clusters the device holds; the 1024 x 1280 x 11520 case is
+        # checked below to split at both widths)
+        pytest.skip(f"the planner runs this shape on {rows} x {cols} tiles without a split reduction")
+    X = synth.normal_f16((M, K), 1.0, seed=M + K)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 1)
+    b = synth.normal_f16((N,), 0.01, seed=N)
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.linear_a8(X, codes, s_ref, sx_ref, b)
+    Xd = dev(X)
+    s, _, packed = device_weights(W, bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    ws = workspace_for(M, N, K, bits)
+    acc = mixdq.linear_acc_i32(Xd, packed, N, bits, sx, workspace=ws, status=st)
+    y = mixdq.linear(Xd, packed, N, bits, s, None, 8, sx, dev(b), workspace=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,Cin,Cout,stride", [(4, 16, 1280, 1280, 1), (4, 16, 1920, 1280, 1), (4, 32, 1280, 1280, 2)])
+def test_conv3x3_on_split_pair_tiles(bits, B, H, Cin, Cout, stride):
+    Ho = (H - 1) // stride + 1
+    rows, cols, splits = mixdq.int8_tile_plan(B * Ho * Ho, Cout, 9 * _kblocks(Cin), bits, with_splits=True)
+    if not (rows == 256 and splits >= 2):
+        pytest.skip(f"the planner runs this shape on {rows} x {cols} tiles without a split reduction")
+    X = synth.normal_f16((B, H, H, Cin), 1.0, seed=41 + Cin)
+    Wt = synth.normal_f16((Cout, 3, 3, Cin), 0.02, seed=42 + Cout)
+    s_ref, _, codes = oracle_weights(Wt.reshape(Cout, -1), bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    acc_ref, y_ref = orc.conv3x3_a8(X, codes.reshape(Cout, 3, 3, Cin), s_ref, sx_ref, None, stride)
+    Xd = dev(X)
+    s, _, packed = device_weights(Wt.reshape(Cout, -1), bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    ws = mixdq.new_workspace(mixdq.conv3x3_workspace_bytes(B, H, H, Cin, Cout, stride, bits, 8))
+    acc = mixdq.conv3x3_acc_i32(Xd, packed, Cout, bits, sx, stride, ws, st)
+    y = mixdq.conv3x3(Xd, packed, Cout, bits, s, None, 8, sx, None, stride, ws, st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert np.array_equal(host(acc), acc_ref)
+    assert_close(host(y), y_ref)
+
+
+def test_planner_splits_the_long_reductions_of_the_16x16_level():
+    for bits in (4, 8):
+        rows, cols, splits = mixdq.int8_tile_plan(1024, 1280, 90, bits, with_splits=True)   # conv 1280 -> 1280 at 16 x 16
+        assert rows == 256 and 2 <= splits <= 4, (rows, cols, splits)
+
+
 def test_planner_keeps_small_layers_on_single_cta_tiles():
     assert mixdq.int8_tile_plan(1024, 1280, 10, 4) == (128, 96)      # attention projection, image batch 4: 112 CTAs
     assert mixdq.int8_tile_plan(256, 1280, 40, 4)[0] == 128          # FFN-2 at image batch 1
