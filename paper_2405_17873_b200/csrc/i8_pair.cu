@@ -761,10 +761,12 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap&
 }
 
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
-                    int num_sms, cudaStream_t stream)
+                    int splits, int num_sms, cudaStream_t stream)
 {
-    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || tp.acc_out) return MIXDQ_ERR_INVALID_ARG;
-    return launch_pair_t<2>(ta, tw, ty, tp, bn, 1, num_sms, stream);
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || tp.acc_out || splits < 1 || splits > 4 ||
+        splits > tp.k_blocks)
+        return MIXDQ_ERR_INVALID_ARG;
+    return launch_pair_t<2>(ta, tw, ty, tp, bn, splits, num_sms, stream);
 }
 
 }  // namespace i8

@@ -189,7 +189,7 @@ int pair_cluster_capacity(bool w4, int cluster_ctas);
 // box of 128 rows x 64 elements, tw the map of the layer's weights expanded to fp16 (q - zero) with a box of
 // bn / 2 rows x 64 elements; tp.k_blocks counts blocks of 64 elements and tp.act_scale is unused.
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
-                    int num_sms, cudaStream_t stream);
+                    int splits, int num_sms, cudaStream_t stream);
 
 }  // namespace i8
 }  // namespace mixdq

@@ -114,18 +114,32 @@ bool conv_box(int Ho, int Wo, int* Wb, int* Hb, int* Bb)
     return true;
 }
 
-// Tile width: whole rounds of 256 x bn tiles over the SM pairs, the per-tile cost growing with the width.
-int pick_tile(int M, int N, int k_blocks, int num_sms)
+// Tile width and reduction split: whole rounds of 256 x bn tiles over the SM pairs, the per-tile cost growing with
+// the width; layers with few tiles and a long reduction give one tile to a cluster of two to four CTA pairs.
+int pick_tile(int M, int N, int k_blocks, int num_sms, int* splits)
 {
     double best = 0;
     int best_bn = 0;
+    *splits = 1;
+    const int pairs = num_sms / 2;
     for (int bn = 96; bn <= 256; bn += 32) {
-        const double tiles = static_cast<double>(ceil_div(M, 2 * BM) * ceil_div(N, bn));
-        const double rounds = std::ceil(tiles / (num_sms / 2));
-        const double t = rounds * (std::max(k_blocks * (250.0 + 1.2 * bn), 30.0 * bn) + 800.0) + 16.0 * bn;
+        const int64_t tiles = ceil_div(M, 2 * BM) * ceil_div(N, bn);
+        const double per_kb = 250.0 + 1.2 * bn;
+        const double rounds = std::ceil(static_cast<double>(tiles) / pairs);
+        const double t = rounds * (std::max(k_blocks * per_kb, 30.0 * bn) + 800.0) + 16.0 * bn;
         if (best_bn == 0 || t < best) {
             best = t;
             best_bn = bn;
+            *splits = 1;
+        }
+        for (int sp = 2; sp <= 4 && tiles * sp <= pairs && k_blocks / sp >= 16; ++sp) {
+            if (tiles > i8::pair_cluster_capacity(false, 2 * sp)) continue;
+            const double ts = std::ceil(static_cast<double>(k_blocks) / sp) * per_kb + 16.0 * bn + 14000.0;
+            if (ts < best) {
+                best = ts;
+                best_bn = bn;
+                *splits = sp;
+            }
         }
     }
     return best_bn;
@@ -206,7 +220,8 @@ int run_pair(const Params& p, int amode, const void* packed, int w_bits, cudaStr
         tp.k_blocks = static_cast<int>(ceil_div(p.K, BKE));
     }
     if (rc != MIXDQ_OK) return rc;
-    const int bn = pick_tile(p.M, p.N, tp.k_blocks, num_sms);
+    int splits = 1;
+    const int bn = pick_tile(p.M, p.N, tp.k_blocks, num_sms, &splits);
     rc = encode_tmap_2d_f16(&tw, wexp, static_cast<uint64_t>(p.K), static_cast<uint64_t>(p.N), static_cast<uint64_t>(ldw),
                             BKE, static_cast<uint32_t>(bn / 2));
     if (rc != MIXDQ_OK) return rc;
@@ -215,7 +230,7 @@ int run_pair(const Params& p, int amode, const void* packed, int w_bits, cudaStr
                                 static_cast<uint64_t>(p.ldy), 32, 32, true);
         if (rc != MIXDQ_OK) return rc;
     }
-    return i8::launch_pair_f16(ta, tw, ty, tp, bn, num_sms, stream);
+    return i8::launch_pair_f16(ta, tw, ty, tp, bn, splits, num_sms, stream);
 }
 
 }  // namespace wo
