@@ -68,6 +68,14 @@ unsigned long long mixdq_kernel_launches(void);
 int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols,
                          int* reduction_splits);
 
+/* Diagnostic (the paper has no counterpart; its implementation runs the activation quantization as a kernel of
+ * its own, Sec. 4.1 "Hardware Profiling"): width of the 128-row output tiles when mixdq_linear, called with a
+ * workspace, 8-bit symmetric activations and a row-major X, runs a layer of M rows, N channels and K inputs as ONE
+ * kernel that quantizes its activation tiles itself; 0 when the layer runs as quantization pass + GEMM (the
+ * one-kernel form pays only for short reductions, K <= 640, on one wave of tiles).  Negative: an error code.
+ * For tests and benchmarks: nothing is launched. */
+int mixdq_linear_fused_quant_tile(int64_t M, int64_t N, int64_t K, int w_bits);
+
 /* Static, NUL-terminated description of an error code (host pointer, never NULL). */
 const char* mixdq_strerror(int code);
 

@@ -204,6 +204,16 @@ extern "C" int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int 
     return MIXDQ_OK;
 }
 
+extern "C" int mixdq_linear_fused_quant_tile(int64_t M, int64_t N, int64_t K, int w_bits)
+{
+    if (M <= 0 || N <= 0 || K <= 0 || M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return MIXDQ_ERR_CUDA;
+    if (K % 16 != 0) return 0;  // (the TMA-fed kernels need 16-byte rows of codes)
+    return i8::plan_fq_tile(static_cast<int>(M), static_cast<int>(N), static_cast<int>(ceil_div(K, 128)), w_bits == 4, sms);
+}
+
 extern "C" const char* mixdq_strerror(int code)
 {
     switch (code) {

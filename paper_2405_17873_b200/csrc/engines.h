@@ -61,6 +61,9 @@ int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* sc
 // M x N over k_blocks k-blocks of 128, else 0 (the single-CTA kernels run).  *splits (optional): how many CTA
 // pairs share one tile's reduction (1: persistent pairs; without the pointer only that form is considered).
 int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits = nullptr);
+// Tile width of the fused-quantization kernel (one launch per layer, 128 x width tiles) when the planner prefers
+// it for a linear layer with symmetric activations, else 0 (quantization pass + GEMM).
+int plan_fq_tile(int M, int N, int k_blocks, bool w4, int num_sms);
 // Tile width (128, 96 or 64) of the one-tile kernel on 128-wide slots.
 int plan_narrow_tile(int M, int N, int k_blocks, int num_sms);
 // The two steps as calls of their own, for activations that are stored as int8 between layers: the codes of

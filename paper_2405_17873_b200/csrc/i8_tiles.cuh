@@ -191,5 +191,11 @@ int pair_cluster_capacity(bool w4, int cluster_ctas);
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
                     int splits, int num_sms, cudaStream_t stream);
 
+// Fused-quantization form (i8_fq.cu): one kernel per linear layer, fp16 activations in.  tx: fp16 map of X with a
+// box of 128 rows x 64 elements (128-byte swizzle), tw: weight map with a box of bn rows, ty: output map with a
+// 32 x 32 box; tile 128 x bn (bn a multiple of 32, <= 256).
+int launch_fq(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
+              cudaStream_t stream);
+
 }  // namespace i8
 }  // namespace mixdq

@@ -1197,6 +1197,23 @@ int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits
     return best_bn;
 }
 
+// Fused-quantization kernel (i8_fq.cu) or the two-kernel forms.  The fused kernel's k-block costs three to four
+// times the two-kernel main loop's (its converter warps' turn bounds it), and its fixed cost is one kernel's
+// instead of two: it wins where the reduction is short (at most five k-blocks), the activations large enough for
+// the quantization pass to matter, and the tiles fit the SMs in one wave.  Measured on B200, fused against
+// two-kernel: 4096 x 640 x 640 W4 9.5 / 10.5 us, W8 7.8 / 9.2; 4096 x 640 x 320 7.5 / 9.9 and 6.5 / 8.7;
+// 1024 x 640 x 640 W8 7.0 / 8.5 (W4 a tie); losing: 1024 x 1280 x 640 (8.9 / 7.1), 16384 x 320 x 640 (two
+// waves: 18.5 / 15.5), anything from ten k-blocks up (1024 x 1280 x 1280: 12.2 / 8.5).
+// Width: the narrowest multiple of 32 whose tiles still fit one wave (less MMA and epilogue work per CTA).
+int plan_fq_tile(int M, int N, int k_blocks, bool w4, int num_sms)
+{
+    if (k_blocks > 5 || N > 1024 || M < 1024 || (M < 2048 && w4)) return 0;
+    const int64_t row_tiles = ceil_div(M, BM);
+    for (int bn = 64; bn <= 256; bn += 32)
+        if (row_tiles * ceil_div(N, bn) <= num_sms) return bn;
+    return 0;
+}
+
 // Width of the one-tile kernel's tiles for a layer the single-CTA kernels run on 128-wide slots: 128, or 96 / 64
 // when that raises the number of CTAs while they still fit the SMs in one wave and the reduction is not split.
 int plan_narrow_tile(int M, int N, int k_blocks, int num_sms)
@@ -1251,9 +1268,49 @@ bool tma_path_ok(const Params& p, int amode, int w_bits)
 // that an earlier kernel of the stream has written ([M, K] dense, or the NHWC image, padded when p.act_zero).
 static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bits, int8_t* aq, cudaStream_t stream);
 
+// One-kernel form: the GEMM kernel quantizes its own activation tiles (i8_fq.cu).
+static int run_fq(const Params& p, const void* packed, int w_bits, int bn, cudaStream_t stream)
+{
+    const bool w4 = w_bits == 4;
+    const int64_t pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
+    CUtensorMap tx, tw, ty{};
+    TmaParams tp{};
+    tp.M = p.M;
+    tp.N = p.N;
+    tp.k_blocks = static_cast<int>(ceil_div(p.K, BK));
+    tp.act_scale = p.act_scale;
+    tp.w_scale = p.w_scale;
+    tp.bias = p.bias;
+    tp.Y = p.Y;
+    tp.ldy = p.ldy;
+    tp.acc_out = p.acc_out;
+    tp.status = p.status;
+    tp.small_acc = static_cast<long long>(p.K) * 127 * (w4 ? 7 : 127) < (1ll << 22);
+    tp.tma_store = p.Y && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
+    int rc = encode_tmap_2d_f16(&tx, p.X, static_cast<uint64_t>(p.K), static_cast<uint64_t>(p.M),
+                                static_cast<uint64_t>(p.ldx), 64, BM, false);
+    if (rc != MIXDQ_OK) return rc;
+    if (w4)
+        rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, static_cast<uint32_t>(bn), false);
+    else
+        rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(p.K), p.N, pitch, BK, static_cast<uint32_t>(bn), true);
+    if (rc != MIXDQ_OK) return rc;
+    if (tp.tma_store) {
+        rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
+                                static_cast<uint64_t>(p.ldy), 32, 32, true);
+        if (rc != MIXDQ_OK) return rc;
+    }
+    return launch_fq(tx, tw, ty, tp, w4, bn, stream);
+}
+
 int run_tma(const Params& p, int amode, const void* packed, int w_bits, void* scratch, cudaStream_t stream)
 {
     int8_t* aq = static_cast<int8_t*>(scratch);
+    if (amode == A_LINEAR && !p.act_zero && !p.addend && !p.test_drop_b_kblock) {
+        const int num_sms = sm_count();
+        const int fq_bn = num_sms > 0 ? plan_fq_tile(p.M, p.N, static_cast<int>(ceil_div(p.K, BK)), w_bits == 4, num_sms) : 0;
+        if (fq_bn > 0) return run_fq(p, packed, w_bits, fq_bn, stream);
+    }
 
     // 1. quantize the activations once
     const bool conv = amode == A_CONV3;

@@ -26,6 +26,7 @@ _SIGNATURES = {
     "mixdq_strerror": (C.c_char_p, [_int]),
     "mixdq_kernel_launches": (C.c_ulonglong, []),
     "mixdq_int8_tile_plan": (_int, [_i64, _i64, _i64, _int, C.POINTER(_int), C.POINTER(_int), C.POINTER(_int)]),
+    "mixdq_linear_fused_quant_tile": (_int, [_i64, _i64, _i64, _int]),
     "mixdq_packed_bytes": (_int, [_i64, _i64, _int, _int, C.POINTER(_sz)]),
     "mixdq_weight_minmax_params": (_int, [_vp, _i64, _i64, _int, _int, _vp, _vp, _vp]),
     "mixdq_pack_weights": (_int, [_vp, _i64, _i64, _int, _vp, _vp, _int, _vp, _vp]),
@@ -129,6 +130,14 @@ def int8_tile_plan(M: int, N: int, k_blocks: int, w_bits: int, with_splits: bool
     r, c, sp = _int(0), _int(0), _int(0)
     _chk(lib().mixdq_int8_tile_plan(M, N, k_blocks, w_bits, C.byref(r), C.byref(c), C.byref(sp)), "mixdq_int8_tile_plan")
     return (r.value, c.value, sp.value) if with_splits else (r.value, c.value)
+
+
+def linear_fused_quant_tile(M: int, N: int, K: int, w_bits: int) -> int:
+    """Tile width of the one-kernel (fused quantization) form for this linear layer, 0 when it runs as two kernels."""
+    r = lib().mixdq_linear_fused_quant_tile(M, N, K, w_bits)
+    if r < 0:
+        _chk(r, "mixdq_linear_fused_quant_tile")
+    return r
 
 
 def packed_bytes(N: int, K: int, bits: int, layout: int = LAYOUT_DEVICE) -> int:

@@ -19,8 +19,9 @@ def _kblocks(K):
 
 
 # ragged rows / columns / reduction lengths, one and several tiles per CTA pair, all tile widths
-LINEAR_SHAPES = [(5567, 776, 784), (3274, 776, 432), (4458, 648, 1952), (6812, 328, 1936), (5968, 1304, 448),
-                 (4096, 640, 640), (1024, 10240, 1280), (16384, 320, 640)]
+# (reductions of more than five k-blocks, or wide outputs: shorter ones on one wave of tiles take the one-kernel form)
+LINEAR_SHAPES = [(5567, 776, 784), (3274, 776, 688), (4458, 648, 1952), (6812, 328, 1936), (5968, 1304, 448),
+                 (4096, 640, 768), (1024, 10240, 1280), (16384, 320, 640)]
 
 
 @pytest.mark.parametrize("bits", [8, 4])
@@ -28,6 +29,7 @@ LINEAR_SHAPES = [(5567, 776, 784), (3274, 776, 432), (4458, 648, 1952), (6812, 3
 def test_linear_on_pair_tiles(bits, M, N, K):
     rows, cols = mixdq.int8_tile_plan(M, N, _kblocks(K), bits)
     assert rows == 256 and cols in (160, 192, 224, 256), (rows, cols)
+    assert mixdq.linear_fused_quant_tile(M, N, K, bits) == 0
     X = synth.normal_f16((M, K), 1.0, seed=M + K)
     W = synth.normal_f16((N, K), 0.02, seed=N + K + 1)
     b = synth.normal_f16((N,), 0.01, seed=N)
