@@ -441,6 +441,45 @@ def config_records(torch, mixdq, synth, stream, peaks, probe_int8):
     return out
 
 
+def fused_quant_records(torch, mixdq, synth, stream):
+    """The W4A8 / W8A8 linear layer as one kernel (activation quantization inside the GEMM) against quantization
+    pass + GEMM, both forms forced through their explicit entry points, beside what the planner picks.  Graph of ten
+    calls, warm L2.  The one-kernel form's tile width is the planner's where it selects that form, else the
+    narrowest that fits one wave (256 when none does)."""
+    dev = lambda a: torch.from_numpy(a).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    out = []
+    for (M, N, K) in [(4096, 640, 640), (4096, 640, 320), (1024, 640, 640), (1024, 1280, 640), (1024, 1280, 1280),
+                      (16384, 320, 640), (1024, 1280, 5120)]:
+        for bits in (4, 8):
+            Xd = dev(synth.normal_f16((M, K), 1.0, seed=9000 + K))
+            Wd = dev(synth.normal_f16((N, K), 0.02, seed=9100 + N))
+            s, _ = mixdq.weight_minmax_params(Wd, bits, True)
+            pk = mixdq.pack_weights(Wd, bits, s)
+            sx = mixdq.act_scale(Xd)
+            ws = mixdq.new_workspace(mixdq.workspace_bytes(M, N, K, bits, 8))
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+            planned = mixdq.linear_fused_quant_tile(M, N, K, bits)
+            cols = planned
+            if cols == 0:
+                fits = [c for c in range(64, 257, 32) if -(-M // 128) * -(-N // c) <= sms]
+                cols = fits[0] if fits else 256
+
+            def two():
+                mixdq.quantize_acts(Xd, sx, out=xq)
+                mixdq.linear_q8(xq, pk, N, bits, s, sx, None, status, out=Y)
+
+            t_two = _time_graph(torch, stream, two)
+            t_one = _time_graph(torch, stream, lambda: mixdq.linear_a8_fused_quant(Xd, pk, N, bits, s, sx, None, cols, status, out=Y))
+            t_plan = _time_graph(torch, stream, lambda: mixdq.linear(Xd, pk, N, bits, s, None, 8, sx, None, ws, status, out=Y))
+            out.append({"M": M, "N": N, "K": K, "w_bits": bits, "two_kernel_us": round(t_two, 2),
+                        "one_kernel_us": round(t_one, 2), "one_kernel_tile": f"128x{cols}",
+                        "planned": "one kernel" if planned else "two kernels", "planned_us": round(t_plan, 2)})
+    return out
+
+
 def weight_bound_records(torch, mixdq, synth, stream, peaks):
     """The weight-only engine where it is bound by the weight stream: the transformer FFN layers on 16 tokens,
     with as many distinct copies of the packed weights as it takes to exceed L2 several times over, walked
@@ -784,6 +823,7 @@ def run_ours(args):
                             "nominal": NOMINAL}
             del sweep.workspace
             out["configs"] = config_records(torch, mixdq, synth, stream, peaks, probe_int8)
+            out["fused_quantization"] = fused_quant_records(torch, mixdq, synth, stream)
             out["weight_bound_layers"] = weight_bound_records(torch, mixdq, synth, stream, peaks)
             sweep = None
             torch.cuda.empty_cache()

@@ -280,6 +280,21 @@ int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void* packed_W, 
                     const float* w_scale, const float* act_scale, const void* bias, void* Y, int32_t* status,
                     void* stream);
 
+/*
+ * The W8A8 / W4A8 linear layer of mixdq_linear as ONE kernel on 128 x tile_cols output tiles, whatever the planner
+ * would choose: the GEMM kernel takes the fp16 activations by TMA and quantizes every tile itself (Sec. 4.1:
+ * symmetric per-tensor 8-bit activations, the same codes as mixdq_quantize_acts), so no workspace is needed and
+ * no quantization kernel runs; the output bits equal mixdq_linear's.  The paper runs the quantization as a kernel
+ * of its own; this form trades that launch for arithmetic repeated in every tile column, and is faster only for
+ * short reductions (mixdq_linear_fused_quant_tile).  tile_cols: a multiple of 32 in [32, 256]
+ * (MIXDQ_ERR_INVALID_ARG otherwise).  X fp16 [M, K] with row stride ldx (K % 16 == 0, ldx % 8 == 0:
+ * MIXDQ_ERR_UNSUPPORTED otherwise; 16-byte aligned), Y fp16 [M, N] with row stride ldy; symmetric weights,
+ * w_bits in {4, 8}; bias may be NULL.  All pointers DEVICE except status (device, may be NULL) and stream.
+ */
+int mixdq_linear_a8_fused_quant(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W, int64_t N,
+                                int w_bits, const float* w_scale, const float* act_scale, const void* bias, void* Y,
+                                int64_t ldy, int tile_cols, int32_t* status, void* stream);
+
 /* The 3x3 convolution on a stored int8 NHWC image [B, H, W, Cin] (codes from mixdq_quantize_acts on the
  * [B*H*W, Cin] pixel matrix); zero padding is code 0.  Geometry as for the two-kernel path of mixdq_conv3x3
  * (Cin % 32 == 0; Wo a multiple of 128, or 128 / Wo a divisor or a multiple of Ho; stride 2 only on even H, W):

@@ -371,6 +371,32 @@ extern "C" int mixdq_linear_q8(const void* Xq, int64_t M, int64_t K, const void*
     return linear_q8_impl(Xq, M, K, packed_W, N, w_bits, w_scale, act_scale, bias, Y, nullptr, status, stream);
 }
 
+extern "C" int mixdq_linear_a8_fused_quant(const void* X, int64_t M, int64_t K, int64_t ldx, const void* packed_W,
+                                           int64_t N, int w_bits, const float* w_scale, const float* act_scale,
+                                           const void* bias, void* Y, int64_t ldy, int tile_cols, int32_t* status,
+                                           void* stream)
+{
+    if (!X || !packed_W || !Y || !w_scale || !act_scale) return MIXDQ_ERR_INVALID_ARG;
+    if (!fits_int(M) || !fits_int(K) || !fits_int(N) || ldx < K || ldy < N) return MIXDQ_ERR_INVALID_ARG;
+    if (tile_cols < 32 || tile_cols > 256 || tile_cols % 32 != 0) return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 4 && w_bits != 8) return MIXDQ_ERR_UNSUPPORTED;
+    if (K % 16 != 0 || ldx % 8 != 0) return MIXDQ_ERR_UNSUPPORTED;
+    if (!aligned16(packed_W) || !aligned16(X)) return MIXDQ_ERR_ALIGNMENT;
+    i8::Params p;
+    p.X = static_cast<const __half*>(X);
+    p.ldx = ldx;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.act_scale = act_scale;
+    p.w_scale = w_scale;
+    p.bias = static_cast<const __half*>(bias);
+    p.Y = static_cast<__half*>(Y);
+    p.ldy = ldy;
+    p.status = status;
+    return i8::run_fq(p, packed_W, w_bits, tile_cols, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int mixdq_selftest_abandoned_wait(const void* Xq, int64_t M, int64_t K, const void* packed_W, int64_t N,
                                              int w_bits, const float* w_scale, const float* act_scale, void* Y,
                                              int drop_k_block, int32_t* status, void* stream)

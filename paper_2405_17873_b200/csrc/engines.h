@@ -64,6 +64,9 @@ int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits
 // Tile width of the fused-quantization kernel (one launch per layer, 128 x width tiles) when the planner prefers
 // it for a linear layer with symmetric activations, else 0 (quantization pass + GEMM).
 int plan_fq_tile(int M, int N, int k_blocks, bool w4, int num_sms);
+// The one-kernel form itself on 128 x bn tiles (bn a multiple of 32, 32 .. 256): a linear layer with symmetric
+// activations, K % 16 == 0, ldx % 8 == 0, X 16-byte aligned; p.Y and / or p.acc_out.
+int run_fq(const Params& p, const void* packed, int w_bits, int bn, cudaStream_t stream);
 // Tile width (128, 96 or 64) of the one-tile kernel on 128-wide slots.
 int plan_narrow_tile(int M, int N, int k_blocks, int num_sms);
 // The two steps as calls of their own, for activations that are stored as int8 between layers: the codes of

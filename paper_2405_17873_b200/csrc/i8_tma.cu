@@ -1202,12 +1202,13 @@ int plan_pair_tile(int M, int N, int k_blocks, bool w4, int num_sms, int* splits
 // instead of two: it wins where the reduction is short (at most five k-blocks), the activations large enough for
 // the quantization pass to matter, and the tiles fit the SMs in one wave.  Measured on B200, fused against
 // two-kernel: 4096 x 640 x 640 W4 9.5 / 10.5 us, W8 7.8 / 9.2; 4096 x 640 x 320 7.5 / 9.9 and 6.5 / 8.7;
-// 1024 x 640 x 640 W8 7.0 / 8.5 (W4 a tie); losing: 1024 x 1280 x 640 (8.9 / 7.1), 16384 x 320 x 640 (two
+// 1024 x 640 x 640 W8 6.8 / 8.7, W4 8.3 / 8.7; losing: 1024 x 1280 x 640 (8.9 / 7.1), 16384 x 320 x 640 (two
 // waves: 18.5 / 15.5), anything from ten k-blocks up (1024 x 1280 x 1280: 12.2 / 8.5).
 // Width: the narrowest multiple of 32 whose tiles still fit one wave (less MMA and epilogue work per CTA).
 int plan_fq_tile(int M, int N, int k_blocks, bool w4, int num_sms)
 {
-    if (k_blocks > 5 || N > 1024 || M < 1024 || (M < 2048 && w4)) return 0;
+    (void)w4;
+    if (k_blocks > 5 || N > 1024 || M < 1024) return 0;
     const int64_t row_tiles = ceil_div(M, BM);
     for (int bn = 64; bn <= 256; bn += 32)
         if (row_tiles * ceil_div(N, bn) <= num_sms) return bn;
@@ -1269,7 +1270,7 @@ bool tma_path_ok(const Params& p, int amode, int w_bits)
 static int run_tma_gemm(const Params& p, int amode, const void* packed, int w_bits, int8_t* aq, cudaStream_t stream);
 
 // One-kernel form: the GEMM kernel quantizes its own activation tiles (i8_fq.cu).
-static int run_fq(const Params& p, const void* packed, int w_bits, int bn, cudaStream_t stream)
+int run_fq(const Params& p, const void* packed, int w_bits, int bn, cudaStream_t stream)
 {
     const bool w4 = w_bits == 4;
     const int64_t pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);

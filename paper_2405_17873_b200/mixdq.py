@@ -47,6 +47,7 @@ _SIGNATURES = {
     "mixdq_quantize_acts": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "mixdq_linear_q8": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
     "mixdq_conv3x3_q8": (_int, [_vp, _i64, _i64, _i64, _i64, _vp, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "mixdq_linear_a8_fused_quant": (_int, [_vp, _i64, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _vp, _i64, _int, _vp, _vp]),
     "mixdq_selftest_abandoned_wait": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp, _int, _vp, _vp]),
     "mixdq_linear_q8_acc_i32": (_int, [_vp, _i64, _i64, _vp, _i64, _int, _vp, _vp, _vp]),
     "mixdq_split_workspace_bytes": (_int, [_i64, _i64, _i64, _i64, _i64, C.POINTER(_sz)]),
@@ -340,6 +341,17 @@ def linear_q8(Xq, packed_W, N: int, w_bits: int, w_scale, act_scale, bias=None, 
     Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=Xq.device)
     _chk(lib().mixdq_linear_q8(_ptr(Xq), M, K, _ptr(packed_W), N, w_bits, _ptr(w_scale), _ptr(act_scale),
                                _ptr(bias), _ptr(Y), _ptr(status), _stream()), "mixdq_linear_q8")
+    return Y
+
+
+def linear_a8_fused_quant(X, packed_W, N: int, w_bits: int, w_scale, act_scale, bias=None, tile_cols: int = 128,
+                          status=None, out=None):
+    """mixdq_linear (8-bit activations) as one kernel on 128 x tile_cols tiles, whatever the planner would choose."""
+    M, K = X.shape
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=X.device)
+    _chk(lib().mixdq_linear_a8_fused_quant(_ptr(X), M, K, X.stride(0), _ptr(packed_W), N, w_bits, _ptr(w_scale),
+                                           _ptr(act_scale), _ptr(bias), _ptr(Y), Y.stride(0), tile_cols, _ptr(status),
+                                           _stream()), "mixdq_linear_a8_fused_quant")
     return Y
 
 

@@ -15,7 +15,7 @@ from helpers import assert_close, dev, device_weights, host, oracle_weights, sta
 pytestmark = pytest.mark.gpu
 
 # the 32 x 32 level's attention projections at image batch 4 and 1, and ragged rows / columns / reduction tails
-SHAPES = [(4096, 640, 640, 4), (4096, 640, 640, 8), (4096, 640, 320, 4), (1024, 640, 640, 8), (3274, 776, 432, 4),
+SHAPES = [(4096, 640, 640, 4), (4096, 640, 640, 8), (4096, 640, 320, 4), (1024, 640, 640, 8), (1024, 640, 640, 4), (3274, 776, 432, 4),
           (2100, 1000, 208, 8), (2049, 40, 16, 4), (5000, 136, 640, 8)]
 
 
@@ -78,4 +78,41 @@ def test_every_finite_fp16_value_through_the_fused_quantizer(scale):
 def test_two_kernel_shapes_stay_two_kernel():
     for M, N, K in [(1024, 1280, 1280), (1024, 1280, 640), (16384, 320, 640), (4096, 5120, 640), (4096, 640, 2560)]:
         assert mixdq.linear_fused_quant_tile(M, N, K, 4) == 0
-    assert mixdq.linear_fused_quant_tile(1024, 640, 640, 4) == 0  # int4 at image batch 1: a tie, left as it was
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("M,N,K,tile_cols", [(1024, 1280, 1280, 256), (1024, 1280, 1280, 96), (1000, 1288, 5136, 160),
+                                             (130, 72, 48, 32), (4096, 640, 2560, 224), (777, 520, 400, 64)])
+def test_explicit_one_kernel_form_equals_the_planned_path(bits, M, N, K, tile_cols):
+    """mixdq_linear_a8_fused_quant on shapes the planner keeps on two kernels (long reductions, several waves,
+    ragged tiles, every tile width class): the same output bits as mixdq_linear, which the other tests hold
+    against the oracle, and the oracle's outputs within tolerance."""
+    X = synth.normal_f16((M, K), 1.0, seed=M + K + 3)
+    W = synth.normal_f16((N, K), 0.02, seed=N + K + 4)
+    b = synth.normal_f16((N,), 0.01, seed=N + 5)
+    s_ref, _, codes = oracle_weights(W, bits, True)
+    sx_ref = orc.act_scale(orc.act_absmax(X), 8)
+    _, y_ref = orc.linear_a8(X, codes, s_ref, sx_ref, b)
+    Xd = dev(X)
+    s, _, packed = device_weights(W, bits, True)
+    sx = mixdq.act_scale(Xd)
+    st = status_word()
+    y_fused = mixdq.linear_a8_fused_quant(Xd, packed, N, bits, s, sx, dev(b), tile_cols, st)
+    y = mixdq.linear(Xd, packed, N, bits, s, None, 8, sx, dev(b), workspace=workspace_for(M, N, K, bits), status=st)
+    torch.cuda.synchronize()
+    assert int(host(st)[0]) == 0
+    assert_close(host(y_fused), y_ref)
+    assert np.array_equal(host(y_fused).view(np.uint16), host(y).view(np.uint16))
+
+
+def test_explicit_one_kernel_form_rejects_bad_arguments():
+    X = dev(synth.normal_f16((128, 64), 1.0, seed=1))
+    s, _, packed = device_weights(synth.normal_f16((32, 64), 0.02, seed=2), 8, True)
+    sx = mixdq.act_scale(X)
+    for bad in (0, 16, 48, 288):
+        with pytest.raises(mixdq.MixdqError):
+            mixdq.linear_a8_fused_quant(X, packed, 32, 8, s, sx, None, bad)
+    X40 = dev(synth.normal_f16((128, 40), 1.0, seed=3))  # rows of 40 codes are not 16-byte multiples
+    s40, _, packed40 = device_weights(synth.normal_f16((32, 40), 0.02, seed=4), 8, True)
+    with pytest.raises(mixdq.MixdqError):
+        mixdq.linear_a8_fused_quant(X40, packed40, 32, 8, s40, sx, None, 64)
