@@ -146,22 +146,30 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar)
 constexpr int PAIR_BN_MAX = 256;
 constexpr int ACC_COLS = 256;  // tensor-memory columns of one accumulator (the widest tile)
 
-// MODE: 0 = int8 weights, 1 = int4 weights (expanded in shared memory), 2 = fp16 operands (kind::f16)
+// MODE: 0 = int8 weights, 1 = int4 weights (expanded in shared memory), 2 = fp16 operands (kind::f16), 3 = fp16
+// activations and packed 2- / 3- / 4- / 8-bit weights expanded to fp16 (code - zero) in shared memory
 template <int MODE>
 struct PairSmem {
     static constexpr bool W4 = MODE == 1;
-    static constexpr bool F16 = MODE == 2;
+    static constexpr bool F16 = MODE == 2 || MODE == 3;
+    static constexpr bool WO = MODE == 3;
+    static constexpr bool PACKED = W4 || WO;  // a ring of packed weight tiles and expansion warps
     static constexpr int BKE = F16 ? BK / 2 : BK;           // elements of a k-block (its rows are 128 bytes either way)
     static constexpr int A_BYTES = BM * BK;                 // this CTA's 128 activation rows of a k-block
     static constexpr int B_BYTES = (PAIR_BN_MAX / 2) * BK;  // this CTA's half of the int8 weight tile
-    static constexpr int P_BYTES = B_BYTES / 2;             // the same as packed int4
+    // packed tiles.  int4 -> int8: one per k-block.  Weight-only: one per TWO k-blocks (128 codes: the bit-plane
+    // formats store blocks of 128), 16 bytes per bit and row, at most 4 bits (8-bit weights keep the expansion pass).
+    static constexpr int P_BYTES = B_BYTES / 2;
     // Depths: everything that is in flight from L2 as deep as shared memory allows; the expanded int8 tiles of
     // the W4 form are staging, one per expansion group.
     // W4: the packed ring must be deeper than the number of expansion groups, or the request for a group's
     // next tile goes out only when its last one has been expanded and the groups stall together once per lap.
+    // Weight-only: a packed tile serves two consecutive k-blocks, i.e. two of the four expansion groups; with an
+    // even number of packed slots a slot always belongs to the same two groups, which then meet every phase of its
+    // barrier.
     static constexpr int AS = W4 ? 5 : 6;
-    static constexpr int ES = W4 ? 4 : 6;
-    static constexpr int PS = W4 ? 6 : 0;
+    static constexpr int ES = PACKED ? 4 : 6;
+    static constexpr int PS = W4 ? 6 : (WO ? 4 : 0);
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + AS * A_BYTES;
     static constexpr int OFF_P = OFF_B + ES * B_BYTES;
@@ -188,7 +196,7 @@ struct PairSmem {
     // warps: 0 activation producer, 1 MMA issuer (leader) and tensor-memory allocation, 2-5 epilogue (first part
     // of the columns), W4: 6-13 nibble expansion, then four epilogue helpers (the other columns), then the weight
     // producer
-    static constexpr int HELPER0 = W4 ? 14 : 6;
+    static constexpr int HELPER0 = PACKED ? 14 : 6;
     static constexpr int B_WARP = HELPER0 + 4;
     static constexpr int MMA2_WARP = B_WARP + 1;  // second MMA issuer (leader)
     static constexpr int THREADS = (MMA2_WARP + 1) * 32;
@@ -199,6 +207,11 @@ struct PairArgs {
     int n_tiles;      // tiles along N
     int total_tiles;  // pair tiles in all
     int splits;       // > 1: one tile per cluster of 2 * splits CTAs, the reduction split over its CTA pairs
+    // weight-only mode: width of the packed codes (2, 3, 4, 8), whether they are signed, per-channel zero-points
+    // (nullptr for signed codes)
+    int w_bits;
+    int w_signed;
+    const int32_t* w_zero;
 };
 
 // Grid (2 * splits * (pairs or tiles), 1, 1) with clusters of 2 * splits CTAs along x: CTAs 2 i and 2 i + 1 of a
@@ -214,6 +227,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     using L = PairSmem<MODE>;
     constexpr bool W4 = L::W4;
     constexpr bool F16 = L::F16;
+    constexpr bool WO = L::WO;
+    constexpr bool PACKED = L::PACKED;
     constexpr int BKE = L::BKE;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -253,12 +268,12 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             mbar_init(bar0 + 8 * (L::EMPTY_A + s), 1);  // one commit
         }
         for (int s = 0; s < L::ES; ++s) {
-            mbar_init(bar0 + 8 * (L::READY_B + s), W4 ? 4 : 1);  // W4: two expansion warps of each CTA
+            mbar_init(bar0 + 8 * (L::READY_B + s), PACKED ? 4 : 1);  // packed: two expansion warps of each CTA
             mbar_init(bar0 + 8 * (L::EMPTY_B + s), 1);
         }
         for (int s = 0; s < L::PS; ++s) {
             mbar_init(bar0 + 8 * (L::FULL_P + s), 1);
-            mbar_init(bar0 + 8 * (L::EMPTY_P + s), 2);
+            mbar_init(bar0 + 8 * (L::EMPTY_P + s), WO ? 4 : 2);  // the warps of the group(s) that read the tile
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar0 + 8 * (L::ACC_FULL + b), 2);    // one commit of each issuer
@@ -284,7 +299,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     // (constants of the layer), whose producer runs ahead
     // (and the warps that expand them, which touch shared memory only)
     // (fp16 mode: the weight operand is the output of the expansion kernel launched just before: everyone waits)
-    if ((F16 || warp != L::B_WARP) && !(W4 && warp >= 6 && warp < L::HELPER0)) pdl_wait();
+    if ((MODE == 2 || warp != L::B_WARP) && !(PACKED && warp >= 6 && warp < L::HELPER0)) pdl_wait();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
@@ -337,7 +352,32 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         __syncwarp();
     } else if (warp == L::B_WARP) {
         // ------------------------------------------------------------ weight-tile producer (own half of the rows)
-        if (lane == 0) {
+        if (lane == 0 && WO) {
+            // packed tiles of 128 codes (two k-blocks), this CTA's half of the tile's rows; the reduction is never
+            // split in this mode, so a tile's k-blocks start at 0
+            constexpr uint32_t PS = L::PS > 0 ? L::PS : 1;
+            const int unit_bytes = 16 * g.w_bits;
+            const int units = (nkb + 1) >> 1;
+            uint32_t s = 0, par = 1;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int tile = pair + t * npairs;
+                const int n0 = (tile % g.n_tiles) * bn + static_cast<int>(rank) * bh;
+                for (int u = 0; u < units; ++u) {
+                    if (!mbar_wait(bar0 + 8 * (L::EMPTY_P + s), par, s_abort)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t full = bar0 + 8 * (L::FULL_P + s);
+                    mbar_arrive_expect_tx(full, static_cast<uint32_t>(bh * unit_bytes));
+                    tma_load_2d(p0 + s * L::P_BYTES, &tmap_w, u * unit_bytes, n0, full);
+                    if (++s == PS) {
+                        s = 0;
+                        par ^= 1;
+                    }
+                }
+            }
+        } else if (lane == 0) {
             constexpr int R = W4 ? L::PS : L::ES;
             constexpr int ROW_BYTES = W4 ? BK / 2 : BK;   // bytes of a k-block of one weight row
             constexpr int ROW_STEP = F16 ? BKE : ROW_BYTES;  // the same in units of the weight map's element
@@ -435,7 +475,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         mbar_arrive(tile_go);
                     }
                     tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa), pair_mask);
-                    if (W4) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
+                    if (PACKED) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
                     sa += 2;
                     if (sa >= static_cast<uint32_t>(L::AS)) {
                         sa -= L::AS;
@@ -557,6 +597,106 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (lane == 0) mbar_arrive_cluster(lead_acc_empty + 8 * buf);
         }
         if (p.tma_store && lane == 0) tma_store_wait_read();  // shared memory stays valid until then
+    } else if (WO && warp >= 6 && warp < L::HELPER0) {
+        // ------------------------------------------------------------ packed codes -> fp16 (code - zero), own half
+        // Four groups of two warps as below; group g takes the k-blocks g, g + 4, ... of the CTA's sequence and owns
+        // slot g of the fp16 weight ring.  A thread turns eight codes of a row into one 16-byte chunk of the
+        // swizzled tile: 1024 + u is the fp16 bit pattern 0x6400 | u for an integer u < 1024, so the difference
+        // (1024 + u) - (1024 + zero) is exact and the weights enter the MMA as exact integers.
+        const int group = (warp - 6) >> 1;
+        const int gt = tid - 192 - group * 64;  // 0..63 within the group
+        const int total_kb = my_tiles * nkb;
+        const int units = (nkb + 1) >> 1;
+        const int unit_bytes = 16 * g.w_bits;
+        constexpr uint32_t PS = L::PS > 0 ? L::PS : 1;
+        const uint32_t lead_ready = lead_bar0 + 8 * (L::READY_B + group);
+        uint8_t* b_stage = sB + group * L::B_BYTES;
+        uint32_t n = 0;
+        int z_tile = -1;
+        __half2 z2r[2] = {__half2half2(__ushort_as_half(0x6400)), __half2half2(__ushort_as_half(0x6400))};
+        for (int it = group; it < total_kb; it += 4, ++n) {
+            const int t = it / nkb, kbi = it - t * nkb;
+            const uint32_t useq = static_cast<uint32_t>(t * units + (kbi >> 1));  // packed tile in the CTA's sequence
+            const uint32_t sp = useq % PS, rp = useq / PS;
+            const uint8_t* stg = sP + sp * L::P_BYTES;
+            bool ok = mbar_wait(bar0 + 8 * (L::FULL_P + sp), rp & 1, s_abort);
+            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * (L::EMPTY_B + group), (n & 1) ^ 1, s_abort);
+            if (!__all_sync(0xffffffffu, ok)) break;  // the warp leaves together
+            const int kofs = (kbi & 1) * 64;  // which half of the packed tile's 128 codes
+            if (t != z_tile) {
+                // zero-points of this thread's rows (rows gt and gt + 64 of the CTA's half tile), as fp16 1024 + zero
+                // (+ the offset that moved signed codes into the unsigned range)
+                z_tile = t;
+                const int tile = pair + t * npairs;
+                const int n_first = (tile % g.n_tiles) * bn + static_cast<int>(rank) * bh;
+                const int code_bias = g.w_signed ? 8 : 0;
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int nrow = n_first + gt + 64 * rr;
+                    const int z = (g.w_zero && nrow < p.N) ? __ldg(g.w_zero + nrow) : 0;
+                    z2r[rr] = __half2half2(__ushort_as_half(static_cast<unsigned short>(0x6400 + z + code_bias)));
+                }
+            }
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int r = gt + 64 * rr;
+                if (r >= bh) break;
+                const uint8_t* prow = stg + r * unit_bytes;
+                // the row's 64 codes as eight pairs of byte words (codes 8 j .. 8 j + 3, 8 j + 4 .. 8 j + 7)
+                uint32_t lo4[8], hi4[8];
+                {
+                    uint32_t w[8];  // eight codes per word, byte i = code i (low nibble) | code i + 4 (high nibble)
+                    if (g.w_bits == 4) {
+                        const uint4* src = reinterpret_cast<const uint4*>(prow + (kofs >> 1));
+                        const uint4 v0 = src[0], v1 = src[1];
+                        const uint32_t flip = g.w_signed ? 0x88888888u : 0u;
+                        w[0] = v0.x ^ flip; w[1] = v0.y ^ flip; w[2] = v0.z ^ flip; w[3] = v0.w ^ flip;
+                        w[4] = v1.x ^ flip; w[5] = v1.y ^ flip; w[6] = v1.z ^ flip; w[7] = v1.w ^ flip;
+                    } else {
+                        // bit planes: 16 bytes per bit and 128 codes; the two words of each plane that hold this half
+                        const uint8_t* base = prow + (kofs >> 5) * 4;
+                        const uint2 p0 = *reinterpret_cast<const uint2*>(base);
+                        const uint2 p1 = *reinterpret_cast<const uint2*>(base + 16);
+                        uint2 p2 = make_uint2(0u, 0u);
+                        if (g.w_bits == 3) p2 = *reinterpret_cast<const uint2*>(base + 32);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int sft = j & 3;
+                            const uint32_t a0 = j < 4 ? p0.x : p0.y, a1 = j < 4 ? p1.x : p1.y, a2 = j < 4 ? p2.x : p2.y;
+                            w[j] = ((a0 >> sft) & 0x11111111u) | (((a1 >> sft) & 0x11111111u) << 1) |
+                                   (((a2 >> sft) & 0x11111111u) << 2);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        lo4[j] = w[j] & 0x0F0F0F0Fu;
+                        hi4[j] = (w[j] >> 4) & 0x0F0F0F0Fu;
+                    }
+                }
+                const __half2 z2 = z2r[rr];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    // byte u -> fp16 bits 0x64uu = 1024 + u, two at a time; minus 1024 + zero: exact
+                    uint32_t h[4] = {__byte_perm(lo4[j], 0x64646464u, 0x5140), __byte_perm(lo4[j], 0x64646464u, 0x7362),
+                                     __byte_perm(hi4[j], 0x64646464u, 0x5140), __byte_perm(hi4[j], 0x64646464u, 0x7362)};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const __half2 d = __hsub2(*reinterpret_cast<const __half2*>(&h[q]), z2);
+                        h[q] = *reinterpret_cast<const uint32_t*>(&d);
+                    }
+                    *reinterpret_cast<uint4*>(b_stage + sw128_offset(r, j)) = make_uint4(h[0], h[1], h[2], h[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster(lead_ready);
+                // the packed tile is free once both of its k-blocks are expanded (four warps); the lone k-block of
+                // a tile with an odd number arrives for the missing one too
+                mbar_arrive(bar0 + 8 * (L::EMPTY_P + sp));
+                if ((kbi & 1) == 0 && kbi == nkb - 1) mbar_arrive(bar0 + 8 * (L::EMPTY_P + sp));
+            }
+        }
     } else if (W4 && warp >= 6 && warp < L::HELPER0) {
         // ------------------------------------------------------------ int4 -> int8 (x16) expansion, own half
         // Four groups of two warps; group g takes the k-blocks g, g + 4, ... of the CTA's sequence and owns slot g
@@ -696,7 +836,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
 template <int MODE>
 int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn, int splits,
-                  int num_sms, cudaStream_t stream)
+                  int num_sms, cudaStream_t stream, int w_bits = 0, const int32_t* w_zero = nullptr)
 {
     using L = PairSmem<MODE>;
     auto kernel = pair_gemm_kernel<MODE>;
@@ -706,6 +846,9 @@ int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMa
     g.n_tiles = static_cast<int>(ceil_div(tp.N, bn));
     g.total_tiles = g.n_tiles * static_cast<int>(ceil_div(tp.M, 2 * BM));
     g.splits = splits;
+    g.w_bits = w_bits;
+    g.w_signed = w_zero ? 0 : 1;
+    g.w_zero = w_zero;
     // persistent pairs, or one cluster of `splits` pairs per tile
     const int pairs = splits > 1 ? g.total_tiles : (g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2);
     return launch_pdl_cluster(kernel, dim3(static_cast<unsigned>(2 * splits * pairs)), dim3(L::THREADS), L::TOTAL, stream,
@@ -767,6 +910,16 @@ int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensor
         splits > tp.k_blocks)
         return MIXDQ_ERR_INVALID_ARG;
     return launch_pair_t<2>(ta, tw, ty, tp, bn, splits, num_sms, stream);
+}
+
+int launch_pair_wo(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+                   int w_bits, const int32_t* w_zero, int num_sms, cudaStream_t stream)
+{
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || tp.acc_out || tp.k_blocks < 1)
+        return MIXDQ_ERR_INVALID_ARG;
+    if (w_bits != 2 && w_bits != 3 && w_bits != 4) return MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits <= 3 && !w_zero) return MIXDQ_ERR_UNSUPPORTED;  // bit-plane codes are unsigned
+    return launch_pair_t<3>(ta, tw, ty, tp, bn, 1, num_sms, stream, w_bits, w_zero);
 }
 
 }  // namespace i8

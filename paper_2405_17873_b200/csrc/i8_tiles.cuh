@@ -191,6 +191,15 @@ int pair_cluster_capacity(bool w4, int cluster_ctas);
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
                     int splits, int num_sms, cudaStream_t stream);
 
+// The same kernel on fp16 activations and PACKED weights (2, 3 or 4 bits, device layout), expanded to fp16
+// (code - zero: exact integers) in shared memory by each CTA for its half of the tile: no expanded copy of the
+// weights exists in global memory and no expansion kernel runs.  ta as for launch_pair_f16; tw: byte map of the
+// packed matrix with a box of bn / 2 rows x 16 * w_bits bytes (128 codes = two k-blocks); tp.k_blocks counts
+// blocks of 64 elements; w_zero: per-channel zero-points (device), nullptr for signed codes.  The reduction is
+// never split.
+int launch_pair_wo(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,
+                   int w_bits, const int32_t* w_zero, int num_sms, cudaStream_t stream);
+
 // Fused-quantization form (i8_fq.cu): one kernel per linear layer, fp16 activations in.  tx: fp16 map of X with a
 // box of 128 rows x 64 elements (128-byte swizzle), tw: weight map with a box of bn rows, ty: output map with a
 // 32 x 32 box; tile 128 x bn (bn a multiple of 32, <= 256).

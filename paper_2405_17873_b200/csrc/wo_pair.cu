@@ -10,6 +10,7 @@
 #include <algorithm>
 #include <cmath>
 
+#include "codes.cuh"
 #include "common.cuh"
 #include "engines.h"
 #include "i8_tiles.cuh"
@@ -21,47 +22,6 @@ namespace {
 
 constexpr int BM = i8::BM;
 constexpr int BKE = 64;  // fp16 elements of a k-block (128-byte rows)
-
-// Eight consecutive codes k0 .. k0 + 7 (k0 a multiple of 8) of a row in the device layout, as integers.
-// 8 bits: eight bytes.  4 bits: one 32-bit word, byte j = code j (low nibble) | code j + 4 (high nibble).
-// 2 / 3 bits: blocks of 128 codes, one 16-byte plane per bit; the eight codes' bits sit in ONE 32-bit word of
-// each plane, code j at bit ((k0 % 32) / 8) + {0, 8, 16, 24, 4, 12, 20, 28}[j] (the interleave that lets the
-// register decode of the few-token kernel rebuild 4-bit fields with shifts).
-template <int BITS, bool SIGNED>
-__device__ __forceinline__ void codes8(const uint8_t* __restrict__ row, int k0, int (&c)[8])
-{
-    if (BITS == 8) {
-        const uint2 v = *reinterpret_cast<const uint2*>(row + k0);
-        const uint32_t w[2] = {v.x, v.y};
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t byte = (w[j >> 2] >> (8 * (j & 3))) & 0xffu;
-            c[j] = SIGNED ? static_cast<int>(static_cast<int8_t>(byte)) : static_cast<int>(byte);
-        }
-    } else if (BITS == 4) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(row + (k0 >> 1));
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int nib = static_cast<int>((w >> (8 * (j & 3) + (j >= 4 ? 4 : 0))) & 0xfu);
-            c[j] = (SIGNED && nib >= 8) ? nib - 16 : nib;
-        }
-    } else {
-        const int blk = k0 >> 7, r = k0 & 127;
-        const int t = r >> 5, sft = (r & 31) >> 3;
-        const uint8_t* base = row + blk * 16 * BITS + t * 4;
-        uint32_t w[BITS];
-#pragma unroll
-        for (int p = 0; p < BITS; ++p) w[p] = *reinterpret_cast<const uint32_t*>(base + p * 16) >> sft;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int pos = (j < 4) ? 8 * j : 8 * (j - 4) + 4;
-            int v = 0;
-#pragma unroll
-            for (int p = 0; p < BITS; ++p) v |= static_cast<int>((w[p] >> pos) & 1u) << p;
-            c[j] = v;
-        }
-    }
-}
 
 // out[n, k] = half(code[n, k] - zero[n]) for k < K, 0 for K <= k < ldw.  One thread per eight elements.
 template <int BITS, bool SIGNED>
@@ -168,25 +128,7 @@ int run_pair(const Params& p, int amode, const void* packed, int w_bits, cudaStr
 {
     const int num_sms = sm_count();
     if (num_sms <= 0) return MIXDQ_ERR_CUDA;
-    // 1. the layer's weights as fp16 integers
-    __half* wexp = static_cast<__half*>(p.workspace);
-    const int ldw = static_cast<int>(round_up(p.K, 8));
-    const long long pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
-    const bool is_signed = p.w_zero == nullptr;
-    int rc = MIXDQ_ERR_UNSUPPORTED;
-    if (w_bits == 8)
-        rc = is_signed ? launch_expand<8, true>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream)
-                       : launch_expand<8, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
-    else if (w_bits == 4)
-        rc = is_signed ? launch_expand<4, true>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream)
-                       : launch_expand<4, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
-    else if (w_bits == 3 && !is_signed)
-        rc = launch_expand<3, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
-    else if (w_bits == 2 && !is_signed)
-        rc = launch_expand<2, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
-    if (rc != MIXDQ_OK) return rc;
-
-    // 2. the GEMM
+    int rc = MIXDQ_OK;
     i8::TmaParams tp{};
     tp.M = p.M;
     tp.N = p.N;
@@ -222,14 +164,45 @@ int run_pair(const Params& p, int amode, const void* packed, int w_bits, cudaStr
     if (rc != MIXDQ_OK) return rc;
     int splits = 1;
     const int bn = pick_tile(p.M, p.N, tp.k_blocks, num_sms, &splits);
-    rc = encode_tmap_2d_f16(&tw, wexp, static_cast<uint64_t>(p.K), static_cast<uint64_t>(p.N), static_cast<uint64_t>(ldw),
-                            BKE, static_cast<uint32_t>(bn / 2));
-    if (rc != MIXDQ_OK) return rc;
     if (tp.tma_store) {
         rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
                                 static_cast<uint64_t>(p.ldy), 32, 32, true);
         if (rc != MIXDQ_OK) return rc;
     }
+    const long long pitch = row_pitch_bytes(p.K, w_bits, MIXDQ_LAYOUT_DEVICE);
+    // Unsplit reductions: the packed weights go to the GEMM kernel as they are and each CTA expands its half of a
+    // weight tile in shared memory (a k-block of a convolution must be a whole block of the flattened reduction
+    // index, i.e. Cin a multiple of 64).  Split reductions (few tiles, long reductions) and 8-bit weights (whose packed
+    // tiles would take the shared memory of two activation slots) keep the expansion pass, and so do layers of more
+    // than 2048 rows: every 256-row tile expands its weights again, and the in-kernel expansion makes the main loop
+    // about 1.3 times slower (measured: 16384 x 640 x 5760 104 against 79 us, 4096 x 640 x 2560 19.0 against 15.6,
+    // while 1024 x 1280 x 1280 gains 0.5 us and 1024 x 1280 x 5120 1.0 us from the launch it saves).
+    if (splits == 1 && w_bits <= 4 && p.M <= 2048 && (amode != A_CONV3 || p.Cin % BKE == 0)) {
+        rc = encode_tmap_2d_u8(&tw, packed, static_cast<uint64_t>(pitch), static_cast<uint64_t>(p.N), static_cast<uint64_t>(pitch),
+                               static_cast<uint32_t>(16 * w_bits), static_cast<uint32_t>(bn / 2), false);
+        if (rc != MIXDQ_OK) return rc;
+        return i8::launch_pair_wo(ta, tw, ty, tp, bn, w_bits, p.w_zero, num_sms, stream);
+    }
+    // the layer's weights as fp16 integers, once per call
+    __half* wexp = static_cast<__half*>(p.workspace);
+    const int ldw = static_cast<int>(round_up(p.K, 8));
+    const bool is_signed = p.w_zero == nullptr;
+    rc = MIXDQ_ERR_UNSUPPORTED;
+    if (w_bits == 8)
+        rc = is_signed ? launch_expand<8, true>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream)
+                       : launch_expand<8, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
+    else if (w_bits == 4)
+        rc = is_signed ? launch_expand<4, true>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream)
+                       : launch_expand<4, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
+    else if (w_bits == 3 && !is_signed)
+        rc = launch_expand<3, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
+    else if (w_bits == 2 && !is_signed)
+        rc = launch_expand<2, false>(packed, pitch, p.N, p.K, ldw, p.w_zero, wexp, stream);
+    if (rc != MIXDQ_OK) return rc;
+
+    rc = encode_tmap_2d_f16(&tw, wexp, static_cast<uint64_t>(p.K), static_cast<uint64_t>(p.N), static_cast<uint64_t>(ldw),
+                            BKE, static_cast<uint32_t>(bn / 2));
+    if (rc != MIXDQ_OK) return rc;
     return i8::launch_pair_f16(ta, tw, ty, tp, bn, splits, num_sms, stream);
 }
 
