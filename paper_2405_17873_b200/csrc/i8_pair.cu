@@ -167,9 +167,12 @@ struct PairSmem {
     // Weight-only: a packed tile serves two consecutive k-blocks, i.e. two of the four expansion groups; with an
     // even number of packed slots a slot always belongs to the same two groups, which then meet every phase of its
     // barrier.
-    static constexpr int AS = W4 ? 5 : 6;
+    static constexpr int AS = W4 ? 4 : 6;
     static constexpr int ES = PACKED ? 4 : 6;
-    static constexpr int PS = W4 ? 6 : (WO ? 4 : 0);
+    static constexpr int PS = W4 ? 8 : (WO ? 4 : 0);
+    // Rings of equal depth move in lockstep: the commit that frees the activation slot of a k-block frees its weight
+    // slot too (one commit per k-block instead of two; measured 4 to 7 % on the large int4 convolutions).
+    static constexpr bool ONE_COMMIT = !PACKED || AS == ES;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + AS * A_BYTES;
     static constexpr int OFF_P = OFF_B + ES * B_BYTES;
@@ -475,7 +478,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         mbar_arrive(tile_go);
                     }
                     tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa), pair_mask);
-                    if (PACKED) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
+                    if (!L::ONE_COMMIT) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
                     sa += 2;
                     if (sa >= static_cast<uint32_t>(L::AS)) {
                         sa -= L::AS;
@@ -620,7 +623,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const uint32_t sp = useq % PS, rp = useq / PS;
             const uint8_t* stg = sP + sp * L::P_BYTES;
             bool ok = mbar_wait(bar0 + 8 * (L::FULL_P + sp), rp & 1, s_abort);
-            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * (L::EMPTY_B + group), (n & 1) ^ 1, s_abort);
+            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * ((L::ONE_COMMIT ? L::EMPTY_A : L::EMPTY_B) + group), (n & 1) ^ 1, s_abort);
             if (!__all_sync(0xffffffffu, ok)) break;  // the warp leaves together
             const int kofs = (kbi & 1) * 64;  // which half of the packed tile's 128 codes
             if (t != z_tile) {
@@ -715,7 +718,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const uint32_t sp = static_cast<uint32_t>(it) % PS, rp = static_cast<uint32_t>(it) / PS;
             const uint8_t* stg = sP + sp * L::P_BYTES;
             bool ok = mbar_wait(bar0 + 8 * (L::FULL_P + sp), rp & 1, s_abort);
-            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * (L::EMPTY_B + group), (n & 1) ^ 1, s_abort);
+            if (ok && n > 0) ok = mbar_wait(bar0 + 8 * ((L::ONE_COMMIT ? L::EMPTY_A : L::EMPTY_B) + group), (n & 1) ^ 1, s_abort);
             if (!__all_sync(0xffffffffu, ok)) break;  // the warp leaves together
             // all loads first: the compiler cannot move a load above a store to the other ring by itself
             uint4 wv[8];
