@@ -147,10 +147,13 @@ constexpr int PAIR_BN_MAX = 256;
 constexpr int ACC_COLS = 256;  // tensor-memory columns of one accumulator (the widest tile)
 
 // MODE: 0 = int8 weights, 1 = int4 weights (expanded in shared memory), 2 = fp16 operands (kind::f16), 3 = fp16
-// activations and packed 2- / 3- / 4- / 8-bit weights expanded to fp16 (code - zero) in shared memory
+// activations and packed 2- / 3- / 4-bit weights expanded to fp16 (code - zero) in shared memory; 4 / 5 = modes 0 / 1
+// with two branches of k-blocks and an accumulator each (instances of their own, so that the one-branch kernels
+// carry none of that code)
 template <int MODE>
 struct PairSmem {
-    static constexpr bool W4 = MODE == 1;
+    static constexpr bool W4 = MODE == 1 || MODE == 5;
+    static constexpr bool TWO = MODE >= 4;  // two-branch instances (shortcut-splitting): 4 = int8, 5 = int4 weights
     static constexpr bool F16 = MODE == 2 || MODE == 3;
     static constexpr bool WO = MODE == 3;
     static constexpr bool PACKED = W4 || WO;  // a ring of packed weight tiles and expansion warps
@@ -188,7 +191,8 @@ struct PairSmem {
     static constexpr int ACC_FULL = EMPTY_P + PS;     // [2]
     static constexpr int ACC_EMPTY = ACC_FULL + 2;    // [2]
     static constexpr int TILE_GO = ACC_EMPTY + 2;     // leader: the first issuer has issued k-block 0 of a tile
-    static constexpr int NUM_BARS = TILE_GO + 1;
+    static constexpr int TILE_GO2 = TILE_GO + 1;      // leader, two-branch mode: the second branch's first k-block is issued
+    static constexpr int NUM_BARS = TILE_GO2 + 1;
     static constexpr int OFF_BARS = RINGS_END;
     static constexpr int OFF_COMB = (OFF_BARS + NUM_BARS * 8 + 15) & ~15;  // [2][PAIR_BN_MAX] floats
     static constexpr int OFF_BIAS = OFF_COMB + 2 * PAIR_BN_MAX * 4;
@@ -215,6 +219,14 @@ struct PairArgs {
     int w_bits;
     int w_signed;
     const int32_t* w_zero;
+    // two-branch mode (shortcut-splitting, Sec. 4.1; int8 modes, one tile per pair): kb_lo > 0 = the first kb_lo
+    // k-blocks are the first branch (tmap_a / tmap_w, TmaParams' geometry and act_scale, accumulator 0), the others
+    // the second branch (tmap_a2 / tmap_w2, the geometry below and *act_scale2, accumulator 1); the epilogue
+    // stores (s_lo * acc_lo + s_hi * acc_hi) * s_w[n] + bias[n].  acc_out2: the second branch's sums (parity hook).
+    int kb_lo;
+    int cblocks2, Cin2;
+    const float* act_scale2;
+    int32_t* acc_out2;
 };
 
 // Grid (2 * splits * (pairs or tiles), 1, 1) with clusters of 2 * splits CTAs along x: CTAs 2 i and 2 i + 1 of a
@@ -225,7 +237,8 @@ struct PairArgs {
 template <int MODE>
 __global__ void __launch_bounds__(PairSmem<MODE>::THREADS, 1)
 pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                 const __grid_constant__ CUtensorMap tmap_y, const TmaParams p, const PairArgs g)
+                 const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_a2,
+                 const __grid_constant__ CUtensorMap tmap_w2, const TmaParams p, const PairArgs g)
 {
     using L = PairSmem<MODE>;
     constexpr bool W4 = L::W4;
@@ -258,6 +271,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int bn = g.bn, bh = g.bn >> 1;
     const int my_tiles = splits > 1 ? 1 : (g.total_tiles - pair + npairs - 1) / npairs;
     const uint16_t pair_mask = static_cast<uint16_t>(3u << leader_rank);  // the two CTAs of this pair
+    const int kb_lo = L::TWO ? g.kb_lo : 0;  // > 0: two branches, two accumulators, one tile per pair
 
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t a0 = smem_u32(smem + L::OFF_A), b0 = smem_u32(sB), p0 = smem_u32(smem + L::OFF_P);
@@ -283,11 +297,16 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             mbar_init(bar0 + 8 * (L::ACC_EMPTY + b), 16);  // eight epilogue warps of each CTA
         }
         mbar_init(bar0 + 8 * L::TILE_GO, 1);
+        mbar_init(bar0 + 8 * L::TILE_GO2, 1);
         *s_abort = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmap_a);
         tma_prefetch_desc(&tmap_w);
         if (p.tma_store) tma_prefetch_desc(&tmap_y);
+        if (kb_lo > 0) {
+            tma_prefetch_desc(&tmap_a2);
+            tma_prefetch_desc(&tmap_w2);
+        }
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(s_tmem), 2 * ACC_COLS);
@@ -324,7 +343,15 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     kh = tap / 3;
                     kw = tap - 3 * kh;
                 }
+                const CUtensorMap* map = &tmap_a;
+                int cblocks = p.cblocks;
                 for (int i = 0; i < nkb; ++i) {
+                    if (kb_lo > 0 && i == kb_lo) {  // second branch: its own map, from its first k-block
+                        map = &tmap_a2;
+                        cblocks = g.cblocks2;
+                        cb = kh = kw = 0;
+                        xa = 0;
+                    }
                     if (!mbar_wait(bar0 + 8 * (L::EMPTY_A + s), par, s_abort)) {
                         ok = false;
                         break;
@@ -332,9 +359,9 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (leader) mbar_arrive_expect_tx(bar0 + 8 * (L::FULL_A + s), 2 * L::A_BYTES);
                     const uint32_t full = lead_bar0 + 8 * (L::FULL_A + s);
                     if (p.conv) {
-                        tma_load_4d_pair(a0 + s * L::A_BYTES, &tmap_a, cb * BKE, p.stride * wo0 + kw - 1 + p.pad,
+                        tma_load_4d_pair(a0 + s * L::A_BYTES, map, cb * BKE, p.stride * wo0 + kw - 1 + p.pad,
                                          p.stride * ho0 + kh - 1 + p.pad, img_b, full);
-                        if (++cb == p.cblocks) {
+                        if (++cb == cblocks) {
                             cb = 0;
                             if (++kw == 3) {
                                 kw = 0;
@@ -342,7 +369,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             }
                         }
                     } else {
-                        tma_load_2d_pair(a0 + s * L::A_BYTES, &tmap_a, xa, m0, full);
+                        tma_load_2d_pair(a0 + s * L::A_BYTES, map, xa, m0, full);
                         xa += BKE;
                     }
                     if (++s == L::AS) {
@@ -395,7 +422,16 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     cb = kb_begin - tap * p.cblocks;
                     kx_tap = tap * p.Cin;  // first reduction index of the filter tap
                 }
+                const CUtensorMap* map = &tmap_w;
+                int cblocks = p.cblocks, cin = p.Cin;
                 for (int i = 0; i < nkb; ++i) {
+                    if (kb_lo > 0 && i == kb_lo) {  // second branch: its own packed matrix, from its first k-block
+                        map = &tmap_w2;
+                        cblocks = g.cblocks2;
+                        cin = g.Cin2;
+                        cb = kx_tap = 0;
+                        xb = 0;
+                    }
                     // W8: the commit that frees the activation slot frees the weight slot (the rings move in lockstep)
                     if (!mbar_wait(bar0 + 8 * ((W4 ? L::EMPTY_P : L::EMPTY_A) + s), par, s_abort)) {
                         ok = false;
@@ -405,9 +441,9 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (p.conv) {
                         const int kx = kx_tap + cb * BKE;
                         x = W4 ? kx / 2 : kx;
-                        if (++cb == p.cblocks) {
+                        if (++cb == cblocks) {
                             cb = 0;
-                            kx_tap += p.Cin;
+                            kx_tap += cin;
                         }
                     }
                     xb += ROW_STEP;
@@ -415,10 +451,10 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         // packed rows are consumed inside this CTA: a barrier of its own
                         const uint32_t full = bar0 + 8 * (L::FULL_P + s);
                         mbar_arrive_expect_tx(full, static_cast<uint32_t>(bh * ROW_BYTES));
-                        tma_load_2d(p0 + s * L::P_BYTES, &tmap_w, x, n0, full);
+                        tma_load_2d(p0 + s * L::P_BYTES, map, x, n0, full);
                     } else {
                         if (leader) mbar_arrive_expect_tx(bar0 + 8 * (L::READY_B + s), static_cast<uint32_t>(bn * ROW_BYTES));
-                        tma_load_2d_pair(b0 + s * L::B_BYTES, &tmap_w, x, n0, lead_bar0 + 8 * (L::READY_B + s));
+                        tma_load_2d_pair(b0 + s * L::B_BYTES, map, x, n0, lead_bar0 + 8 * (L::READY_B + s));
                     }
                     if (++s == R) {
                         s = 0;
@@ -465,17 +501,29 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         ok = false;
                         break;
                     }
+                    // two-branch mode: the second branch's k-blocks go to the other accumulator, whose overwriting
+                    // MMA (first of k-block kb_lo) must precede the other thread's first addition to it
+                    const bool second = kb_lo > 0 && i >= kb_lo;
+                    if (second && i == kb_lo + 1 && !mbar_wait(bar0 + 8 * L::TILE_GO2, 0, s_abort)) {
+                        ok = false;
+                        break;
+                    }
                     tc_fence_after_sync();
                     const uint64_t a_desc = a_desc0 + sa * (L::A_BYTES >> 4);
                     const uint64_t b_desc = b_desc0 + se * (L::B_BYTES >> 4);
+                    const uint32_t acc_i = second ? tmem_base + ACC_COLS : acc;
                     // four instructions of 32 bytes along the reduction: 32 int8 or 16 fp16 elements each
-                    mma_pair<F16>(acc, a_desc, b_desc, idesc, i != 0);
+                    mma_pair<F16>(acc_i, a_desc, b_desc, idesc, i != 0 && !(second && i == kb_lo));
 #pragma unroll
-                    for (int k = 1; k < BK / 32; ++k) mma_pair<F16>(acc, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
+                    for (int k = 1; k < BK / 32; ++k) mma_pair<F16>(acc_i, a_desc + 2 * k, b_desc + 2 * k, idesc, 1u);
                     if (i == 0 && nkb > 1) {
                         // the overwriting MMA is in the pipe's queue: the other thread may add to the accumulator
                         tc_fence_before_sync();
                         mbar_arrive(tile_go);
+                    }
+                    if (second && i == kb_lo) {
+                        tc_fence_before_sync();
+                        mbar_arrive(bar0 + 8 * L::TILE_GO2);
                     }
                     tc_commit_pair(bar0 + 8 * (L::EMPTY_A + sa), pair_mask);
                     if (!L::ONE_COMMIT) tc_commit_pair(bar0 + 8 * (L::EMPTY_B + se), pair_mask);
@@ -528,6 +576,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 }
                 comb[j] = c;
                 bias[j] = b;
+                // two-branch mode (one tile): the second table holds the second branch's factors
+                if (kb_lo > 0) s_comb[PAIR_BN_MAX + j] = (n < p.N && p.w_scale) ? __ldg(g.act_scale2) * __ldg(p.w_scale + n) : 0.f;
             }
             if (ok) ok = mbar_wait(bar0 + 8 * (L::ACC_FULL + buf), use & 1, s_abort);
             tc_fence_after_sync();
@@ -584,12 +634,25 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             }
                         }
                     }
+                    if (kb_lo > 0 && g.acc_out2) {
+                        tmem_ld_32x32(acc + ACC_COLS + c0, r);
+                        tmem_ld_wait();
+                        if (m < p.M) {
+                            int32_t* dst = g.acc_out2 + static_cast<long long>(m) * p.N + n0 + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + c0 + j < p.N) dst[j] = W4 ? (static_cast<int32_t>(r[j]) >> 4) : static_cast<int32_t>(r[j]);
+                        }
+                    }
                 }
             }
             if (splits == 1 && p.Y && c_count > 0) {
                 if (F16)
                     store_rows32_f32(acc + c_begin, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
                                      m0 + lg * 32, n0 + c_begin, lane);
+                else if (kb_lo > 0)
+                    store_rows32_two<W4>(acc + c_begin, ACC_COLS, c_count, comb + c_begin, s_comb + PAIR_BN_MAX + c_begin,
+                                         bias + c_begin, stage, p, &tmap_y, m0 + lg * 32, n0 + c_begin, lane);
                 else
                     store_rows32_dispatch<W4>(acc + c_begin, 0, c_count, comb + c_begin, bias + c_begin, stage, p, &tmap_y,
                                               m0 + lg * 32, n0 + c_begin, lane);
@@ -839,7 +902,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
 template <int MODE>
 int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn, int splits,
-                  int num_sms, cudaStream_t stream, int w_bits = 0, const int32_t* w_zero = nullptr)
+                  int num_sms, cudaStream_t stream, int w_bits = 0, const int32_t* w_zero = nullptr,
+                  const PairBranch* second = nullptr)
 {
     using L = PairSmem<MODE>;
     auto kernel = pair_gemm_kernel<MODE>;
@@ -852,10 +916,23 @@ int launch_pair_t(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMa
     g.w_bits = w_bits;
     g.w_signed = w_zero ? 0 : 1;
     g.w_zero = w_zero;
-    // persistent pairs, or one cluster of `splits` pairs per tile
-    const int pairs = splits > 1 ? g.total_tiles : (g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2);
+    g.kb_lo = 0;
+    g.cblocks2 = g.Cin2 = 0;
+    g.act_scale2 = nullptr;
+    g.acc_out2 = nullptr;
+    if (second) {
+        g.kb_lo = second->kb_first;
+        g.cblocks2 = second->cblocks;
+        g.Cin2 = second->Cin;
+        g.act_scale2 = second->act_scale;
+        g.acc_out2 = second->acc_out;
+    }
+    // persistent pairs; one cluster of `splits` pairs per tile; two-branch mode: one pair per tile (both
+    // accumulators belong to the tile)
+    const int pairs = (splits > 1 || second) ? g.total_tiles : (g.total_tiles < num_sms / 2 ? g.total_tiles : num_sms / 2);
     return launch_pdl_cluster(kernel, dim3(static_cast<unsigned>(2 * splits * pairs)), dim3(L::THREADS), L::TOTAL, stream,
-                              static_cast<unsigned>(2 * splits), 1u, ta, tw, ty, tp, g);
+                              static_cast<unsigned>(2 * splits), 1u, ta, tw, ty, second ? *second->ta : ta,
+                              second ? *second->tw : tw, tp, g);
 }
 
 }  // namespace
@@ -904,6 +981,17 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap&
         return MIXDQ_ERR_INVALID_ARG;
     return w4 ? launch_pair_t<1>(ta, tw, ty, tp, bn, splits, num_sms, stream)
               : launch_pair_t<0>(ta, tw, ty, tp, bn, splits, num_sms, stream);
+}
+
+int launch_pair_two(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
+                    const PairBranch& second, int num_sms, cudaStream_t stream)
+{
+    // tp.k_blocks counts both branches' k-blocks; a split reduction and asymmetric activations are not supported
+    if (bn < 32 || bn > PAIR_BN_MAX || bn % 32 != 0 || num_sms < 2 || second.kb_first < 1 || second.kb_first >= tp.k_blocks ||
+        !second.ta || !second.tw || !second.act_scale || tp.act_zero || tp.addend || tp.bos)
+        return MIXDQ_ERR_INVALID_ARG;
+    return w4 ? launch_pair_t<5>(ta, tw, ty, tp, bn, 1, num_sms, stream, 0, nullptr, &second)
+              : launch_pair_t<4>(ta, tw, ty, tp, bn, 1, num_sms, stream, 0, nullptr, &second);
 }
 
 int launch_pair_f16(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, int bn,

@@ -60,23 +60,30 @@ __device__ __forceinline__ float acc_to_float(uint32_t r)
 constexpr int EPI32_ROW = 80;
 constexpr int EPI32_TILE = 32 * EPI32_ROW;  // 2560: a multiple of 512, the period of the 64-byte swizzle
 
-template <bool W4, bool SMALL, bool TMA, bool F32 = false>
+// TWO: the second accumulator holds the sums of the second branch of a shortcut-split layer (Sec. 4.1), with
+// per-column factors comb2 of its own: y = acc2 * comb2[c] + (acc * comb[c] + bias[c]).
+template <bool W4, bool SMALL, bool TMA, bool F32 = false, bool TWO = false>
 __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
                                                        const float* bias, uint8_t* stage, const TmaParams& p,
-                                                       const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+                                                       const CUtensorMap* tmap_y, int m_first, int n0, int lane,
+                                                       const float* comb2 = nullptr)
 {
     const bool vec = ((p.ldy & 7) == 0) && ((p.N & 7) == 0);
     if (TMA && m_first >= p.M) return;  // uniform across the warp
     for (int c0 = 0; c0 < ncols; c0 += 32) {
         if (n0 + c0 >= p.N) break;  // uniform across the warp
         uint32_t r[32];
+        uint32_t r2[TWO ? 32 : 1];
         tmem_ld_32x32(acc + c0, r);
-        if (acc2_off) {
-            uint32_t r2[32];
-            tmem_ld_32x32(acc + acc2_off + c0, r2);
+        if (TWO) {
+            tmem_ld_32x32(acc + acc2_off + c0, reinterpret_cast<uint32_t(&)[32]>(r2));
+            tmem_ld_wait();
+        } else if (acc2_off) {
+            uint32_t rs[32];
+            tmem_ld_32x32(acc + acc2_off + c0, rs);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] += r2[j];
+            for (int j = 0; j < 32; ++j) r[j] += rs[j];
         } else {
             tmem_ld_wait();
         }
@@ -86,8 +93,32 @@ __device__ __forceinline__ void store_rows32_from_tmem(uint32_t acc, uint32_t ac
             const int c = c0 + j;
             const float4 ca = *reinterpret_cast<const float4*>(comb + c);
             const float4 cb = *reinterpret_cast<const float4*>(comb + c + 4);
-            const float4 ba = *reinterpret_cast<const float4*>(bias + c);
-            const float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+            float4 ba = *reinterpret_cast<const float4*>(bias + c);
+            float4 bb = *reinterpret_cast<const float4*>(bias + c + 4);
+            if (TWO) {
+                // the first branch's term joins the bias; the second branch's sums take the place of `r` below
+                const float4 da = *reinterpret_cast<const float4*>(comb2 + c);
+                const float4 db = *reinterpret_cast<const float4*>(comb2 + c + 4);
+                ba.x = fmaf(acc_to_float<W4, SMALL, F32>(r[j]), ca.x, ba.x);
+                ba.y = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 1]), ca.y, ba.y);
+                ba.z = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 2]), ca.z, ba.z);
+                ba.w = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 3]), ca.w, ba.w);
+                bb.x = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 4]), cb.x, bb.x);
+                bb.y = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 5]), cb.y, bb.y);
+                bb.z = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 6]), cb.z, bb.z);
+                bb.w = fmaf(acc_to_float<W4, SMALL, F32>(r[j + 7]), cb.w, bb.w);
+                __half2 hv[4];
+                hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j : 0]), da.x, ba.x),
+                                          fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 1 : 0]), da.y, ba.y));
+                hv[1] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 2 : 0]), da.z, ba.z),
+                                          fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 3 : 0]), da.w, ba.w));
+                hv[2] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 4 : 0]), db.x, bb.x),
+                                          fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 5 : 0]), db.y, bb.y));
+                hv[3] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 6 : 0]), db.z, bb.z),
+                                          fmaf(acc_to_float<W4, SMALL, F32>(r2[TWO ? j + 7 : 0]), db.w, bb.w));
+                out[j >> 3] = *reinterpret_cast<const uint4*>(hv);
+                continue;
+            }
             __half2 hv[4];
             hv[0] = __floats2half2_rn(fmaf(acc_to_float<W4, SMALL, F32>(r[j]), ca.x, ba.x),
                                       fmaf(acc_to_float<W4, SMALL, F32>(r[j + 1]), ca.y, ba.y));
@@ -150,6 +181,20 @@ __device__ __forceinline__ void store_rows32_f32(uint32_t acc, int ncols, const 
                                                  uint8_t* stage, const TmaParams& p, const CUtensorMap* tmap_y,
                                                  int m_first, int n0, int lane);
 
+// The two-scale form (see store_rows32_from_tmem, TWO).
+template <bool W4>
+__device__ __forceinline__ void store_rows32_two(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
+                                                 const float* comb2, const float* bias, uint8_t* stage, const TmaParams& p,
+                                                 const CUtensorMap* tmap_y, int m_first, int n0, int lane)
+{
+    if (p.tma_store)
+        store_rows32_from_tmem<W4, false, true, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0,
+                                                             lane, comb2);
+    else
+        store_rows32_from_tmem<W4, false, false, false, true>(acc, acc2_off, ncols, comb, bias, stage, p, tmap_y, m_first, n0,
+                                                              lane, comb2);
+}
+
 template <bool W4>
 __device__ __forceinline__ void store_rows32_dispatch(uint32_t acc, uint32_t acc2_off, int ncols, const float* comb,
                                                       const float* bias, uint8_t* stage, const TmaParams& p,
@@ -185,6 +230,23 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap&
                 int splits, int num_sms, cudaStream_t stream);
 // Clusters of `cluster_ctas` CTAs of that kernel the current device can hold at once (0 on error).
 int pair_cluster_capacity(bool w4, int cluster_ctas);
+// Two-branch form of the same kernel for a shortcut-split layer (Sec. 4.1: the input is a concatenation whose two
+// parts keep an activation scale each): ONE launch, one pair per tile; the first `kb_first` k-blocks of a tile are the
+// first branch (ta, tw, tp's convolution geometry and tp.act_scale) and accumulate in one accumulator, the others the
+// second branch (the maps, geometry and scale below) in the other; the epilogue stores
+// y = (s_first * acc_first + s_second * acc_second) * w_scale[n] + bias[n].  tp.acc_out / acc_out: the two branches'
+// int32 sums (parity hook).  tp.k_blocks = k-blocks of both branches.
+struct PairBranch {
+    const CUtensorMap* ta;
+    const CUtensorMap* tw;
+    int kb_first;            // k-blocks of the FIRST branch
+    int cblocks, Cin;        // convolution: k-blocks per filter tap and channels of the second branch
+    const float* act_scale;  // activation scale of the second branch (device)
+    int32_t* acc_out;        // its sums [M, N], or nullptr
+};
+int launch_pair_two(const CUtensorMap& ta, const CUtensorMap& tw, const CUtensorMap& ty, const TmaParams& tp, bool w4, int bn,
+                    const PairBranch& second, int num_sms, cudaStream_t stream);
+
 // The same kernel on fp16 operands (kind::f16, fp32 accumulators) for the weight-only layers: ta an fp16 map with a
 // box of 128 rows x 64 elements, tw the map of the layer's weights expanded to fp16 (q - zero) with a box of
 // bn / 2 rows x 64 elements; tp.k_blocks counts blocks of 64 elements and tp.act_scale is unused.

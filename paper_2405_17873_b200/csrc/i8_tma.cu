@@ -1519,6 +1519,80 @@ int run_tma_split(const Params& p, int amode, int split_at, const void* packed_l
                         p.X, ldx, in_rows, row_len, split_at, scale_lo, scale_hi, aq_lo, aq_hi);
     if (rc != MIXDQ_OK) return rc;
 
+    // One launch where the two-CTA form suits the layer: both branches' k-blocks in one kernel, an accumulator per
+    // branch in tensor memory, the two-scale epilogue straight from there (no int32 round trip through memory).
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MIXDQ_ERR_CUDA;
+    const bool w4 = w_bits == 4;
+    const int c_lo = split_at, c_hi = row_len - split_at;
+    const int kb_lo = static_cast<int>(conv ? 9 * ceil_div(c_lo, BK) : ceil_div(c_lo, BK));
+    const int kb_hi = static_cast<int>(conv ? 9 * ceil_div(c_hi, BK) : ceil_div(c_hi, BK));
+    const int pair_bn = plan_pair_tile(p.M, p.N, kb_lo + kb_hi, w4, num_sms, nullptr);
+    if (pair_bn > 0) {
+        CUtensorMap ta[2], tw[2], ty{};
+        const int8_t* aq[2] = {aq_lo, aq_hi};
+        const void* pk[2] = {packed_lo, packed_hi};
+        const int cin[2] = {c_lo, c_hi};
+        for (int b = 0; b < 2; ++b) {
+            const int64_t kb = conv ? 9ll * cin[b] : cin[b];
+            const int64_t pitch = row_pitch_bytes(kb, w_bits, MIXDQ_LAYOUT_DEVICE);
+            if (conv) {
+                int Wb, Hb, Bb;
+                if (!conv_box(p.Ho, p.Wo, &Wb, &Hb, &Bb)) return MIXDQ_ERR_UNSUPPORTED;
+                const uint64_t dims[4] = {static_cast<uint64_t>(cin[b]), static_cast<uint64_t>(p.W), static_cast<uint64_t>(p.H),
+                                          static_cast<uint64_t>(p.batch)};
+                const uint64_t strides[3] = {static_cast<uint64_t>(cin[b]), static_cast<uint64_t>(cin[b]) * p.W,
+                                             static_cast<uint64_t>(cin[b]) * p.W * p.H};
+                const uint32_t box[4] = {BK, static_cast<uint32_t>(Wb), static_cast<uint32_t>(Hb), static_cast<uint32_t>(Bb)};
+                rc = encode_tmap_4d_u8(&ta[b], aq[b], dims, strides, box, static_cast<uint32_t>(p.stride));
+            } else {
+                rc = encode_tmap_2d_u8(&ta[b], aq[b], static_cast<uint64_t>(cin[b]), static_cast<uint64_t>(p.M),
+                                       static_cast<uint64_t>(cin[b]), BK, BM, true);
+            }
+            if (rc != MIXDQ_OK) return rc;
+            if (w4)
+                rc = encode_tmap_2d_u8(&tw[b], pk[b], static_cast<uint64_t>(pitch), p.N, pitch, BK / 2, pair_bn / 2, false);
+            else
+                rc = encode_tmap_2d_u8(&tw[b], pk[b], static_cast<uint64_t>(kb), p.N, pitch, BK, pair_bn / 2, true);
+            if (rc != MIXDQ_OK) return rc;
+        }
+        TmaParams tp{};
+        tp.M = p.M;
+        tp.N = p.N;
+        tp.k_blocks = kb_lo + kb_hi;
+        tp.act_scale = scale_lo;
+        tp.w_scale = p.w_scale;
+        tp.bias = p.bias;
+        tp.Y = p.Y;
+        tp.ldy = p.ldy;
+        tp.acc_out = p.Y ? nullptr : acc_lo_out;
+        tp.status = p.status;
+        tp.small_acc = 0;
+        tp.tma_store = p.Y && p.ldy % 8 == 0 && (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
+        if (conv) {
+            tp.conv = 1;
+            tp.stride = p.stride;
+            tp.cblocks = static_cast<int>(ceil_div(c_lo, BK));
+            tp.Cin = c_lo;
+            tp.HoWo = p.Ho * p.Wo;
+            tp.Wo = p.Wo;
+        }
+        if (tp.tma_store) {
+            rc = encode_tmap_2d_f16(&ty, p.Y, static_cast<uint64_t>(p.N), static_cast<uint64_t>(p.M),
+                                    static_cast<uint64_t>(p.ldy), 32, 32, true);
+            if (rc != MIXDQ_OK) return rc;
+        }
+        PairBranch second{};
+        second.ta = &ta[1];
+        second.tw = &tw[1];
+        second.kb_first = kb_lo;
+        second.cblocks = conv ? static_cast<int>(ceil_div(c_hi, BK)) : 0;
+        second.Cin = conv ? c_hi : 0;
+        second.act_scale = scale_hi;
+        second.acc_out = p.Y ? nullptr : acc_hi_out;
+        return launch_pair_two(ta[0], tw[0], ty, tp, w4, pair_bn, second, num_sms, stream);
+    }
+
     Params q = p;
     q.Y = nullptr;
     q.bias = nullptr;

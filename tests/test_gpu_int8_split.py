@@ -127,6 +127,31 @@ def test_split_conv_parity(bits, B, H, W_, C_lo, C_hi, N, stride):
     _run_conv(B, H, W_, C_lo, C_hi, N, bits, stride, seed=H + C_lo + N)
 
 
+def _kb(c):
+    return (c + 127) // 128
+
+
+# Layers large enough for the two-CTA form run both branches in ONE kernel (an accumulator per branch in tensor
+# memory, two-scale epilogue): channel counts that are no multiples of 128 (the last k-block of a tap reads past
+# the branch), unequal halves, stride 2, ragged rows and columns.
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("B,H,W_,C_lo,C_hi,N,stride", [(4, 64, 64, 160, 96, 328, 1), (8, 64, 64, 96, 160, 320, 2),
+                                                       (5, 32, 32, 320, 320, 648, 1)])
+def test_split_conv_in_one_kernel(bits, B, H, W_, C_lo, C_hi, N, stride):
+    Ho = (H - 1) // stride + 1
+    rows, cols = mixdq.int8_tile_plan(B * Ho * Ho, N, 9 * (_kb(C_lo) + _kb(C_hi)), bits)
+    assert rows == 256, (rows, cols)
+    _run_conv(B, H, W_, C_lo, C_hi, N, bits, stride, seed=H + C_lo + N + 7)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,C_lo,C_hi,N", [(5567, 400, 384, 776), (16384, 320, 320, 320), (4458, 1296, 656, 648)])
+def test_split_linear_in_one_kernel(bits, M, C_lo, C_hi, N):
+    rows, cols = mixdq.int8_tile_plan(M, N, _kb(C_lo) + _kb(C_hi), bits)
+    assert rows == 256, (rows, cols)
+    _run_linear(M, C_lo, C_hi, N, bits, seed=M + C_lo + N + 7)
+
+
 def test_split_argument_errors():
     X = dev(synth.normal_f16((64, 64), 1.0, seed=1))
     W = synth.normal_f16((32, 64), 0.02, seed=2)
