@@ -63,8 +63,11 @@ unsigned long long mixdq_kernel_launches(void);
  * share a tile (tcgen05 cta_group::2), else 128 x {64, 96, 128, 256}.  The BOS-aware projection and the second branch
  * of a shortcut-split layer always run on 128-row tiles.  *reduction_splits (HOST): for 256-row tiles the number
  * of CTA pairs that share one tile's reduction (1: each pair walks whole tiles; 2 to 4: layers with few tiles and
- * a long reduction, partial sums added through distributed shared memory); 0 for 128-row tiles.  For tests and
- * benchmarks: nothing is launched. */
+ * a long reduction, partial sums added through distributed shared memory); 0 for 128-row tiles.  A linear layer for
+ * which mixdq_linear_fused_quant_tile is positive runs as one kernel on 128-row tiles of that width instead, and a
+ * shortcut-split layer (mixdq_linear_a8_split, mixdq_conv3x3_a8_split) takes the 256-row tiles reported for the sum of
+ * its branches' reduction blocks, without a split reduction, or else 128-row tiles.  For tests and benchmarks: nothing
+ * is launched. */
 int mixdq_int8_tile_plan(int64_t M, int64_t N, int64_t k_blocks, int w_bits, int* tile_rows, int* tile_cols,
                          int* reduction_splits);
 
